@@ -1,0 +1,300 @@
+#!/usr/bin/env python
+"""Benchmark of the top-2 MoE layer forward on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config c4_2048e] [--impl reference]
+
+One step = one forward pass of the whole layer (gating GEMM + softmax/top-2, capacity
+assignment, dispatch, expert FFN, combine) over one batch of seeded synthetic input shaped
+like the paper's MoE(2048E) layer.  Prints ONE JSON line:
+  value     tokens/s with every input resident in HBM (CUDA events, max over ranks)
+  e2e       tokens/s through gshard_moe_top2_forward_host: x, u copied from pinned host memory
+            and y, l_aux copied back inside the timed region (expert weights are model state
+            and stay on the device)
+  roofline  the dominant kernel (the grouped tcgen05 GEMM of the expert FFN): algorithmic bytes
+            (expert weights + dispatched inputs + expert outputs) / its measured duration, against
+            the measured HBM copy bandwidth
+  cpu_baseline  the CPU oracle timed on this machine's host cores on a bounded sample
+With --impl reference only the oracle runs (rank 0), on the same configuration.
+N > 1 runs N independent replicas (the path has no exchange step on one node): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "MoE layer tokens/sec at E=2048,M=1024,H=8192 (1 B200); % of layer roofline"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index = index
+        self.samples = []
+        self.stop_flag = threading.Event()
+
+    def run(self):
+        while not self.stop_flag.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                parts = [p.strip() for p in out.strip().split(",")]
+                if len(parts) >= 6:
+                    self.samples.append(parts)
+            except Exception:
+                pass
+            self.stop_flag.wait(0.1)
+
+    def summary(self):
+        sm = [float(s[0]) for s in self.samples if s[0].replace(".", "").isdigit()]
+        mx = [float(s[1]) for s in self.samples if s[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.samples)}
+
+
+def oracle_sample(cfg, n_tokens_ffn=24, seed_offset=0):
+    """Times the CPU oracle on a bounded sample of the configuration: gating + Algorithm 1 for one
+    whole group, eq. (2)-(3) for a few of its tokens.  Returns (tokens/s of a full layer at that
+    per-token cost, description, threads)."""
+    import numpy as np
+    import torch
+    from oracle import gshard_oracle as orc
+    from paper_2006_16668_b200.inputs import make_inputs
+
+    small = cfg.scaled(G=1)                                   # one group of the same S, M, E
+    inp = make_inputs(small, "cpu", with_experts=False)
+    x = inp["x"][0].float().numpy()
+    wg = inp["wg"].float().numpy()
+    u = inp["u"][0].numpy()
+    t0 = time.perf_counter()
+    _, p = orc.gates(x, wg)
+    m = orc.mean_gates(p)
+    e1, e2, g1, g2, _ = orc.top2(p)
+    r = orc.capacity(cfg.E, cfg.C, e1, e2, g1, g2, u, m)
+    t_gate = time.perf_counter() - t0
+    # expert FFN for a few tokens; weights of the needed experts drawn with the recipe's scales
+    gen = torch.Generator().manual_seed(cfg.seed + 99 + seed_offset)
+    rows = 0
+    t_ffn = 0.0
+    for s in range(min(n_tokens_ffn, cfg.S)):
+        for k in range(2):
+            if r.slot[s, k] < 0:
+                continue
+            wi_e = (torch.randn(cfg.M, cfg.H, generator=gen) * cfg.M ** -0.5).to(cfg.torch_dtype).float().numpy()
+            wo_e = (torch.randn(cfg.H, cfg.M, generator=gen) * cfg.H ** -0.5).to(cfg.torch_dtype).float().numpy()
+            t1 = time.perf_counter()
+            orc.ffn_rows(x[s:s + 1], wi_e, wo_e)
+            t_ffn += time.perf_counter() - t1
+            rows += 1
+    kept_per_token = float((r.slot >= 0).sum()) / cfg.S
+    per_token = t_gate / cfg.S + (t_ffn / max(rows, 1)) * kept_per_token
+    desc = (f"gating+Algorithm 1 for 1 group of {cfg.S} tokens ({t_gate:.2f} s) + eq.(2)-(3) for {rows} "
+            f"token-expert rows ({t_ffn:.2f} s); tokens/s extrapolated at {kept_per_token:.2f} kept choices/token")
+    return 1.0 / per_token, desc, orc.num_threads()
+
+
+def run_reference(args, cfg):
+    """The reference arm of this tier: the CPU oracle as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    desc, cores = "", 0
+    for i in range(args.warmup + args.steps):
+        v, desc, cores = oracle_sample(cfg, n_tokens_ffn=8, seed_offset=i)
+        if i >= args.warmup:
+            vals.append(v)
+    value = statistics.mean(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cfg.N / value,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": cfg.name, "G": cfg.G, "S": cfg.S, "M": cfg.M, "H": cfg.H,
+                                            "E": cfg.E, "C": cfg.C},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", default="c4_2048e")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    from paper_2006_16668_b200.inputs import CONFIGS, make_inputs
+    cfg = CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2006_16668_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl")
+    dev = torch.device("cuda", local_rank)
+    args.warmup = max(args.warmup, 3)
+
+    # ---- resident inputs --------------------------------------------------------------------
+    rcfg = cfg.scaled(seed=cfg.seed + rank)           # every replica draws its own batch
+    inp = make_inputs(rcfg, dev)
+    shape = B.make_shape(cfg)
+    ws = B.alloc_workspace(shape, host_staging=True, device=dev)
+    y = torch.empty_like(inp["x"])
+    l_aux = torch.zeros(1, dtype=torch.float32, device=dev)
+    rt, rs = B.alloc_routing(shape, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        B.gshard_moe_top2_forward(shape, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l_aux, rs,
+                                  None, ws, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    if B.gshard_moe_last_device_status(ws) != B.GSHARD_OK:
+        raise SystemExit("device status is not OK after warm-up")
+    launches_per_step = B.gshard_moe_last_launch_count()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    ev[0].record(stream)
+    for i in range(args.steps):
+        step()
+        ev[i + 1].record(stream)
+    barrier()
+    total_ms = ev[0].elapsed_time(ev[-1])
+    sampler.stop_flag.set()
+    sampler.join(timeout=2)
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * cfg.N / (ms_per_step * 1e-3)
+
+    # ---- dominant kernel: the expert FFN's grouped GEMM (two launches per step) -----------------
+    peaks = load_peaks()
+    buf = torch.empty(cfg.E, cfg.G * cfg.C, cfg.M, dtype=cfg.torch_dtype, device=dev)
+    B.gshard_moe_dispatch(shape, inp["x"], rt["slot_token"], buf, stream)
+    out = torch.empty_like(buf)
+    for _ in range(2):
+        B.gshard_moe_expert_ffn(shape, buf, inp["wi"], inp["wo"], out, ws, stream)
+    torch.cuda.synchronize()
+    k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    k0.record(stream)
+    for _ in range(args.steps):
+        B.gshard_moe_expert_ffn(shape, buf, inp["wi"], inp["wo"], out, ws, stream)
+    k1.record(stream)
+    torch.cuda.synchronize()
+    ffn_ms = k0.elapsed_time(k1) / args.steps
+    es = 2 if cfg.dtype == "bf16" else 4
+    R = cfg.E * cfg.G * cfg.C
+    ffn_bytes = 2 * cfg.E * cfg.M * cfg.H * es + 2 * R * cfg.M * es      # weights + buf in + out
+    ffn_flops = 4.0 * R * cfg.M * cfg.H
+    launch_ms = ffn_ms / 2.0                                             # two launches of the kernel
+    achieved = (ffn_bytes / 2.0) / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "kernel": "umma_gemm_kernel (expert FFN)",
+                "peak_source": peaks["source"], "launch_ms": launch_ms,
+                "ffn_tflops": ffn_flops / (ffn_ms * 1e-3) / 1e12}
+    # whole-layer roofline: slower of FLOPs at the tensor peak and bytes at the HBM peak
+    layer_flops = 2.0 * cfg.N * cfg.M * cfg.E + ffn_flops
+    layer_bytes = 2 * cfg.E * cfg.M * cfg.H * es + 2 * cfg.N * cfg.M * es + cfg.M * cfg.E * es + cfg.N * 4
+    t_roof = max(layer_flops / (peaks["bf16_tflops"] * 1e12), layer_bytes / (peaks["hbm_gbs"] * 1e9))
+    layer = {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_per_step, "flops": layer_flops,
+             "bytes": layer_bytes, "peak_source": peaks["source"]}
+
+    # ---- end to end through the host-buffer entry point -------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        xh = inp["x"].cpu().pin_memory()
+        uh = inp["u"].cpu().pin_memory()
+        yh = torch.empty_like(xh).pin_memory()
+        lh = torch.zeros(1, dtype=torch.float32).pin_memory()
+        for _ in range(2):
+            B.gshard_moe_top2_forward_host(shape, xh, inp["wg"], inp["wi"], inp["wo"], uh, yh, lh, None, ws, stream)
+        barrier()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        for _ in range(args.steps):
+            B.gshard_moe_top2_forward_host(shape, xh, inp["wg"], inp["wi"], inp["wo"], uh, yh, lh, None, ws, stream)
+        h1.record(stream)
+        barrier()
+        tt = torch.tensor([h0.elapsed_time(h1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item()) / args.steps
+        e2e = {"value": world * cfg.N / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": xh.numel() * xh.element_size() + uh.numel() * 4,
+               "d2h_bytes_per_step": yh.numel() * yh.element_size() + 4, "ms_per_step": e2e_ms,
+               "note": "expert and gating weights stay resident on the device (model state)"}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, desc, cores = oracle_sample(cfg)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+
+    if rank == 0:
+        stats = rt["stats"].cpu().tolist()
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+                "config": {"workload": cfg.name, "G": cfg.G, "S": cfg.S, "M": cfg.M, "H": cfg.H, "E": cfg.E,
+                           "C": cfg.C, "tokens_per_step_per_gpu": cfg.N, "parallelism": f"replicas x{world}",
+                           "l2": "inputs larger than L2 (expert weights are streamed once per step)",
+                           "slots_filled_frac": stats[4] / float(R)},
+                "roofline": roofline, "layer_roofline": layer, "cpu_baseline": cpu, "e2e": e2e,
+                "gpu_launches": launches_per_step * args.steps, "clocks": sampler.summary()}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

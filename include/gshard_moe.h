@@ -1,0 +1,182 @@
+/*
+ * gshard_moe.h - C ABI of the B200 (sm_100a) top-2 gated Mixture-of-Experts FFN layer.
+ *
+ * The layer is the one defined by the GShard paper (arxiv 2006.16668):
+ *   eq. (1)-(3)   y_s = sum_e G_{s,e} * FFN_e(x_s),  FFN_e(x) = wo_e . ReLU(wi_e . x), no bias
+ *   Algorithm 1   group-level top-2 gating: softmax gates, mean gates m_e, first-choice
+ *                 loop, auxiliary loss l_aux = (1/E) sum_e (c_e/S) m_e, second-choice loop
+ *                 with random routing (keep iff c < C and 2*g2 > rnd)
+ *   Algorithm 2   tensor layouts: inputs [G,S,M], wg [M,E], wi [E,M,H], wo [E,H,M],
+ *                 dispatched expert inputs [E,G,C,M], outputs [G,S,M]
+ *
+ * Conventions for every call
+ *   - All tensor arguments are DEVICE pointers unless the name ends in _host; tensors are
+ *     contiguous, row-major, 16-byte aligned, owned by the caller.  The library allocates no
+ *     device memory: scratch comes from the caller's `workspace`.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = default
+ *     stream) and the call returns without synchronising, except the *_host calls and
+ *     gshard_moe_last_device_status.
+ *   - Return value: a gshard_status.  Errors that the host can detect (null or misaligned
+ *     pointer, non-positive size, unsupported shape, short workspace, device that is not
+ *     sm_100) launch nothing.  Anomalies seen on the device (a bounded wait that ran out)
+ *     set a status word in the workspace, never trap, and are read back with
+ *     gshard_moe_last_device_status.
+ *   - dtype GSHARD_F32: x, wg, wi, wo, y (and dy, dx, dwi, dwo) are float; all arithmetic is
+ *     fp32 on CUDA cores.  dtype GSHARD_BF16: they are bfloat16; contractions run on the
+ *     tcgen05 tensor cores with fp32 accumulation; softmax, top-2, weights, l_aux are fp32.
+ *     u, l_aux, weight, m, dwg are always float.
+ *   - Outputs are bit-reproducible from run to run (no atomics in any reduction).
+ */
+#ifndef GSHARD_MOE_H_
+#define GSHARD_MOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GSHARD_OK = 0,
+  GSHARD_ERR_INVALID_ARG = 1,
+  GSHARD_ERR_UNSUPPORTED_SHAPE = 2,
+  GSHARD_ERR_WORKSPACE_TOO_SMALL = 3,
+  GSHARD_ERR_CUDA = 4,
+  GSHARD_ERR_ARCH = 5,
+  GSHARD_ERR_TIMEOUT = 6,
+  GSHARD_ERR_INTERNAL = 7
+} gshard_status;
+
+typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
+
+/* flags of gshard_moe_shape */
+#define GSHARD_FLAG_SAVE_FOR_BACKWARD 1u   /* forward fills `context` for the backward call */
+#define GSHARD_FLAG_SECOND_SKIP_FREES_SLOT 2u /* other reading of Algorithm 1's second loop: a
+                                                 token that fails 2*g2 > rnd does not advance
+                                                 the counter of its second expert */
+#define GSHARD_FLAG_SIMT_CONTRACTIONS 4u   /* bf16 only: run every contraction on CUDA cores
+                                              (fp32 FMA) instead of tcgen05; for debugging */
+
+/* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
+ * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,
+ * E >= 2, S < 65536, E <= 16384; dtype BF16 without SIMT flag also needs M % 64 == 0,
+ * H % 64 == 0, E % 16 == 0. */
+typedef struct {
+  int32_t G, S, M, H, E, C;
+  int32_t dtype;   /* gshard_dtype */
+  uint32_t flags;
+} gshard_moe_shape;
+
+/* Compact routing result (the non-zeros of Algorithm 2's combine_weights [G,S,E,C] and
+ * dispatch_mask).  Device pointers, caller-allocated; any may be NULL to skip that output. */
+typedef struct {
+  int32_t* expert_idx;   /* [G,S,2]  e1, e2 (Algorithm 1 top_2)                              */
+  int32_t* slot;         /* [G,S,2]  buffer position c in [0,C) or -1 when not dispatched     */
+  float* weight;         /* [G,S,2]  g1/(g1+g2), g2/(g1+g2) (normalised values, kept or not) */
+  uint8_t* flags;        /* [G,S]    bit0 first kept, bit1 2*g2>rnd passed, bit2 second kept  */
+  int32_t* first_count;  /* [G,E]    c_e after the first loop (unclipped; enters l_aux)       */
+  int32_t* total_count;  /* [G,E]    c_e after the second loop                                */
+  int32_t* slot_token;   /* [E,G,C]  token index s within the group, or -1 for an empty slot  */
+  float* m;              /* [G,E]    mean gates m_e                                           */
+  float* l_aux_group;    /* [G]      Algorithm 1's per-group l_aux                            */
+  int64_t* stats;        /* [8] 0 first choices dropped, 1 second choices that failed the
+                                random test, 2 second choices that passed but found no room,
+                                3 tokens with both choices dropped, 4 slots filled, 5..7 zero */
+} gshard_moe_routing;
+
+int gshard_version(void);
+const char* gshard_status_string(int status);
+
+/* Scratch sizes in bytes for a shape.  for_backward != 0 gives the size the backward call
+ * needs.  Returns 0 for an invalid or unsupported shape. */
+size_t gshard_moe_top2_workspace_bytes(const gshard_moe_shape* shape, int for_backward);
+/* Size of the saved-for-backward `context` buffer that the forward fills when
+ * GSHARD_FLAG_SAVE_FOR_BACKWARD is set. */
+size_t gshard_moe_top2_context_bytes(const gshard_moe_shape* shape);
+/* Extra workspace the *_host call needs for its device copies of x, u, y, l_aux. */
+size_t gshard_moe_top2_host_staging_bytes(const gshard_moe_shape* shape);
+
+/* The whole layer forward (Algorithm 2 with Algorithm 1 as Top2Gating), eq. (1)-(3).
+ *   x [G,S,M], wg [M,E], wi [E,M,H], wo [E,H,M]: dtype; u [G,S] float in [0,1): the `rnd`
+ *   of Algorithm 1, one per token (all zeros: every second choice passes the test).
+ *   y [G,S,M] dtype: layer output WITHOUT the residual connection; a token whose two
+ *   choices were both dropped gets zeros.  l_aux: one float, the mean over groups of
+ *   Algorithm 1's group loss.  routing_out: NULL or a struct of optional outputs.
+ *   context: NULL, or gshard_moe_top2_context_bytes() bytes when SAVE_FOR_BACKWARD is set.
+ *   workspace: at least gshard_moe_top2_workspace_bytes(shape, 0) bytes, 256-byte aligned;
+ *   its contents are scratch. */
+int gshard_moe_top2_forward(const gshard_moe_shape* shape, const void* x, const void* wg,
+                            const void* wi, const void* wo, const float* u, void* y,
+                            float* l_aux, const gshard_moe_routing* routing_out, void* context,
+                            void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* Same layer, activations on the HOST: x_host, u_host are read and y_host, l_aux_host are
+ * written in (preferably pinned) host memory; weights wg, wi, wo stay device pointers (they
+ * are model state, not a step's input).  Copies run on `cuda_stream` inside the call and the
+ * call synchronises the stream before returning.  workspace must hold
+ * gshard_moe_top2_workspace_bytes(shape,0) + gshard_moe_top2_host_staging_bytes(shape). */
+int gshard_moe_top2_forward_host(const gshard_moe_shape* shape, const void* x_host,
+                                 const void* wg, const void* wi, const void* wo,
+                                 const float* u_host, void* y_host, float* l_aux_host,
+                                 const gshard_moe_routing* routing_out, void* workspace,
+                                 size_t workspace_bytes, void* cuda_stream);
+
+/* Backward of L = <dy, y> + l_aux_weight * l_aux with the routing of the forward call held
+ * constant (the paper leaves the backward to automatic differentiation and states that the
+ * counts c_e are not differentiable; section 2.2, auxiliary-loss paragraph).
+ *   context: the buffer filled by the forward.  dy [G,S,M] dtype.
+ *   dx [G,S,M] dtype, dwg [M,E] float, dwi [E,M,H] dtype, dwo [E,H,M] dtype: overwritten. */
+int gshard_moe_top2_backward(const gshard_moe_shape* shape, const void* x, const void* wg,
+                             const void* wi, const void* wo, const void* context,
+                             const void* dy, float l_aux_weight, void* dx, float* dwg,
+                             void* dwi, void* dwo, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream);
+
+/* ---- the stages of the forward, callable on their own (same conventions) ---------------- */
+
+/* Algorithm 1, gates and top_2: logits = x . wg, softmax in fp32, two largest gates per
+ * token (lowest index wins ties), and the mean gates m_e.
+ *   expert_idx [G,S,2] int32, gate12 [G,S,2] float (raw softmax values g1, g2), m [G,E] float.
+ *   workspace: gshard_moe_top2_workspace_bytes(shape, 0). */
+int gshard_moe_gate(const gshard_moe_shape* shape, const void* x, const void* wg,
+                    int32_t* expert_idx, float* gate12, float* m, void* workspace,
+                    size_t workspace_bytes, void* cuda_stream);
+
+/* Algorithm 1, the two token loops and l_aux, for all groups: positions are the stable rank of
+ * a token among the tokens of its group that chose the same expert (first choices before
+ * second choices).  Inputs expert_idx, gate12, u, m as produced by gshard_moe_gate.
+ * routing_out->expert_idx and ->m are ignored; l_aux may be NULL.
+ * workspace: gshard_moe_top2_workspace_bytes(shape, 0). */
+int gshard_moe_capacity(const gshard_moe_shape* shape, const int32_t* expert_idx,
+                        const float* gate12, const float* u, const float* m,
+                        const gshard_moe_routing* routing_out, float* l_aux, void* workspace,
+                        size_t workspace_bytes, void* cuda_stream);
+
+/* Algorithm 2 dispatch as an index gather: buf[e, g*C+c, :] = x[g, slot_token[e,g,c], :],
+ * zero row for an empty slot.  buf [E, G*C, M] dtype. */
+int gshard_moe_dispatch(const gshard_moe_shape* shape, const void* x, const int32_t* slot_token,
+                        void* buf, void* cuda_stream);
+
+/* Eq. (2) for every expert: out[e] = relu(buf[e] . wi[e]) . wo[e]; buf, out [E, G*C, M] dtype.
+ * workspace holds the hidden activations (gshard_moe_top2_workspace_bytes(shape, 0)). */
+int gshard_moe_expert_ffn(const gshard_moe_shape* shape, const void* buf, const void* wi,
+                          const void* wo, void* out, void* workspace, size_t workspace_bytes,
+                          void* cuda_stream);
+
+/* Eq. (3) / Algorithm 2 combine as a per-token gather:
+ * y[g,s,:] = sum over k in {0,1} with slot[g,s,k] >= 0 of weight[g,s,k] * out[e_k, g*C+slot, :]. */
+int gshard_moe_combine(const gshard_moe_shape* shape, const void* out, const int32_t* expert_idx,
+                       const int32_t* slot, const float* weight, void* y, void* cuda_stream);
+
+/* Synchronises `cuda_stream` and returns the device status word of `workspace`
+ * (GSHARD_OK, GSHARD_ERR_TIMEOUT, ...) or GSHARD_ERR_CUDA if the stream reported an error. */
+int gshard_moe_last_device_status(void* workspace, void* cuda_stream);
+
+/* Number of kernels the last forward/backward/stage call on this thread launched. */
+int gshard_moe_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GSHARD_MOE_H_ */

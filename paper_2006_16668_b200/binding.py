@@ -1,0 +1,228 @@
+"""Thin ctypes binding of ``include/gshard_moe.h``: same names, argument marshalling only.
+
+torch tensors supply device memory and the current stream; every step of the layer runs
+inside the CUDA library.  If the library has not been built the first call raises - there
+is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, c_float, c_int, c_int32, c_size_t, c_uint32, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgshard_moe.so")
+
+GSHARD_OK = 0
+GSHARD_ERR_INVALID_ARG = 1
+GSHARD_ERR_UNSUPPORTED_SHAPE = 2
+GSHARD_ERR_WORKSPACE_TOO_SMALL = 3
+GSHARD_ERR_CUDA = 4
+GSHARD_ERR_ARCH = 5
+GSHARD_ERR_TIMEOUT = 6
+GSHARD_ERR_INTERNAL = 7
+GSHARD_F32 = 0
+GSHARD_BF16 = 1
+GSHARD_FLAG_SAVE_FOR_BACKWARD = 1
+GSHARD_FLAG_SECOND_SKIP_FREES_SLOT = 2
+GSHARD_FLAG_SIMT_CONTRACTIONS = 4
+
+
+class gshard_moe_shape(Structure):
+    _fields_ = [("G", c_int32), ("S", c_int32), ("M", c_int32), ("H", c_int32), ("E", c_int32),
+                ("C", c_int32), ("dtype", c_int32), ("flags", c_uint32)]
+
+
+class gshard_moe_routing(Structure):
+    _fields_ = [(n, c_void_p) for n in ("expert_idx", "slot", "weight", "flags", "first_count",
+                                        "total_count", "slot_token", "m", "l_aux_group", "stats")]
+
+
+EXPORTS = {
+    # name: (restype, argtypes)
+    "gshard_version": (c_int, []),
+    "gshard_status_string": (ctypes.c_char_p, [c_int]),
+    "gshard_moe_top2_workspace_bytes": (c_size_t, [POINTER(gshard_moe_shape), c_int]),
+    "gshard_moe_top2_context_bytes": (c_size_t, [POINTER(gshard_moe_shape)]),
+    "gshard_moe_top2_host_staging_bytes": (c_size_t, [POINTER(gshard_moe_shape)]),
+    "gshard_moe_top2_forward": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 7 +
+                                [POINTER(gshard_moe_routing), c_void_p, c_void_p, c_size_t, c_void_p]),
+    "gshard_moe_top2_forward_host": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 7 +
+                                     [POINTER(gshard_moe_routing), c_void_p, c_size_t, c_void_p]),
+    "gshard_moe_top2_backward": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6 + [c_float] +
+                                 [c_void_p] * 5 + [c_size_t, c_void_p]),
+    "gshard_moe_gate": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6 + [c_size_t, c_void_p]),
+    "gshard_moe_capacity": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 4 +
+                            [POINTER(gshard_moe_routing), c_void_p, c_void_p, c_size_t, c_void_p]),
+    "gshard_moe_dispatch": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 4),
+    "gshard_moe_expert_ffn": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 5 + [c_size_t, c_void_p]),
+    "gshard_moe_combine": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6),
+    "gshard_moe_last_device_status": (c_int, [c_void_p, c_void_p]),
+    "gshard_moe_last_launch_count": (c_int, []),
+}
+
+_lib = None
+
+
+def load():
+    """Load the CUDA library; raises if it is missing (build it with __graft_entry__.build())."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build the CUDA library first "
+                "(python -c 'import __graft_entry__ as g; g.build()'); there is no fallback path")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in EXPORTS.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+class GshardError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+def _check(code: int, where: str):
+    if code != GSHARD_OK:
+        raise GshardError(code, where)
+
+
+def status_string(code: int) -> str:
+    return load().gshard_status_string(int(code)).decode()
+
+
+def make_shape(cfg=None, *, G=None, S=None, M=None, H=None, E=None, C=None, dtype=None, flags=0) -> gshard_moe_shape:
+    """Shape struct from a MoEConfig or explicit sizes; dtype is "f32" | "bf16"."""
+    if cfg is not None:
+        G, S, M, H, E, C = cfg.G, cfg.S, cfg.M, cfg.H, cfg.E, cfg.C
+        dtype = cfg.dtype if dtype is None else dtype
+    code = {"f32": GSHARD_F32, "bf16": GSHARD_BF16}[dtype]
+    return gshard_moe_shape(G, S, M, H, E, C, code, flags)
+
+
+def _p(t):
+    """Device/host pointer of a tensor (or None)."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+def _stream(stream=None):
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def alloc_routing(shape: gshard_moe_shape, device="cuda"):
+    """Allocate every optional routing output; returns (dict of tensors, struct)."""
+    G, S, E, C = shape.G, shape.S, shape.E, shape.C
+    t = {
+        "expert_idx": torch.empty(G, S, 2, dtype=torch.int32, device=device),
+        "slot": torch.empty(G, S, 2, dtype=torch.int32, device=device),
+        "weight": torch.empty(G, S, 2, dtype=torch.float32, device=device),
+        "flags": torch.empty(G, S, dtype=torch.uint8, device=device),
+        "first_count": torch.empty(G, E, dtype=torch.int32, device=device),
+        "total_count": torch.empty(G, E, dtype=torch.int32, device=device),
+        "slot_token": torch.empty(E, G, C, dtype=torch.int32, device=device),
+        "m": torch.empty(G, E, dtype=torch.float32, device=device),
+        "l_aux_group": torch.empty(G, dtype=torch.float32, device=device),
+        "stats": torch.zeros(8, dtype=torch.int64, device=device),
+    }
+    return t, routing_struct(t)
+
+
+def routing_struct(tensors: dict) -> gshard_moe_routing:
+    r = gshard_moe_routing()
+    for name, _ in gshard_moe_routing._fields_:
+        setattr(r, name, _p(tensors.get(name)))
+    return r
+
+
+def gshard_moe_top2_workspace_bytes(shape, for_backward=False) -> int:
+    return int(load().gshard_moe_top2_workspace_bytes(ctypes.byref(shape), int(bool(for_backward))))
+
+
+def gshard_moe_top2_context_bytes(shape) -> int:
+    return int(load().gshard_moe_top2_context_bytes(ctypes.byref(shape)))
+
+
+def gshard_moe_top2_host_staging_bytes(shape) -> int:
+    return int(load().gshard_moe_top2_host_staging_bytes(ctypes.byref(shape)))
+
+
+def alloc_workspace(shape, for_backward=False, host_staging=False, device="cuda") -> torch.Tensor:
+    n = gshard_moe_top2_workspace_bytes(shape, for_backward)
+    if n == 0:
+        raise GshardError(GSHARD_ERR_UNSUPPORTED_SHAPE, "workspace_bytes")
+    if host_staging:
+        n += gshard_moe_top2_host_staging_bytes(shape)
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def gshard_moe_top2_forward(shape, x, wg, wi, wo, u, y, l_aux, routing_out=None, context=None,
+                            workspace=None, stream=None):
+    rp = ctypes.byref(routing_out) if routing_out is not None else None
+    _check(load().gshard_moe_top2_forward(ctypes.byref(shape), _p(x), _p(wg), _p(wi), _p(wo), _p(u), _p(y),
+                                          _p(l_aux), rp, _p(context), _p(workspace), workspace.numel(),
+                                          _stream(stream)), "gshard_moe_top2_forward")
+
+
+def gshard_moe_top2_forward_host(shape, x_host, wg, wi, wo, u_host, y_host, l_aux_host, routing_out=None,
+                                 workspace=None, stream=None):
+    rp = ctypes.byref(routing_out) if routing_out is not None else None
+    _check(load().gshard_moe_top2_forward_host(ctypes.byref(shape), _p(x_host), _p(wg), _p(wi), _p(wo),
+                                               _p(u_host), _p(y_host), _p(l_aux_host), rp, _p(workspace),
+                                               workspace.numel(), _stream(stream)),
+           "gshard_moe_top2_forward_host")
+
+
+def gshard_moe_top2_backward(shape, x, wg, wi, wo, context, dy, l_aux_weight, dx, dwg, dwi, dwo,
+                             workspace=None, stream=None):
+    _check(load().gshard_moe_top2_backward(ctypes.byref(shape), _p(x), _p(wg), _p(wi), _p(wo), _p(context),
+                                           _p(dy), float(l_aux_weight), _p(dx), _p(dwg), _p(dwi), _p(dwo),
+                                           _p(workspace), workspace.numel(), _stream(stream)),
+           "gshard_moe_top2_backward")
+
+
+def gshard_moe_gate(shape, x, wg, expert_idx, gate12, m, workspace, stream=None):
+    _check(load().gshard_moe_gate(ctypes.byref(shape), _p(x), _p(wg), _p(expert_idx), _p(gate12), _p(m),
+                                  _p(workspace), workspace.numel(), _stream(stream)), "gshard_moe_gate")
+
+
+def gshard_moe_capacity(shape, expert_idx, gate12, u, m, routing_out, l_aux, workspace, stream=None):
+    _check(load().gshard_moe_capacity(ctypes.byref(shape), _p(expert_idx), _p(gate12), _p(u), _p(m),
+                                      ctypes.byref(routing_out), _p(l_aux), _p(workspace), workspace.numel(),
+                                      _stream(stream)), "gshard_moe_capacity")
+
+
+def gshard_moe_dispatch(shape, x, slot_token, buf, stream=None):
+    _check(load().gshard_moe_dispatch(ctypes.byref(shape), _p(x), _p(slot_token), _p(buf), _stream(stream)),
+           "gshard_moe_dispatch")
+
+
+def gshard_moe_expert_ffn(shape, buf, wi, wo, out, workspace, stream=None):
+    _check(load().gshard_moe_expert_ffn(ctypes.byref(shape), _p(buf), _p(wi), _p(wo), _p(out), _p(workspace),
+                                        workspace.numel(), _stream(stream)), "gshard_moe_expert_ffn")
+
+
+def gshard_moe_combine(shape, out, expert_idx, slot, weight, y, stream=None):
+    _check(load().gshard_moe_combine(ctypes.byref(shape), _p(out), _p(expert_idx), _p(slot), _p(weight), _p(y),
+                                     _stream(stream)), "gshard_moe_combine")
+
+
+def gshard_moe_last_device_status(workspace, stream=None) -> int:
+    return int(load().gshard_moe_last_device_status(_p(workspace), _stream(stream)))
+
+
+def gshard_moe_last_launch_count() -> int:
+    return int(load().gshard_moe_last_launch_count())

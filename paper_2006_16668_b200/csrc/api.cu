@@ -1,0 +1,347 @@
+// C-ABI layer: argument validation, workspace planning and the launch sequences of the forward
+// pass and its stages.  Declarations and semantics: include/gshard_moe.h.
+#include <cstring>
+
+#include "kernels.cuh"
+#include "gemm_dispatch.cuh"
+#include "plan.cuh"
+
+namespace gshard {
+
+LaunchCounter& launch_counter() {
+  static thread_local LaunchCounter c;
+  return c;
+}
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_device() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return GSHARD_ERR_CUDA; }
+  int major = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return GSHARD_ERR_CUDA;
+  return major == 10 ? GSHARD_OK : GSHARD_ERR_ARCH;
+}
+
+#define GS_REQUIRE_PTR(p)                                          \
+  do {                                                             \
+    if ((p) == nullptr || !aligned16(p)) return GSHARD_ERR_INVALID_ARG; \
+  } while (0)
+#define GS_TRY(expr)                       \
+  do {                                     \
+    const int _rc = (expr);                \
+    if (_rc != GSHARD_OK) return _rc;      \
+  } while (0)
+
+}  // namespace
+
+// logits[N,E] = x[N,M] . wg[M,E], fp32 out.
+int gate_logits(const Dims& d, const void* x, const void* wg, float* logits, int* status, cudaStream_t st) {
+  UmmaGemm g{};
+  g.A = x; g.B = wg; g.C = logits;
+  g.rows = (int)d.N; g.cols = d.E; g.K = d.M; g.batch = 1;
+  g.a_kmajor = true; g.b_kmajor = false;
+  g.a_ld = d.M; g.b_ld = d.E; g.c_ld = d.E;
+  g.out_f32 = 1; g.a_stream = 1;
+  return run_gemm(d, g, status, st);
+}
+
+namespace {
+
+int gate_stage(const Dims& d, const FwdPlan& pl, unsigned char* ws, const void* x, const void* wg,
+               int32_t* expert_idx, float* gate12, float* m, float* rowmax, float* rowinv, cudaStream_t st) {
+  float* logits = reinterpret_cast<float*>(ws + pl.logits);
+  GS_TRY(gate_logits(d, x, wg, logits, reinterpret_cast<int*>(ws + pl.status), st));
+  launch_gate_rows(d, logits, expert_idx, gate12, rowmax, rowinv, reinterpret_cast<float*>(ws + pl.partial), m, st);
+  return GSHARD_OK;
+}
+
+// h = relu(buf . wi), out = h . wo for every expert (eq. (2)); weights are read once.
+int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, void* out, int* status,
+              cudaStream_t st) {
+  const long long rows = d.rows;
+  UmmaGemm g{};
+  g.A = buf; g.B = wi; g.C = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;
+  g.a_kmajor = true; g.b_kmajor = false;
+  g.a_ld = d.M; g.a_bs = rows * d.M; g.b_ld = d.H; g.b_bs = (long long)d.M * d.H; g.c_ld = d.H; g.c_bs = rows * d.H;
+  g.relu = 1; g.b_stream = 1;
+  GS_TRY(run_gemm(d, g, status, st));
+  UmmaGemm g2{};
+  g2.A = h; g2.B = wo; g2.C = out; g2.rows = d.rows; g2.cols = d.M; g2.K = d.H; g2.batch = d.E;
+  g2.a_kmajor = true; g2.b_kmajor = false;
+  g2.a_ld = d.H; g2.a_bs = rows * d.H; g2.b_ld = d.M; g2.b_bs = (long long)d.H * d.M; g2.c_ld = d.M; g2.c_bs = rows * d.M;
+  g2.b_stream = 1;
+  return run_gemm(d, g2, status, st);
+}
+
+template <typename T> T* pick(T* user, unsigned char* ws, size_t off) {
+  return user ? user : reinterpret_cast<T*>(ws + off);
+}
+
+}  // namespace
+
+int validate_shape(const gshard_moe_shape* s) {
+  if (!s) return GSHARD_ERR_INVALID_ARG;
+  if (s->G <= 0 || s->S <= 0 || s->M <= 0 || s->H <= 0 || s->E <= 0 || s->C <= 0) return GSHARD_ERR_INVALID_ARG;
+  if (s->dtype != GSHARD_F32 && s->dtype != GSHARD_BF16) return GSHARD_ERR_INVALID_ARG;
+  if (s->flags & ~7u) return GSHARD_ERR_INVALID_ARG;
+  if (s->E < 2) return GSHARD_ERR_INVALID_ARG;
+  if (s->M % 8 || s->H % 8) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  if (s->S > 32767 || s->E > 16384 || s->C > 32767) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)s->G * s->S > (1ll << 30) || (long long)s->E * s->G * s->C > (1ll << 30)) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  if (capacity_warps_for(s->E) == 0) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  const bool umma = s->dtype == GSHARD_BF16 && !(s->flags & GSHARD_FLAG_SIMT_CONTRACTIONS);
+  if (umma && (s->M % 64 || s->H % 64 || s->E % 16)) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  return GSHARD_OK;
+}
+
+// The forward launch sequence on device buffers.
+int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg, const void* wi, const void* wo,
+                   const float* u, void* y, float* l_aux, const gshard_moe_routing* ro, void* context,
+                   void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  const Dims d = make_dims(*shape);
+  const FwdPlan pl = plan_forward(d);
+  if (workspace_bytes < pl.total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  const bool save = (shape->flags & GSHARD_FLAG_SAVE_FOR_BACKWARD) != 0;
+  if (save && !context) return GSHARD_ERR_INVALID_ARG;
+  unsigned char* ctx = static_cast<unsigned char*>(context);
+  const CtxPlan cp = plan_context(d);
+  gshard_moe_routing r{};
+  if (ro) r = *ro;
+  int* status = reinterpret_cast<int*>(ws + pl.status);
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+
+  // with SAVE_FOR_BACKWARD the small routing tensors and the big activations live in the context
+  int32_t* expert_idx = save ? reinterpret_cast<int32_t*>(ctx + cp.expert_idx) : pick(r.expert_idx, ws, pl.expert_idx);
+  int32_t* slot = save ? reinterpret_cast<int32_t*>(ctx + cp.slot) : pick(r.slot, ws, pl.slot);
+  float* weight = save ? reinterpret_cast<float*>(ctx + cp.weight) : pick(r.weight, ws, pl.weight);
+  int32_t* first_count = save ? reinterpret_cast<int32_t*>(ctx + cp.first_count) : pick(r.first_count, ws, pl.first_count);
+  int32_t* slot_token = save ? reinterpret_cast<int32_t*>(ctx + cp.slot_token) : pick(r.slot_token, ws, pl.slot_token);
+  float* gate12 = save ? reinterpret_cast<float*>(ctx + cp.gate12) : reinterpret_cast<float*>(ws + pl.gate12);
+  float* rowmax = save ? reinterpret_cast<float*>(ctx + cp.rowmax) : reinterpret_cast<float*>(ws + pl.rowmax);
+  float* rowinv = save ? reinterpret_cast<float*>(ctx + cp.rowinv) : reinterpret_cast<float*>(ws + pl.rowinv);
+  void* h = save ? static_cast<void*>(ctx + cp.h) : static_cast<void*>(ws + pl.h);
+  void* out = save ? static_cast<void*>(ctx + cp.out) : static_cast<void*>(ws + pl.out);
+  uint8_t* flags = pick(r.flags, ws, pl.flags);
+  int32_t* total_count = pick(r.total_count, ws, pl.total_count);
+  float* m = pick(r.m, ws, pl.m);
+  float* l_aux_group = pick(r.l_aux_group, ws, pl.l_aux_group);
+  int32_t* stats_group = reinterpret_cast<int32_t*>(ws + pl.stats_group);
+  void* buf = ws + pl.buf;
+
+  GS_TRY(gate_stage(d, pl, ws, x, wg, expert_idx, gate12, m, rowmax, rowinv, st));
+  GS_TRY(launch_capacity(d, expert_idx, gate12, u, m, slot, weight, flags, first_count, total_count, slot_token,
+                         l_aux_group, stats_group, l_aux, reinterpret_cast<long long*>(r.stats), st));
+  launch_dispatch(d, x, slot_token, buf, st);
+  GS_TRY(ffn_stage(d, buf, wi, wo, h, out, status, st));
+  launch_combine(d, out, expert_idx, slot, weight, y, st);
+
+  if (save) {   // hand the caller the routing tensors it asked for
+    struct { void* dst; const void* src; size_t n; } cps[] = {
+        {r.expert_idx, expert_idx, (size_t)d.N * 2 * 4}, {r.slot, slot, (size_t)d.N * 2 * 4},
+        {r.weight, weight, (size_t)d.N * 2 * 4},         {r.first_count, first_count, (size_t)d.G * d.E * 4},
+        {r.slot_token, slot_token, (size_t)d.R * 4}};
+    for (auto& c : cps)
+      if (c.dst && cudaMemcpyAsync(c.dst, c.src, c.n, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  }
+  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+int backward_device(const gshard_moe_shape* shape, const void* x, const void* wg, const void* wi, const void* wo,
+                    const void* context, const void* dy, float k_aux, void* dx, float* dwg, void* dwi, void* dwo,
+                    void* workspace, size_t workspace_bytes, cudaStream_t st);
+
+}  // namespace gshard
+
+using namespace gshard;
+
+extern "C" {
+
+int gshard_version(void) { return 100; }
+
+const char* gshard_status_string(int s) {
+  switch (s) {
+    case GSHARD_OK: return "ok";
+    case GSHARD_ERR_INVALID_ARG: return "invalid argument";
+    case GSHARD_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case GSHARD_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case GSHARD_ERR_CUDA: return "CUDA error";
+    case GSHARD_ERR_ARCH: return "device is not sm_100";
+    case GSHARD_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case GSHARD_ERR_INTERNAL: return "internal error";
+    default: return "unknown status";
+  }
+}
+
+size_t gshard_moe_top2_workspace_bytes(const gshard_moe_shape* shape, int for_backward) {
+  if (validate_shape(shape) != GSHARD_OK) return 0;
+  const Dims d = make_dims(*shape);
+  return for_backward ? plan_backward(d).total : plan_forward(d).total;
+}
+
+size_t gshard_moe_top2_context_bytes(const gshard_moe_shape* shape) {
+  if (validate_shape(shape) != GSHARD_OK) return 0;
+  return plan_context(make_dims(*shape)).total;
+}
+
+size_t gshard_moe_top2_host_staging_bytes(const gshard_moe_shape* shape) {
+  if (validate_shape(shape) != GSHARD_OK) return 0;
+  return plan_staging(make_dims(*shape)).total;
+}
+
+int gshard_moe_top2_forward(const gshard_moe_shape* shape, const void* x, const void* wg, const void* wi,
+                            const void* wo, const float* u, void* y, float* l_aux,
+                            const gshard_moe_routing* routing_out, void* context, void* workspace,
+                            size_t workspace_bytes, void* cuda_stream) {
+  launch_counter().n = 0;
+  GS_TRY(validate_shape(shape));
+  GS_REQUIRE_PTR(x); GS_REQUIRE_PTR(wg); GS_REQUIRE_PTR(wi); GS_REQUIRE_PTR(wo); GS_REQUIRE_PTR(u);
+  GS_REQUIRE_PTR(y); GS_REQUIRE_PTR(workspace);
+  if (l_aux == nullptr) return GSHARD_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  if (workspace_bytes < gshard_moe_top2_workspace_bytes(shape, 0)) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  GS_TRY(check_device());
+  return forward_device(shape, x, wg, wi, wo, u, y, l_aux, routing_out, context, workspace, workspace_bytes,
+                        static_cast<cudaStream_t>(cuda_stream));
+}
+
+int gshard_moe_top2_forward_host(const gshard_moe_shape* shape, const void* x_host, const void* wg, const void* wi,
+                                 const void* wo, const float* u_host, void* y_host, float* l_aux_host,
+                                 const gshard_moe_routing* routing_out, void* workspace, size_t workspace_bytes,
+                                 void* cuda_stream) {
+  launch_counter().n = 0;
+  GS_TRY(validate_shape(shape));
+  if (!x_host || !u_host || !y_host || !l_aux_host) return GSHARD_ERR_INVALID_ARG;
+  GS_REQUIRE_PTR(wg); GS_REQUIRE_PTR(wi); GS_REQUIRE_PTR(wo); GS_REQUIRE_PTR(workspace);
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  if (shape->flags & GSHARD_FLAG_SAVE_FOR_BACKWARD) return GSHARD_ERR_INVALID_ARG;
+  const Dims d = make_dims(*shape);
+  const size_t fwd = plan_forward(d).total;
+  const StagePlan sp = plan_staging(d);
+  if (workspace_bytes < fwd + sp.total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  GS_TRY(check_device());
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* stg = static_cast<unsigned char*>(workspace) + fwd;
+  void* xd = stg + sp.x; float* ud = reinterpret_cast<float*>(stg + sp.u);
+  void* yd = stg + sp.y; float* ld = reinterpret_cast<float*>(stg + sp.l_aux);
+  const size_t act_bytes = (size_t)d.N * d.M * d.esize;
+  if (cudaMemcpyAsync(xd, x_host, act_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  if (cudaMemcpyAsync(ud, u_host, (size_t)d.N * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  GS_TRY(forward_device(shape, xd, wg, wi, wo, ud, yd, ld, routing_out, nullptr, workspace, fwd, st));
+  if (cudaMemcpyAsync(y_host, yd, act_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  if (cudaMemcpyAsync(l_aux_host, ld, 4, cudaMemcpyDeviceToHost, st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  int status = 0;
+  if (cudaMemcpy(&status, workspace, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return GSHARD_ERR_CUDA;
+  return status;
+}
+
+int gshard_moe_top2_backward(const gshard_moe_shape* shape, const void* x, const void* wg, const void* wi,
+                             const void* wo, const void* context, const void* dy, float l_aux_weight, void* dx,
+                             float* dwg, void* dwi, void* dwo, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream) {
+  launch_counter().n = 0;
+  GS_TRY(validate_shape(shape));
+  GS_REQUIRE_PTR(x); GS_REQUIRE_PTR(wg); GS_REQUIRE_PTR(wi); GS_REQUIRE_PTR(wo); GS_REQUIRE_PTR(context);
+  GS_REQUIRE_PTR(dy); GS_REQUIRE_PTR(dx); GS_REQUIRE_PTR(dwg); GS_REQUIRE_PTR(dwi); GS_REQUIRE_PTR(dwo);
+  GS_REQUIRE_PTR(workspace);
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  if (workspace_bytes < gshard_moe_top2_workspace_bytes(shape, 1)) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  GS_TRY(check_device());
+  return backward_device(shape, x, wg, wi, wo, context, dy, l_aux_weight, dx, dwg, dwi, dwo, workspace,
+                         workspace_bytes, static_cast<cudaStream_t>(cuda_stream));
+}
+
+int gshard_moe_gate(const gshard_moe_shape* shape, const void* x, const void* wg, int32_t* expert_idx,
+                    float* gate12, float* m, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  launch_counter().n = 0;
+  GS_TRY(validate_shape(shape));
+  GS_REQUIRE_PTR(x); GS_REQUIRE_PTR(wg); GS_REQUIRE_PTR(expert_idx); GS_REQUIRE_PTR(gate12); GS_REQUIRE_PTR(m);
+  GS_REQUIRE_PTR(workspace);
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  const Dims d = make_dims(*shape);
+  const FwdPlan pl = plan_forward(d);
+  if (workspace_bytes < pl.total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  GS_TRY(check_device());
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  if (cudaMemsetAsync(ws + pl.status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  GS_TRY(gate_stage(d, pl, ws, x, wg, expert_idx, gate12, m, reinterpret_cast<float*>(ws + pl.rowmax),
+                    reinterpret_cast<float*>(ws + pl.rowinv), st));
+  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+int gshard_moe_capacity(const gshard_moe_shape* shape, const int32_t* expert_idx, const float* gate12,
+                        const float* u, const float* m, const gshard_moe_routing* ro, float* l_aux,
+                        void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  launch_counter().n = 0;
+  GS_TRY(validate_shape(shape));
+  GS_REQUIRE_PTR(expert_idx); GS_REQUIRE_PTR(gate12); GS_REQUIRE_PTR(u); GS_REQUIRE_PTR(m);
+  GS_REQUIRE_PTR(workspace);
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  const Dims d = make_dims(*shape);
+  const FwdPlan pl = plan_forward(d);
+  if (workspace_bytes < pl.total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  GS_TRY(check_device());
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  gshard_moe_routing r{};
+  if (ro) r = *ro;
+  return launch_capacity(d, expert_idx, gate12, u, m, pick(r.slot, ws, pl.slot), pick(r.weight, ws, pl.weight),
+                         pick(r.flags, ws, pl.flags), pick(r.first_count, ws, pl.first_count),
+                         pick(r.total_count, ws, pl.total_count), pick(r.slot_token, ws, pl.slot_token),
+                         pick(r.l_aux_group, ws, pl.l_aux_group), reinterpret_cast<int32_t*>(ws + pl.stats_group),
+                         l_aux, reinterpret_cast<long long*>(r.stats), static_cast<cudaStream_t>(cuda_stream));
+}
+
+int gshard_moe_dispatch(const gshard_moe_shape* shape, const void* x, const int32_t* slot_token, void* buf,
+                        void* cuda_stream) {
+  launch_counter().n = 0;
+  GS_TRY(validate_shape(shape));
+  GS_REQUIRE_PTR(x); GS_REQUIRE_PTR(slot_token); GS_REQUIRE_PTR(buf);
+  GS_TRY(check_device());
+  launch_dispatch(make_dims(*shape), x, slot_token, buf, static_cast<cudaStream_t>(cuda_stream));
+  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+int gshard_moe_expert_ffn(const gshard_moe_shape* shape, const void* buf, const void* wi, const void* wo,
+                          void* out, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  launch_counter().n = 0;
+  GS_TRY(validate_shape(shape));
+  GS_REQUIRE_PTR(buf); GS_REQUIRE_PTR(wi); GS_REQUIRE_PTR(wo); GS_REQUIRE_PTR(out); GS_REQUIRE_PTR(workspace);
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  const Dims d = make_dims(*shape);
+  const FwdPlan pl = plan_forward(d);
+  if (workspace_bytes < pl.total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  GS_TRY(check_device());
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  if (cudaMemsetAsync(ws + pl.status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  GS_TRY(ffn_stage(d, buf, wi, wo, ws + pl.h, out, reinterpret_cast<int*>(ws + pl.status), st));
+  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+int gshard_moe_combine(const gshard_moe_shape* shape, const void* out, const int32_t* expert_idx,
+                       const int32_t* slot, const float* weight, void* y, void* cuda_stream) {
+  launch_counter().n = 0;
+  GS_TRY(validate_shape(shape));
+  GS_REQUIRE_PTR(out); GS_REQUIRE_PTR(expert_idx); GS_REQUIRE_PTR(slot); GS_REQUIRE_PTR(weight); GS_REQUIRE_PTR(y);
+  GS_TRY(check_device());
+  launch_combine(make_dims(*shape), out, expert_idx, slot, weight, y, static_cast<cudaStream_t>(cuda_stream));
+  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+int gshard_moe_last_device_status(void* workspace, void* cuda_stream) {
+  if (!workspace) return GSHARD_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  int status = 0;
+  if (cudaMemcpy(&status, workspace, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return GSHARD_ERR_CUDA;
+  return status;
+}
+
+int gshard_moe_last_launch_count(void) { return launch_counter().n; }
+
+}  // extern "C"

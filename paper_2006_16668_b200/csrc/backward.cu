@@ -1,0 +1,312 @@
+// Backward of L = <dy, y> + k * l_aux with the routing frozen.  The paper leaves the backward
+// to automatic differentiation; these are the derivatives of eq. (1)-(3) and of Algorithm 1's
+// combine weights and auxiliary loss, with the counts c_e constant (the paper states they are
+// not differentiable).  Per token with raw gates a = g_{e1}, b = g_{e2}, D = a + b:
+//   y = k1 (a/D) o1 + k2 (b/D) o2,  dw1 = k1 <dy,o1>,  dw2 = k2 <dy,o2>
+//   dL/da = (b/D^2)(dw1 - dw2),  dL/db = (a/D^2)(dw2 - dw1)
+//   dL/dg_{g,s,e} += k (1/G)(1/E)(c_{g,e}/S)(1/S)                      (dense, from l_aux)
+//   dlogit = g * (dg - <g, dg>),  dwg = x^T dlogit,  dx += dlogit wg^T
+//   expert path: dout[slot] = w dy,  dh = (dout wo^T) * 1[h > 0],  dwo = h^T dout,
+//                dwi = buf^T dh,  dbuf = dh wi^T,  dx += dbuf[slot]
+#include "gemm_dispatch.cuh"
+#include "plan.cuh"
+
+namespace gshard {
+
+int gate_logits(const Dims& d, const void* x, const void* wg, float* logits, int* status, cudaStream_t st);
+
+namespace {
+
+template <typename T> struct Row16;
+template <> struct Row16<float> {
+  static constexpr int n = 4;
+  __device__ static void load(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
+  __device__ static uint4 store(const float* f) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+  }
+};
+template <> struct Row16<__nv_bfloat16> {
+  static constexpr int n = 8;
+  __device__ static void load(const uint4& v, float* f) {
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+  }
+  __device__ static uint4 store(const float* f) {
+    unsigned w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+      w[i] = *reinterpret_cast<const unsigned*>(&p);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+  }
+};
+
+// dw[t,k] = <dy[t,:], out[e_k, g*C+slot_k, :]> for kept choices, else 0.  One warp per token.
+template <typename T>
+__global__ void __launch_bounds__(256) combine_bwd_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ out,
+                                                          const int32_t* __restrict__ expert_idx,
+                                                          const int32_t* __restrict__ slot, float* __restrict__ dw,
+                                                          long long N, int G, int S, int C, int row_vec) {
+  constexpr int n = Row16<T>::n;
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long t = warp; t < N; t += nwarps) {
+    const int g = (int)(t / S);
+    float acc[2] = {0.f, 0.f};
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int sl = slot[2 * t + k];
+      if (sl < 0) continue;
+      const uint4* r = out + (((long long)expert_idx[2 * t + k] * G + g) * C + sl) * row_vec;
+      const uint4* dyr = dy + t * row_vec;
+      for (int i = lane; i < row_vec; i += 32) {
+        float a[n], b[n];
+        Row16<T>::load(__ldg(r + i), a);
+        Row16<T>::load(__ldg(dyr + i), b);
+#pragma unroll
+        for (int j = 0; j < n; ++j) acc[k] = fmaf(a[j], b[j], acc[k]);
+      }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      acc[0] += __shfl_xor_sync(0xffffffffu, acc[0], off);
+      acc[1] += __shfl_xor_sync(0xffffffffu, acc[1], off);
+    }
+    if (lane == 0) { dw[2 * t] = acc[0]; dw[2 * t + 1] = acc[1]; }
+  }
+}
+
+// dout[e, g*C+c, :] = weight_k * dy[g, tok, :] for the token in the slot, zeros for an empty slot.
+template <typename T>
+__global__ void __launch_bounds__(256) dout_kernel(const uint4* __restrict__ dy, const int32_t* __restrict__ slot_token,
+                                                   const int32_t* __restrict__ expert_idx,
+                                                   const int32_t* __restrict__ slot, const float* __restrict__ weight,
+                                                   uint4* __restrict__ dout, long long R, int G, int S, int C,
+                                                   int row_vec) {
+  constexpr int n = Row16<T>::n;
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long r = warp; r < R; r += nwarps) {
+    const int tok = slot_token[r];
+    const int c = (int)(r % C);
+    const int g = (int)((r / C) % G);
+    const int e = (int)(r / ((long long)C * G));
+    uint4* dst = dout + r * row_vec;
+    if (tok < 0) {
+      for (int i = lane; i < row_vec; i += 32) dst[i] = make_uint4(0, 0, 0, 0);
+      continue;
+    }
+    const long long t = (long long)g * S + tok;
+    const int k = (expert_idx[2 * t] == e && slot[2 * t] == c) ? 0 : 1;
+    const float w = weight[2 * t + k];
+    const uint4* src = dy + t * row_vec;
+    for (int i = lane; i < row_vec; i += 32) {
+      float f[n];
+      Row16<T>::load(__ldg(src + i), f);
+#pragma unroll
+      for (int j = 0; j < n; ++j) f[j] *= w;
+      dst[i] = Row16<T>::store(f);
+    }
+  }
+}
+
+// Softmax backward per token (one warp): dlogit_e = p_e (dg_e - sum_e' p_e' dg_e').
+template <typename T>
+__global__ void __launch_bounds__(256) gate_bwd_kernel(const float* __restrict__ logits, const float* __restrict__ rowmax,
+                                                       const float* __restrict__ rowinv,
+                                                       const int32_t* __restrict__ expert_idx,
+                                                       const float* __restrict__ gate12, const float* __restrict__ dw,
+                                                       const int32_t* __restrict__ first_count, float aux_coef,
+                                                       T* __restrict__ dlogits, long long N, int S, int E) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long t = warp; t < N; t += nwarps) {
+    const int g = (int)(t / S);
+    const float mx = rowmax[t], inv = rowinv[t];
+    const int e1 = expert_idx[2 * t], e2 = expert_idx[2 * t + 1];
+    const float a = gate12[2 * t], b = gate12[2 * t + 1], D = a + b;
+    const float d1 = dw[2 * t], d2 = dw[2 * t + 1];
+    const float dga = (b / (D * D)) * (d1 - d2), dgb = (a / (D * D)) * (d2 - d1);
+    const float* row = logits + t * E;
+    const int32_t* fc = first_count + (long long)g * E;
+    float dot = 0.f;
+    for (int e = lane; e < E; e += 32) {
+      const float p = expf(row[e] - mx) * inv;
+      float dg = aux_coef * (float)fc[e];
+      if (e == e1) dg += dga;
+      if (e == e2) dg += dgb;
+      dot = fmaf(p, dg, dot);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, off);
+    for (int e = lane; e < E; e += 32) {
+      const float p = expf(row[e] - mx) * inv;
+      float dg = aux_coef * (float)fc[e];
+      if (e == e1) dg += dga;
+      if (e == e2) dg += dgb;
+      dlogits[t * E + e] = from_f32<T>(p * (dg - dot));
+    }
+  }
+}
+
+// dx[t,:] = dxg[t,:] (fp32, from the gating GEMM) + dbuf rows of the kept choices.
+template <typename T>
+__global__ void __launch_bounds__(256) dx_kernel(const float4* __restrict__ dxg, const uint4* __restrict__ dbuf,
+                                                 const int32_t* __restrict__ expert_idx, const int32_t* __restrict__ slot,
+                                                 uint4* __restrict__ dx, long long N, int G, int S, int C, int row_vec) {
+  constexpr int n = Row16<T>::n;
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long t = warp; t < N; t += nwarps) {
+    const int g = (int)(t / S);
+    const uint4* r[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int sl = slot[2 * t + k];
+      r[k] = sl >= 0 ? dbuf + (((long long)expert_idx[2 * t + k] * G + g) * C + sl) * row_vec : nullptr;
+    }
+    for (int i = lane; i < row_vec; i += 32) {
+      float acc[n];
+      const float4* gsrc = dxg + (t * row_vec + i) * (n / 4);
+#pragma unroll
+      for (int j = 0; j < n / 4; ++j) {
+        const float4 v = gsrc[j];
+        acc[4 * j] = v.x; acc[4 * j + 1] = v.y; acc[4 * j + 2] = v.z; acc[4 * j + 3] = v.w;
+      }
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        if (!r[k]) continue;
+        float f[n];
+        Row16<T>::load(__ldg(r[k] + i), f);
+#pragma unroll
+        for (int j = 0; j < n; ++j) acc[j] += f[j];
+      }
+      dx[t * row_vec + i] = Row16<T>::store(acc);
+    }
+  }
+}
+
+int grid_rows(long long rows) {
+  long long blocks = (rows + 7) / 8;
+  const long long cap = 148LL * 32;
+  return (int)(blocks < cap ? (blocks > 0 ? blocks : 1) : cap);
+}
+
+template <typename T>
+int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, const void* wo, const unsigned char* ctx,
+               const void* dy, float k_aux, void* dx, float* dwg, void* dwi, void* dwo, unsigned char* ws,
+               cudaStream_t st) {
+  const BwdPlan bp = plan_backward(d);
+  const CtxPlan cp = plan_context(d);
+  int* status = reinterpret_cast<int*>(ws + bp.status);
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  const int32_t* expert_idx = reinterpret_cast<const int32_t*>(ctx + cp.expert_idx);
+  const int32_t* slot = reinterpret_cast<const int32_t*>(ctx + cp.slot);
+  const float* weight = reinterpret_cast<const float*>(ctx + cp.weight);
+  const int32_t* first_count = reinterpret_cast<const int32_t*>(ctx + cp.first_count);
+  const int32_t* slot_token = reinterpret_cast<const int32_t*>(ctx + cp.slot_token);
+  const float* gate12 = reinterpret_cast<const float*>(ctx + cp.gate12);
+  const float* rowmax = reinterpret_cast<const float*>(ctx + cp.rowmax);
+  const float* rowinv = reinterpret_cast<const float*>(ctx + cp.rowinv);
+  const void* h = ctx + cp.h;
+  const void* out = ctx + cp.out;
+  float* logits = reinterpret_cast<float*>(ws + bp.logits);
+  T* dlogits = reinterpret_cast<T*>(ws + bp.dlogits);
+  float* dw = reinterpret_cast<float*>(ws + bp.dw);
+  void* buf = ws + bp.buf;
+  void* dout = ws + bp.dout;
+  void* dh = ws + bp.dh;
+  void* dbuf = ws + bp.dbuf;
+  float* dxg = reinterpret_cast<float*>(ws + bp.dxg);
+  const int row_vec = (int)((size_t)d.M * d.esize / 16);
+  const long long rows = d.rows;
+
+  // combine backward
+  combine_bwd_kernel<T><<<grid_rows(d.N), 256, 0, st>>>(reinterpret_cast<const uint4*>(dy),
+                                                        reinterpret_cast<const uint4*>(out), expert_idx, slot, dw, d.N,
+                                                        d.G, d.S, d.C, row_vec);
+  dout_kernel<T><<<grid_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(dy), slot_token, expert_idx, slot,
+                                                 weight, reinterpret_cast<uint4*>(dout), d.R, d.G, d.S, d.C, row_vec);
+  count_launch(2);
+  launch_dispatch(d, x, slot_token, buf, st);
+
+  // expert FFN backward
+  UmmaGemm g{};
+  // dh = (dout . wo^T) masked by h > 0
+  g.A = dout; g.B = wo; g.C = dh; g.mask = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;
+  g.a_kmajor = true; g.b_kmajor = true;
+  g.a_ld = d.M; g.a_bs = rows * d.M; g.b_ld = d.M; g.b_bs = (long long)d.H * d.M; g.c_ld = d.H; g.c_bs = rows * d.H;
+  g.b_stream = 1;
+  int rc = run_gemm(d, g, status, st);
+  if (rc) return rc;
+  // dwo[e] = h[e]^T . dout[e]   [H x M]
+  g = UmmaGemm{};
+  g.A = h; g.B = dout; g.C = dwo; g.rows = d.H; g.cols = d.M; g.K = d.rows; g.batch = d.E;
+  g.a_kmajor = false; g.b_kmajor = false;
+  g.a_ld = d.H; g.a_bs = rows * d.H; g.b_ld = d.M; g.b_bs = rows * d.M; g.c_ld = d.M; g.c_bs = (long long)d.H * d.M;
+  rc = run_gemm(d, g, status, st);
+  if (rc) return rc;
+  // dwi[e] = buf[e]^T . dh[e]   [M x H]
+  g = UmmaGemm{};
+  g.A = buf; g.B = dh; g.C = dwi; g.rows = d.M; g.cols = d.H; g.K = d.rows; g.batch = d.E;
+  g.a_kmajor = false; g.b_kmajor = false;
+  g.a_ld = d.M; g.a_bs = rows * d.M; g.b_ld = d.H; g.b_bs = rows * d.H; g.c_ld = d.H; g.c_bs = (long long)d.M * d.H;
+  rc = run_gemm(d, g, status, st);
+  if (rc) return rc;
+  // dbuf = dh . wi^T   [rows x M]
+  g = UmmaGemm{};
+  g.A = dh; g.B = wi; g.C = dbuf; g.rows = d.rows; g.cols = d.M; g.K = d.H; g.batch = d.E;
+  g.a_kmajor = true; g.b_kmajor = true;
+  g.a_ld = d.H; g.a_bs = rows * d.H; g.b_ld = d.H; g.b_bs = (long long)d.M * d.H; g.c_ld = d.M; g.c_bs = rows * d.M;
+  g.b_stream = 1;
+  rc = run_gemm(d, g, status, st);
+  if (rc) return rc;
+
+  // gating backward: recompute the logits, softmax backward, two GEMMs
+  rc = gate_logits(d, x, wg, logits, status, st);
+  if (rc) return rc;
+  const float aux_coef = k_aux / ((float)d.G * (float)d.E * (float)d.S * (float)d.S);
+  gate_bwd_kernel<T><<<grid_rows(d.N), 256, 0, st>>>(logits, rowmax, rowinv, expert_idx, gate12, dw, first_count,
+                                                     aux_coef, dlogits, d.N, d.S, d.E);
+  count_launch();
+  // dwg = x^T . dlogits   [M x E] fp32
+  g = UmmaGemm{};
+  g.A = x; g.B = dlogits; g.C = dwg; g.rows = d.M; g.cols = d.E; g.K = (int)d.N; g.batch = 1;
+  g.a_kmajor = false; g.b_kmajor = false; g.a_ld = d.M; g.b_ld = d.E; g.c_ld = d.E; g.out_f32 = 1;
+  rc = run_gemm(d, g, status, st);
+  if (rc) return rc;
+  // dxg = dlogits . wg^T   [N x M] fp32
+  g = UmmaGemm{};
+  g.A = dlogits; g.B = wg; g.C = dxg; g.rows = (int)d.N; g.cols = d.M; g.K = d.E; g.batch = 1;
+  g.a_kmajor = true; g.b_kmajor = true; g.a_ld = d.E; g.b_ld = d.E; g.c_ld = d.M; g.out_f32 = 1;
+  rc = run_gemm(d, g, status, st);
+  if (rc) return rc;
+  dx_kernel<T><<<grid_rows(d.N), 256, 0, st>>>(reinterpret_cast<const float4*>(dxg), reinterpret_cast<const uint4*>(dbuf),
+                                               expert_idx, slot, reinterpret_cast<uint4*>(dx), d.N, d.G, d.S, d.C,
+                                               row_vec);
+  count_launch();
+  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+}  // namespace
+
+int backward_device(const gshard_moe_shape* shape, const void* x, const void* wg, const void* wi, const void* wo,
+                    const void* context, const void* dy, float k_aux, void* dx, float* dwg, void* dwi, void* dwo,
+                    void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  const Dims d = make_dims(*shape);
+  if (workspace_bytes < plan_backward(d).total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  const unsigned char* ctx = static_cast<const unsigned char*>(context);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  if (d.bf16) return backward_t<__nv_bfloat16>(d, x, wg, wi, wo, ctx, dy, k_aux, dx, dwg, dwi, dwo, ws, st);
+  return backward_t<float>(d, x, wg, wi, wo, ctx, dy, k_aux, dx, dwg, dwi, dwo, ws, st);
+}
+
+}  // namespace gshard

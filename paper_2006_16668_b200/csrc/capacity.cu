@@ -1,0 +1,228 @@
+// Capacity assignment (Algorithm 1, the two token loops and l_aux) without a sequential scan
+// over tokens.  The paper's running counter c_e gives token s the position
+//   first choice : #{s' < s : e1(s') = e1(s)}
+//   second choice: c1[e2(s)] + #{s' < s : e2(s') = e2(s)}      (c1 = counts after loop 1)
+// i.e. a stable rank among the tokens of the group that picked the same expert.  One CTA
+// handles one group: every warp owns a contiguous chunk of tokens, ranks its tokens inside the
+// chunk with warp match/popcount against a per-warp histogram in shared memory, then an
+// exclusive scan over the warps' histograms (per expert, in warp order) gives each chunk's
+// offset.  Compact index lists are written; the dense [G,S,E,C] masks never exist.
+#include "kernels.cuh"
+
+namespace gshard {
+
+constexpr int kCapThreads = 512;
+
+struct CapacityArgs {
+  int S, E, C, G, warps_used, variant_a;
+  const int32_t* expert_idx;   // [G,S,2]
+  const float* gate12;         // [G,S,2]
+  const float* u;              // [G,S]
+  const float* m;              // [G,E]
+  int32_t* slot;               // [G,S,2]  (also scratch for in-chunk ranks)
+  float* weight;               // [G,S,2]
+  uint8_t* flags;              // [G,S]
+  int32_t* first_count;        // [G,E]
+  int32_t* total_count;        // [G,E]
+  int32_t* slot_token;         // [E,G,C]
+  float* l_aux_group;          // [G]
+  int32_t* stats_group;        // [G,8]
+};
+
+// Deterministic block sum (fixed tree), result valid in thread 0.
+template <typename T>
+__device__ T block_sum(T v, T* scratch) {
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) v += __shfl_down_sync(0xffffffffu, v, off);
+  __syncthreads();
+  if (lane == 0) scratch[w] = v;
+  __syncthreads();
+  T r = 0;
+  if (threadIdx.x == 0)
+    for (int i = 0; i < (int)(blockDim.x >> 5); ++i) r += scratch[i];
+  return r;
+}
+
+// Ranks one choice (k = 0 first, 1 second) of every token of the chunk inside the chunk and
+// leaves the chunk's per-expert counts in hist_w.  In-chunk ranks go to slot[.,k] as scratch.
+__device__ __forceinline__ void rank_chunk(const CapacityArgs& a, int g, int k, int lo, int hi,
+                                           unsigned short* hist_w, bool second_pass) {
+  const int lane = threadIdx.x & 31;
+  const unsigned lt = (1u << lane) - 1u;
+  for (int base = lo; base < hi; base += 32) {
+    const int s = base + lane;
+    const bool valid = s < hi;
+    const long long t = (long long)g * a.S + (valid ? s : lo);
+    int key = valid ? a.expert_idx[2 * t + k] : -1 - lane;
+    bool counts = valid;
+    if (second_pass && a.variant_a && valid) counts = (a.flags[t] & 2u) != 0;
+    if (!counts) key = -1 - lane;           // unique key: matches nobody
+    const unsigned mask = __match_any_sync(0xffffffffu, key);
+    const int rank = __popc(mask & lt);
+    int before = 0;
+    if (counts) before = hist_w[key];
+    __syncwarp();
+    if (counts && rank == 0) hist_w[key] = (unsigned short)(before + __popc(mask));
+    __syncwarp();
+    if (valid) a.slot[2 * t + k] = counts ? before + rank : 0;
+  }
+}
+
+__global__ void __launch_bounds__(kCapThreads) capacity_kernel(CapacityArgs a) {
+  extern __shared__ unsigned char smem_raw[];
+  int32_t* cnt = reinterpret_cast<int32_t*>(smem_raw);                       // [E] running c_e
+  unsigned short* hist = reinterpret_cast<unsigned short*>(cnt + a.E);       // [warps_used][E]
+  __shared__ float red_f[kCapThreads / 32];
+  __shared__ int red_i[kCapThreads / 32];
+
+  const int g = blockIdx.x;
+  const int tid = threadIdx.x, w = tid >> 5;
+  const int W = a.warps_used;
+  const int chunk = (a.S + W - 1) / W;
+  const int lo = min(a.S, w * chunk), hi = (w < W) ? min(a.S, lo + chunk) : lo;
+
+  // empty slots are -1; this group's part of slot_token is E rows of C entries
+  for (int i = tid; i < a.E * a.C; i += blockDim.x) {
+    const int e = i / a.C, c = i % a.C;
+    a.slot_token[((long long)e * a.G + g) * a.C + c] = -1;
+  }
+  for (int i = tid; i < W * a.E; i += blockDim.x) hist[i] = 0;
+  __syncthreads();
+
+  // ---- first loop of Algorithm 1 ---------------------------------------------------------
+  if (w < W) rank_chunk(a, g, 0, lo, hi, hist + (size_t)w * a.E, false);
+  __syncthreads();
+  float aux = 0.f;
+  for (int e = tid; e < a.E; e += blockDim.x) {
+    int run = 0;
+    for (int ww = 0; ww < W; ++ww) {
+      const int t = hist[(size_t)ww * a.E + e];
+      hist[(size_t)ww * a.E + e] = (unsigned short)run;
+      run += t;
+    }
+    cnt[e] = run;                                     // c_e after the first loop, unclipped
+    a.first_count[(long long)g * a.E + e] = run;
+    aux += ((float)run / (float)a.S) * a.m[(long long)g * a.E + e];
+  }
+  __syncthreads();
+  const float aux_sum = block_sum<float>(aux, red_f);
+  if (tid == 0) a.l_aux_group[g] = aux_sum / (float)a.E;
+
+  int n_first_dropped = 0, n_rnd_skipped = 0, n_cap_dropped = 0, n_overflowed = 0, n_filled = 0;
+  for (int s = lo + (tid & 31); s < hi; s += 32) {
+    const long long t = (long long)g * a.S + s;
+    const int e1 = a.expert_idx[2 * t];
+    const float g1 = a.gate12[2 * t], g2 = a.gate12[2 * t + 1];
+    const float den = g1 + g2;
+    const float w1 = g1 / den, w2 = g2 / den;
+    const int pos = (int)hist[(size_t)w * a.E + e1] + a.slot[2 * t];
+    unsigned f = 0;
+    if (pos < a.C) {
+      f |= 1u;
+      a.slot[2 * t] = pos;
+      a.slot_token[((long long)e1 * a.G + g) * a.C + pos] = s;
+      ++n_filled;
+    } else {
+      a.slot[2 * t] = -1;
+      ++n_first_dropped;
+    }
+    if (2.0f * w2 > a.u[t]) f |= 2u;                   // random routing test, strict >
+    a.weight[2 * t] = w1;
+    a.weight[2 * t + 1] = w2;
+    a.flags[t] = (uint8_t)f;
+  }
+  __syncthreads();
+
+  // ---- second loop: counters continue from the first loop --------------------------------
+  for (int i = tid; i < W * a.E; i += blockDim.x) hist[i] = 0;
+  __syncthreads();
+  if (w < W) rank_chunk(a, g, 1, lo, hi, hist + (size_t)w * a.E, true);
+  __syncthreads();
+  for (int e = tid; e < a.E; e += blockDim.x) {
+    int run = cnt[e];
+    for (int ww = 0; ww < W; ++ww) {
+      const int t = hist[(size_t)ww * a.E + e];
+      hist[(size_t)ww * a.E + e] = (unsigned short)min(run, 65535);
+      run += t;
+    }
+    a.total_count[(long long)g * a.E + e] = run;
+  }
+  __syncthreads();
+  for (int s = lo + (tid & 31); s < hi; s += 32) {
+    const long long t = (long long)g * a.S + s;
+    const int e2 = a.expert_idx[2 * t + 1];
+    unsigned f = a.flags[t];
+    const bool pass = (f & 2u) != 0;
+    const int pos = (int)hist[(size_t)w * a.E + e2] + a.slot[2 * t + 1];
+    if (pass && pos < a.C) {
+      f |= 4u;
+      a.slot[2 * t + 1] = pos;
+      a.slot_token[((long long)e2 * a.G + g) * a.C + pos] = s;
+      ++n_filled;
+    } else {
+      a.slot[2 * t + 1] = -1;
+      if (!pass) ++n_rnd_skipped; else ++n_cap_dropped;
+    }
+    if ((f & 5u) == 0) ++n_overflowed;
+    a.flags[t] = (uint8_t)f;
+  }
+  const int vals[5] = {n_first_dropped, n_rnd_skipped, n_cap_dropped, n_overflowed, n_filled};
+#pragma unroll
+  for (int i = 0; i < 5; ++i) {
+    const int r = block_sum<int>(vals[i], red_i);
+    if (tid == 0) a.stats_group[g * 8 + i] = r;
+  }
+  if (tid < 3) a.stats_group[g * 8 + 5 + tid] = 0;
+}
+
+// Layer-level results: l_aux = mean over groups (fixed order), stats summed over groups.
+__global__ void capacity_finalize_kernel(const float* l_aux_group, const int32_t* stats_group, int G,
+                                         float* l_aux, long long* stats) {
+  if (threadIdx.x == 0 && l_aux) {
+    float acc = 0.f;
+    for (int g = 0; g < G; ++g) acc += l_aux_group[g];
+    *l_aux = acc / (float)G;
+  }
+  if (stats && threadIdx.x < 8) {
+    long long acc = 0;
+    for (int g = 0; g < G; ++g) acc += stats_group[g * 8 + threadIdx.x];
+    stats[threadIdx.x] = acc;
+  }
+}
+
+size_t capacity_smem_bytes(int E, int warps) { return (size_t)E * 4 + (size_t)warps * E * 2; }
+
+int capacity_warps_for(int E) {
+  int w = kCapThreads / 32;
+  while (w > 1 && capacity_smem_bytes(E, w) > 200 * 1024) w >>= 1;
+  return capacity_smem_bytes(E, w) <= 200 * 1024 ? w : 0;
+}
+
+int launch_capacity(const Dims& d, const int32_t* expert_idx, const float* gate12, const float* u,
+                    const float* m, int32_t* slot, float* weight, uint8_t* flags, int32_t* first_count,
+                    int32_t* total_count, int32_t* slot_token, float* l_aux_group, int32_t* stats_group,
+                    float* l_aux, long long* stats, cudaStream_t st) {
+  CapacityArgs a;
+  a.S = d.S; a.E = d.E; a.C = d.C; a.G = d.G;
+  a.warps_used = capacity_warps_for(d.E);
+  if (a.warps_used == 0) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  a.variant_a = d.variant_a ? 1 : 0;
+  a.expert_idx = expert_idx; a.gate12 = gate12; a.u = u; a.m = m;
+  a.slot = slot; a.weight = weight; a.flags = flags; a.first_count = first_count;
+  a.total_count = total_count; a.slot_token = slot_token; a.l_aux_group = l_aux_group;
+  a.stats_group = stats_group;
+  const size_t smem = capacity_smem_bytes(d.E, a.warps_used);
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(capacity_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+      return GSHARD_ERR_CUDA;
+    attr_set = true;
+  }
+  capacity_kernel<<<d.G, kCapThreads, smem, st>>>(a);
+  capacity_finalize_kernel<<<1, 32, 0, st>>>(l_aux_group, stats_group, d.G, l_aux, stats);
+  count_launch(2);
+  return GSHARD_OK;
+}
+
+}  // namespace gshard

@@ -1,0 +1,60 @@
+// Shared declarations of the CUDA library: shape helpers, status word, element conversion.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/gshard_moe.h"
+
+namespace gshard {
+
+constexpr int kGateTile = 128;        // tokens per column-sum partial of the mean gates
+constexpr size_t kAlign = 256;        // alignment of every workspace region
+
+__host__ __device__ inline size_t align_up(size_t v, size_t a = kAlign) { return (v + a - 1) / a * a; }
+__host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// Device status word: first error wins; 0 = OK.
+__device__ inline void set_device_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+template <typename T> __device__ inline float to_f32(T v);
+template <> __device__ inline float to_f32<float>(float v) { return v; }
+template <> __device__ inline float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ inline T from_f32(float v);
+template <> __device__ inline float from_f32<float>(float v) { return v; }
+template <> __device__ inline __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+struct LaunchCounter {
+  int n = 0;
+};
+LaunchCounter& launch_counter();   // thread-local
+inline void count_launch(int k = 1) { launch_counter().n += k; }
+
+// Sizes derived from a shape.
+struct Dims {
+  int G, S, M, H, E, C;
+  long long N;          // tokens
+  long long R;          // slots = E*G*C
+  int rows;             // rows per expert = G*C
+  int tiles_per_group;  // ceil(S / kGateTile)
+  size_t esize;         // bytes of one x / weight element
+  bool bf16;
+  bool simt;            // contractions on CUDA cores
+  bool variant_a;
+};
+
+inline Dims make_dims(const gshard_moe_shape& s) {
+  Dims d;
+  d.G = s.G; d.S = s.S; d.M = s.M; d.H = s.H; d.E = s.E; d.C = s.C;
+  d.N = (long long)s.G * s.S;
+  d.R = (long long)s.E * s.G * s.C;
+  d.rows = s.G * s.C;
+  d.tiles_per_group = ceil_div(s.S, kGateTile);
+  d.bf16 = s.dtype == GSHARD_BF16;
+  d.esize = d.bf16 ? 2 : 4;
+  d.simt = !d.bf16 || (s.flags & GSHARD_FLAG_SIMT_CONTRACTIONS);
+  d.variant_a = (s.flags & GSHARD_FLAG_SECOND_SKIP_FREES_SLOT) != 0;
+  return d;
+}
+
+}  // namespace gshard

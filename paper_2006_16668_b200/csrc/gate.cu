@@ -1,0 +1,123 @@
+// Gating kernels on stored fp32 logits: row softmax statistics, the top-2 pick and the
+// per-tile column sums of the gates (Algorithm 1: "g <- softmax(wg . x)", "top_2",
+// "m_E <- (1/S) sum_s g_{s,E}").
+#include "kernels.cuh"
+
+namespace gshard {
+
+struct Top2 {
+  float v1, v2;
+  int i1, i2;
+};
+
+// "a before b": larger value first, lower index on equal values.
+__device__ __forceinline__ bool before(float va, int ia, float vb, int ib) {
+  return va > vb || (va == vb && ia < ib);
+}
+
+__device__ __forceinline__ void top2_insert(Top2& t, float v, int i) {
+  if (before(v, i, t.v1, t.i1)) { t.v2 = t.v1; t.i2 = t.i1; t.v1 = v; t.i1 = i; }
+  else if (before(v, i, t.v2, t.i2)) { t.v2 = v; t.i2 = i; }
+}
+
+__device__ __forceinline__ Top2 top2_merge(const Top2& a, const Top2& b) {
+  Top2 r;
+  if (before(b.v1, b.i1, a.v1, a.i1)) {
+    r.v1 = b.v1; r.i1 = b.i1;
+    if (before(a.v1, a.i1, b.v2, b.i2)) { r.v2 = a.v1; r.i2 = a.i1; } else { r.v2 = b.v2; r.i2 = b.i2; }
+  } else {
+    r.v1 = a.v1; r.i1 = a.i1;
+    if (before(b.v1, b.i1, a.v2, a.i2)) { r.v2 = b.v1; r.i2 = b.i1; } else { r.v2 = a.v2; r.i2 = a.i2; }
+  }
+  return r;
+}
+
+// One warp per token: row max, 1/sum(exp), the two largest logits and their indices.
+// Softmax is monotone, so top-2 of the gates is top-2 of the logits.
+__global__ void __launch_bounds__(256) gate_rows_kernel(const float* __restrict__ logits, long long N,
+                                                        int E, int32_t* __restrict__ expert_idx,
+                                                        float* __restrict__ gate12,
+                                                        float* __restrict__ rowmax,
+                                                        float* __restrict__ rowinv) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  const float ninf = __int_as_float(0xff800000);
+  for (long long t = warp; t < N; t += nwarps) {
+    const float* row = logits + t * E;
+    Top2 tp{ninf, ninf, 0x7fffffff, 0x7fffffff};
+    for (int e = lane; e < E; e += 32) top2_insert(tp, row[e], e);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      Top2 o;
+      o.v1 = __shfl_xor_sync(0xffffffffu, tp.v1, off);
+      o.v2 = __shfl_xor_sync(0xffffffffu, tp.v2, off);
+      o.i1 = __shfl_xor_sync(0xffffffffu, tp.i1, off);
+      o.i2 = __shfl_xor_sync(0xffffffffu, tp.i2, off);
+      tp = top2_merge(tp, o);
+    }
+    float sum = 0.f;
+    for (int e = lane; e < E; e += 32) sum += expf(row[e] - tp.v1);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, off);
+    if (lane == 0) {
+      const float inv = 1.0f / sum;
+      expert_idx[2 * t] = tp.i1;
+      expert_idx[2 * t + 1] = tp.i2;
+      gate12[2 * t] = inv;                        // exp(l1 - max) = 1
+      gate12[2 * t + 1] = expf(tp.v2 - tp.v1) * inv;
+      rowmax[t] = tp.v1;
+      rowinv[t] = inv;
+    }
+  }
+}
+
+// Column sums of the gates over one tile of kGateTile tokens of one group; thread = expert.
+// partial[(g*tiles_per_group + tile), e] = sum over the tile's tokens of softmax value.
+__global__ void __launch_bounds__(128) gate_colsum_kernel(const float* __restrict__ logits,
+                                                          const float* __restrict__ rowmax,
+                                                          const float* __restrict__ rowinv, int S,
+                                                          int E, int tiles_per_group,
+                                                          float* __restrict__ partial) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  const int tile = blockIdx.y;
+  const int g = tile / tiles_per_group;
+  const int s0 = (tile % tiles_per_group) * kGateTile;
+  const int s1 = min(S, s0 + kGateTile);
+  __shared__ float smax[kGateTile], sinv[kGateTile];
+  for (int i = threadIdx.x; i < s1 - s0; i += blockDim.x) {
+    smax[i] = rowmax[(long long)g * S + s0 + i];
+    sinv[i] = rowinv[(long long)g * S + s0 + i];
+  }
+  __syncthreads();
+  if (e >= E) return;
+  float acc = 0.f;
+  const float* base = logits + ((long long)g * S + s0) * E + e;
+  for (int i = 0; i < s1 - s0; ++i) acc += expf(base[(long long)i * E] - smax[i]) * sinv[i];
+  partial[(long long)tile * E + e] = acc;
+}
+
+// m[g,e] = (1/S) * sum of the group's tile partials, added in tile order (reproducible).
+__global__ void __launch_bounds__(128) gate_mean_kernel(const float* __restrict__ partial, int S, int E,
+                                                        int tiles_per_group, float* __restrict__ m) {
+  const int e = blockIdx.x * blockDim.x + threadIdx.x;
+  const int g = blockIdx.y;
+  if (e >= E) return;
+  float acc = 0.f;
+  for (int t = 0; t < tiles_per_group; ++t) acc += partial[((long long)g * tiles_per_group + t) * E + e];
+  m[(long long)g * E + e] = acc / (float)S;
+}
+
+void launch_gate_rows(const Dims& d, const float* logits, int32_t* expert_idx, float* gate12,
+                      float* rowmax, float* rowinv, float* partial, float* m, cudaStream_t st) {
+  const long long warps_needed = d.N;
+  int blocks = (int)((warps_needed + 7) / 8);
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  gate_rows_kernel<<<blocks, 256, 0, st>>>(logits, d.N, d.E, expert_idx, gate12, rowmax, rowinv);
+  dim3 grid(ceil_div(d.E, 128), d.G * d.tiles_per_group);
+  gate_colsum_kernel<<<grid, 128, 0, st>>>(logits, rowmax, rowinv, d.S, d.E, d.tiles_per_group, partial);
+  gate_mean_kernel<<<dim3(ceil_div(d.E, 128), d.G), 128, 0, st>>>(partial, d.S, d.E, d.tiles_per_group, m);
+  count_launch(3);
+}
+
+}  // namespace gshard

@@ -1,0 +1,26 @@
+// One description of a batched contraction, run either on tcgen05 (bf16) or on CUDA cores.
+#pragma once
+#include "kernels.cuh"
+#include "simt_gemm.cuh"
+
+namespace gshard {
+
+// A and B hold the configuration dtype; C holds float when g.out_f32, else the dtype.
+inline int run_gemm(const Dims& d, const UmmaGemm& g, int* status, cudaStream_t st) {
+  if (!d.simt) return launch_umma_gemm(g, status, st);
+  SimtGemm s{};
+  s.A = g.A; s.B = g.B; s.C = g.C; s.mask = g.mask;
+  s.rows = g.rows; s.cols = g.cols; s.K = g.K; s.batch = g.batch;
+  s.a_rs = g.a_kmajor ? g.a_ld : 1; s.a_cs = g.a_kmajor ? 1 : g.a_ld; s.a_bs = g.a_bs;
+  s.b_rs = g.b_kmajor ? 1 : g.b_ld; s.b_cs = g.b_kmajor ? g.b_ld : 1; s.b_bs = g.b_bs;
+  s.c_rs = g.c_ld; s.c_bs = g.c_bs; s.relu = g.relu; s.accumulate = 0;
+  if (d.bf16) {
+    if (g.out_f32) launch_simt_gemm<__nv_bfloat16, __nv_bfloat16, float>(s, st);
+    else launch_simt_gemm<__nv_bfloat16, __nv_bfloat16, __nv_bfloat16>(s, st);
+  } else {
+    launch_simt_gemm<float, float, float>(s, st);
+  }
+  return GSHARD_OK;
+}
+
+}  // namespace gshard

@@ -1,0 +1,39 @@
+// Launchers of the library's kernels (one .cu file each) as seen by the C-ABI layer.
+#pragma once
+#include "common.cuh"
+
+namespace gshard {
+
+// gate.cu: row statistics + top-2 on stored logits, tile column sums, mean gates.
+void launch_gate_rows(const Dims& d, const float* logits, int32_t* expert_idx, float* gate12, float* rowmax,
+                      float* rowinv, float* partial, float* m, cudaStream_t st);
+
+// capacity.cu
+int launch_capacity(const Dims& d, const int32_t* expert_idx, const float* gate12, const float* u, const float* m,
+                    int32_t* slot, float* weight, uint8_t* flags, int32_t* first_count, int32_t* total_count,
+                    int32_t* slot_token, float* l_aux_group, int32_t* stats_group, float* l_aux, long long* stats,
+                    cudaStream_t st);
+int capacity_warps_for(int E);
+
+// dispatch_combine.cu
+void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st);
+void launch_combine(const Dims& d, const void* out, const int32_t* expert_idx, const int32_t* slot,
+                    const float* weight, void* y, cudaStream_t st);
+
+// umma_gemm.cu: batched bf16 GEMM on tcgen05, C[b] = act(A[b] . B[b]).
+struct UmmaGemm {
+  const void* A; const void* B; void* C;
+  const void* mask;          // optional bf16 tensor laid out like C: output zeroed where mask <= 0
+  int rows, cols, K, batch;
+  bool a_kmajor;             // A stored [rows, K] (K contiguous); else stored [K, rows]
+  bool b_kmajor;             // B stored [cols, K] (K contiguous); else stored [K, cols]
+  long long a_ld, a_bs;      // elements between consecutive stored rows / between batches
+  long long b_ld, b_bs;
+  long long c_ld, c_bs;      // C is [rows, cols] row-major
+  int out_f32;               // C is float instead of bf16
+  int relu;
+  int a_stream, b_stream;    // operand is read once: load with an evict-first L2 hint
+};
+int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st);
+
+}  // namespace gshard

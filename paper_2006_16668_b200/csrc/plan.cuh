@@ -1,0 +1,102 @@
+// Byte offsets of every region of the caller's workspace / context buffers.  All regions are
+// 256-byte aligned; the status word is the first word of the workspace.
+#pragma once
+#include "common.cuh"
+
+namespace gshard {
+
+struct Carver {
+  size_t off = 0;
+  size_t take(size_t bytes) { const size_t o = off; off = align_up(off + bytes); return o; }
+};
+
+struct FwdPlan {
+  size_t status, logits, rowmax, rowinv, partial, gate12, m, expert_idx, slot, weight, flags, first_count,
+      total_count, slot_token, l_aux_group, stats_group, buf, h, out, total;
+};
+
+inline FwdPlan plan_forward(const Dims& d) {
+  Carver c; FwdPlan p;
+  const size_t N = (size_t)d.N, R = (size_t)d.R;
+  p.status = c.take(256);
+  p.logits = c.take(N * d.E * 4);
+  p.rowmax = c.take(N * 4);
+  p.rowinv = c.take(N * 4);
+  p.partial = c.take((size_t)d.G * d.tiles_per_group * d.E * 4);
+  p.gate12 = c.take(N * 2 * 4);
+  p.m = c.take((size_t)d.G * d.E * 4);
+  p.expert_idx = c.take(N * 2 * 4);
+  p.slot = c.take(N * 2 * 4);
+  p.weight = c.take(N * 2 * 4);
+  p.flags = c.take(N);
+  p.first_count = c.take((size_t)d.G * d.E * 4);
+  p.total_count = c.take((size_t)d.G * d.E * 4);
+  p.slot_token = c.take(R * 4);
+  p.l_aux_group = c.take((size_t)d.G * 4);
+  p.stats_group = c.take((size_t)d.G * 8 * 4);
+  p.buf = c.take(R * d.M * d.esize);
+  p.h = c.take(R * d.H * d.esize);
+  p.out = c.take(R * d.M * d.esize);
+  p.total = c.off;
+  return p;
+}
+
+// Saved by the forward for the backward: routing, softmax row statistics, hidden activations
+// and expert outputs.
+struct CtxPlan {
+  size_t expert_idx, slot, weight, first_count, slot_token, gate12, rowmax, rowinv, h, out, total;
+};
+
+inline CtxPlan plan_context(const Dims& d) {
+  Carver c; CtxPlan p;
+  const size_t N = (size_t)d.N, R = (size_t)d.R;
+  p.expert_idx = c.take(N * 2 * 4);
+  p.slot = c.take(N * 2 * 4);
+  p.weight = c.take(N * 2 * 4);
+  p.first_count = c.take((size_t)d.G * d.E * 4);
+  p.slot_token = c.take(R * 4);
+  p.gate12 = c.take(N * 2 * 4);
+  p.rowmax = c.take(N * 4);
+  p.rowinv = c.take(N * 4);
+  p.h = c.take(R * d.H * d.esize);
+  p.out = c.take(R * d.M * d.esize);
+  p.total = c.off;
+  return p;
+}
+
+struct StagePlan { size_t x, u, y, l_aux, total; };
+
+inline StagePlan plan_staging(const Dims& d) {
+  Carver c; StagePlan p;
+  p.x = c.take((size_t)d.N * d.M * d.esize);
+  p.u = c.take((size_t)d.N * 4);
+  p.y = c.take((size_t)d.N * d.M * d.esize);
+  p.l_aux = c.take(256);
+  p.total = c.off;
+  return p;
+}
+
+// Backward scratch: logits / dlogits [N,E], dispatched inputs, dout, dh, dbuf, per-token dw.
+struct BwdPlan {
+  size_t status, logits, dlogits, dw, buf, dout, dh, dbuf, dxg, total;
+};
+
+inline BwdPlan plan_backward(const Dims& d) {
+  Carver c; BwdPlan p;
+  const size_t N = (size_t)d.N, R = (size_t)d.R;
+  p.status = c.take(256);
+  p.logits = c.take(N * d.E * 4);
+  p.dlogits = c.take(N * d.E * d.esize);
+  p.dw = c.take(N * 2 * 4);
+  p.buf = c.take(R * d.M * d.esize);
+  p.dout = c.take(R * d.M * d.esize);
+  p.dh = c.take(R * d.H * d.esize);
+  p.dbuf = c.take(R * d.M * d.esize);
+  p.dxg = c.take(N * d.M * 4);
+  p.total = c.off;
+  return p;
+}
+
+int validate_shape(const gshard_moe_shape* s);
+
+}  // namespace gshard

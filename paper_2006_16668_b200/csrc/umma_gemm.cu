@@ -1,0 +1,314 @@
+// Grouped bf16 GEMM on the 5th-generation tensor cores: C[b] = act(A[b] . B[b]) for a batch of
+// independent problems (the experts), fp32 accumulation in tensor memory.
+//
+// One persistent CTA per SM walks a static list of 128 x BN output tiles.  Warp roles:
+//   warp 0      TMA producer: cp.async.bulk.tensor loads of A and B k-blocks (64 deep) into a
+//               ring of 128-byte-swizzled shared-memory stages, completion on mbarriers
+//   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=BN, K=16) from shared-memory
+//               descriptors into one of two TMEM accumulators; tcgen05.commit frees the stage
+//   warps 2..5  epilogue: tcgen05.ld the finished accumulator (thread = row), apply ReLU / mask,
+//               convert and store; overlaps the next tile's MMAs through the second accumulator
+// Operands may be K-major or MN-major in global memory (the expert weights wi [M,H] and wo [H,M]
+// are contiguous along the non-contracted dimension); the layout goes into the tensor map, the
+// shared-memory descriptor and the instruction descriptor - nothing is transposed in memory.
+// Tile order: row tiles fastest, then column tiles, then batch, so CTAs that run together share
+// the same weight tile through L2 and each weight byte leaves HBM once.
+#include <cuda.h>
+
+#include "kernels.cuh"
+#include "sm100_ptx.cuh"
+
+namespace gshard {
+
+namespace {
+
+constexpr int BM = 128, BK = 64;
+constexpr int kThreads = 192;
+constexpr int kABytes = BM * BK * 2;        // 16 KB
+constexpr int kBoxBytes = 64 * 64 * 2;      // one 64x64 box of an MN-major operand
+
+template <int BN> struct Cfg {
+  static constexpr int b_bytes = BN * BK * 2;
+  static constexpr int stage_bytes = kABytes + b_bytes;
+  static constexpr int stages = (BN == 256) ? 4 : 6;
+  static constexpr int tmem_cols = 2 * BN;   // two accumulators
+  static constexpr int smem_bytes = stages * stage_bytes + 1024 /*align*/ + 256 /*barriers*/;
+};
+
+struct Params {
+  void* C;
+  const void* mask;
+  int rows, cols, K, batch;
+  long long c_ld, c_bs;
+  int m_tiles, n_tiles, total_tiles, k_blocks;
+  int out_f32, relu;
+  int a_stream, b_stream;
+  int* status;
+};
+
+template <bool A_K, bool B_K, int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                 const Params p) {
+  using C_ = Cfg<BN>;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C_::stages * C_::stage_bytes);
+  uint64_t* full = bars;                       // [stages]
+  uint64_t* empty = bars + C_::stages;         // [stages]
+  uint64_t* acc_full = bars + 2 * C_::stages;  // [2]
+  uint64_t* acc_empty = acc_full + 2;          // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C_::stages; ++s) { ptx::mbar_init(full + s, 1); ptx::mbar_init(empty + s, 1); }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full + a, 1); ptx::mbar_init(acc_empty + a, 4); }
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&map_a);
+    ptx::prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, C_::tmem_cols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  bool ok = true;
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (lane == 0) {
+      const uint64_t pol_a = p.a_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
+      const uint64_t pol_b = p.b_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
+      int stage = 0; uint32_t phase = 0;
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+        const int mt = tile % p.m_tiles;
+        const int nt = (tile / p.m_tiles) % p.n_tiles;
+        const int b = tile / (p.m_tiles * p.n_tiles);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!ptx::mbar_wait(empty + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          unsigned char* sa = smem + stage * C_::stage_bytes;
+          unsigned char* sb = sa + kABytes;
+          ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)C_::stage_bytes);
+          if (A_K) {
+            ptx::tma_load_3d(sa, &map_a, full + stage, kb * BK, mt * BM, b, pol_a);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j)
+              ptx::tma_load_3d(sa + j * kBoxBytes, &map_a, full + stage, mt * BM + j * 64, kb * BK, b, pol_a);
+          }
+          if (B_K) {
+            ptx::tma_load_3d(sb, &map_b, full + stage, kb * BK, nt * BN, b, pol_b);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BN / 64; ++j)
+              ptx::tma_load_3d(sb + j * kBoxBytes, &map_b, full + stage, nt * BN + j * 64, kb * BK, b, pol_b);
+          }
+          if (++stage == C_::stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer --------------------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_bf16(BM, BN, !A_K, !B_K);
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+        if (!ptx::mbar_wait(acc_empty + acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!ptx::mbar_wait(full + stage, phase, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after_sync();
+          const uint32_t sa = ptx::smem_u32(smem + stage * C_::stage_bytes);
+          const uint32_t sb = sa + kABytes;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = A_K ? ptx::make_smem_desc(sa + k * 32, 16, 1024)
+                                    : ptx::make_smem_desc(sa + k * 2048, kBoxBytes, 1024);
+            const uint64_t db = B_K ? ptx::make_smem_desc(sb + k * 32, 16, 1024)
+                                    : ptx::make_smem_desc(sb + k * 2048, kBoxBytes, 1024);
+            ptx::umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          ptx::umma_commit(empty + stage);           // stage reusable once these MMAs have read it
+          if (++stage == C_::stages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        ptx::umma_commit(acc_full + acc);            // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue ----------------------------------------------
+    const int q = warp & 3;                          // TMEM lane quarter this warp may access
+    int acc = 0; uint32_t acc_phase = 0;
+    for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+      const int mt = tile % p.m_tiles;
+      const int nt = (tile / p.m_tiles) % p.n_tiles;
+      const int b = tile / (p.m_tiles * p.n_tiles);
+      if (!ptx::mbar_wait(acc_full + acc, acc_phase, abort_flag)) { ok = false; break; }
+      ptx::tc_fence_after_sync();
+      const int row = mt * BM + q * 32 + lane;
+      const bool row_ok = row < p.rows;
+      const long long row_off = (long long)b * p.c_bs + (long long)row * p.c_ld;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        const int col0 = nt * BN + c * 32;
+        if (col0 >= p.cols) break;                   // uniform over the warp
+        uint32_t r[32];
+        ptx::tmem_ld_32x32(tmem_base + (uint32_t)(acc * BN + c * 32) + ((uint32_t)(q * 32) << 16), r);
+        ptx::tmem_ld_wait();
+        if (!row_ok) continue;
+        float v[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          v[i] = __uint_as_float(r[i]);
+          if (p.relu) v[i] = fmaxf(v[i], 0.f);
+        }
+        const bool full_chunk = col0 + 32 <= p.cols;
+        if (p.mask) {
+          const __nv_bfloat16* mk = reinterpret_cast<const __nv_bfloat16*>(p.mask) + row_off + col0;
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (col0 + i < p.cols && !(__bfloat162float(mk[i]) > 0.f)) v[i] = 0.f;
+        }
+        if (p.out_f32) {
+          float* dst = reinterpret_cast<float*>(p.C) + row_off + col0;
+          if (full_chunk) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              reinterpret_cast<float4*>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          } else {
+            for (int i = 0; i < 32; ++i) if (col0 + i < p.cols) dst[i] = v[i];
+          }
+        } else {
+          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + row_off + col0;
+          if (full_chunk) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              uint32_t w[4];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const __nv_bfloat162 pr = __floats2bfloat162_rn(v[8 * i + 2 * j], v[8 * i + 2 * j + 1]);
+                w[j] = *reinterpret_cast<const uint32_t*>(&pr);
+              }
+              reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          } else {
+            for (int i = 0; i < 32; ++i) if (col0 + i < p.cols) dst[i] = __float2bfloat16_rn(v[i]);
+          }
+        }
+      }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ------------------------------ teardown ---------------------------------------------------
+  if (!ok) {
+    *abort_flag = 1;
+    set_device_status(p.status, GSHARD_ERR_TIMEOUT);
+    // give copies and MMAs already in flight a bounded time to land before the CTA's shared and
+    // tensor memory are released
+    const uint64_t t0 = ptx::globaltimer_ns();
+    while (ptx::globaltimer_ns() - t0 < 2000000ull) { __nanosleep(1000); }
+  }
+  __syncwarp();
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, C_::tmem_cols);
+  }
+}
+
+// ---- host side ------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* f = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+      f = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(f);
+  }();
+  return fn;
+}
+
+// 3-D bf16 tensor map {inner, outer, batch} with a {box_inner, box_outer, 1} box, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, long long inner, long long outer, long long batch,
+              long long ld_elems, long long bs_elems, int box_inner, int box_outer) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)batch};
+  cuuint64_t strides[2] = {(cuuint64_t)ld_elems * 2, (cuuint64_t)(batch > 1 ? bs_elems : ld_elems * outer) * 2};
+  cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool A_K, bool B_K, int BN>
+int launch_t(const UmmaGemm& g, const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int grid,
+             cudaStream_t st) {
+  auto kern = umma_gemm_kernel<A_K, B_K, BN>;
+  static bool attr_done = false;
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::smem_bytes) != cudaSuccess)
+      return GSHARD_ERR_CUDA;
+    attr_done = true;
+  }
+  kern<<<grid, kThreads, Cfg<BN>::smem_bytes, st>>>(ma, mb, p);
+  count_launch();
+  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+}  // namespace
+
+int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
+  if (g.rows <= 0 || g.cols <= 0 || g.K <= 0 || g.batch <= 0) return GSHARD_OK;
+  const int BN = g.cols > 128 ? 256 : 128;
+  CUtensorMap ma, mb;
+  bool okm;
+  if (g.a_kmajor) okm = make_map(&ma, g.A, g.K, g.rows, g.batch, g.a_ld, g.a_bs, BK, BM);
+  else            okm = make_map(&ma, g.A, g.rows, g.K, g.batch, g.a_ld, g.a_bs, 64, BK);
+  if (g.b_kmajor) okm = okm && make_map(&mb, g.B, g.K, g.cols, g.batch, g.b_ld, g.b_bs, BK, BN);
+  else            okm = okm && make_map(&mb, g.B, g.cols, g.K, g.batch, g.b_ld, g.b_bs, 64, BK);
+  if (!okm) return GSHARD_ERR_CUDA;
+  Params p;
+  p.C = g.C; p.mask = g.mask; p.rows = g.rows; p.cols = g.cols; p.K = g.K; p.batch = g.batch;
+  p.c_ld = g.c_ld; p.c_bs = g.c_bs;
+  p.m_tiles = ceil_div(g.rows, BM); p.n_tiles = ceil_div(g.cols, BN);
+  p.total_tiles = p.m_tiles * p.n_tiles * g.batch;
+  p.k_blocks = ceil_div(g.K, BK);
+  p.out_f32 = g.out_f32; p.relu = g.relu; p.a_stream = g.a_stream; p.b_stream = g.b_stream;
+  p.status = status;
+  int sms = 148;
+  int dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = p.total_tiles < sms ? p.total_tiles : sms;
+#define GSHARD_DISPATCH(AK, BKM)                                                         \
+  (BN == 256 ? launch_t<AK, BKM, 256>(g, ma, mb, p, grid, st) : launch_t<AK, BKM, 128>(g, ma, mb, p, grid, st))
+  if (g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH(true, true);
+  if (g.a_kmajor && !g.b_kmajor) return GSHARD_DISPATCH(true, false);
+  if (!g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH(false, true);
+  return GSHARD_DISPATCH(false, false);
+#undef GSHARD_DISPATCH
+}
+
+}  // namespace gshard
