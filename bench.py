@@ -46,7 +46,7 @@ def load_peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons with one looping nvidia-smi while timed regions run."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -54,66 +54,90 @@ class ClockSampler(threading.Thread):
         super().__init__(daemon=True)
         self.index = index
         self.samples = []
-        self.stop_flag = threading.Event()
+        self.proc = None
 
     def run(self):
-        while not self.stop_flag.is_set():
-            try:
-                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
-                parts = [p.strip() for p in out.strip().split(",")]
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "50"], stdout=subprocess.PIPE, text=True)
+            for line in self.proc.stdout:
+                parts = [p.strip() for p in line.strip().split(",")]
                 if len(parts) >= 6:
                     self.samples.append(parts)
-            except Exception:
-                pass
-            self.stop_flag.wait(0.1)
+        except Exception:
+            pass
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()          # the exact process started above
+        self.join(timeout=3)
 
     def summary(self):
-        sm = [float(s[0]) for s in self.samples if s[0].replace(".", "").isdigit()]
-        mx = [float(s[1]) for s in self.samples if s[1].replace(".", "").isdigit()]
+        def num(v):
+            try:
+                return float(v)
+            except ValueError:
+                return None
+        sm = [num(s[0]) for s in self.samples if num(s[0]) is not None]
+        mx = [num(s[1]) for s in self.samples if num(s[1]) is not None]
+        # samples taken while the GPU was busy run well above the idle clock
+        busy = [v for v in sm if v > 500.0] or sm
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         reasons = [n for i, n in enumerate(names) if any(s[2 + i].lower().startswith("active") for s in self.samples)]
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": reasons, "samples": len(self.samples)}
+        return {"sm_mhz": statistics.median(busy) if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(self.samples), "samples_under_load": len(busy)}
 
 
-def oracle_sample(cfg, n_tokens_ffn=24, seed_offset=0):
-    """Times the CPU oracle on a bounded sample of the configuration: gating + Algorithm 1 for one
-    whole group, eq. (2)-(3) for a few of its tokens.  Returns (tokens/s of a full layer at that
-    per-token cost, description, threads)."""
-    import numpy as np
+def oracle_sample(cfg, n_groups=8, n_rows=400, seed_offset=0):
+    """Times the CPU oracle on a bounded sample of the configuration: gating + Algorithm 1 for
+    n_groups whole groups, eq. (2)-(3) for n_rows token-expert rows of those groups.  Returns
+    (tokens/s of a full layer at that per-token cost, description, threads)."""
     import torch
     from oracle import gshard_oracle as orc
     from paper_2006_16668_b200.inputs import make_inputs
 
-    small = cfg.scaled(G=1)                                   # one group of the same S, M, E
+    n_groups = min(n_groups, cfg.G)
+    small = cfg.scaled(G=n_groups, seed=cfg.seed + seed_offset)     # groups of the same S, M, E
     inp = make_inputs(small, "cpu", with_experts=False)
-    x = inp["x"][0].float().numpy()
+    x = inp["x"].float().numpy()
     wg = inp["wg"].float().numpy()
-    u = inp["u"][0].numpy()
-    t0 = time.perf_counter()
-    _, p = orc.gates(x, wg)
-    m = orc.mean_gates(p)
-    e1, e2, g1, g2, _ = orc.top2(p)
-    r = orc.capacity(cfg.E, cfg.C, e1, e2, g1, g2, u, m)
-    t_gate = time.perf_counter() - t0
-    # expert FFN for a few tokens; weights of the needed experts drawn with the recipe's scales
+    u = inp["u"].numpy()
+    # a few experts' weights drawn with the recipe's scales; rows cycle through them
     gen = torch.Generator().manual_seed(cfg.seed + 99 + seed_offset)
+    experts = []
+    for _ in range(4):
+        wi_e = (torch.randn(cfg.M, cfg.H, generator=gen) * cfg.M ** -0.5).to(cfg.torch_dtype).float().numpy()
+        wo_e = (torch.randn(cfg.H, cfg.M, generator=gen) * cfg.H ** -0.5).to(cfg.torch_dtype).float().numpy()
+        experts.append((wi_e, wo_e))
+    t_gate = 0.0
+    kept = 0
+    routings = []
+    for g in range(n_groups):
+        t0 = time.perf_counter()
+        _, p = orc.gates(x[g], wg)
+        m = orc.mean_gates(p)
+        e1, e2, g1, g2, _ = orc.top2(p)
+        r = orc.capacity(cfg.E, cfg.C, e1, e2, g1, g2, u[g], m)
+        t_gate += time.perf_counter() - t0
+        kept += int((r.slot >= 0).sum())
+        routings.append(r)
     rows = 0
     t_ffn = 0.0
-    for s in range(min(n_tokens_ffn, cfg.S)):
-        for k in range(2):
-            if r.slot[s, k] < 0:
-                continue
-            wi_e = (torch.randn(cfg.M, cfg.H, generator=gen) * cfg.M ** -0.5).to(cfg.torch_dtype).float().numpy()
-            wo_e = (torch.randn(cfg.H, cfg.M, generator=gen) * cfg.H ** -0.5).to(cfg.torch_dtype).float().numpy()
-            t1 = time.perf_counter()
-            orc.ffn_rows(x[s:s + 1], wi_e, wo_e)
-            t_ffn += time.perf_counter() - t1
-            rows += 1
-    kept_per_token = float((r.slot >= 0).sum()) / cfg.S
-    per_token = t_gate / cfg.S + (t_ffn / max(rows, 1)) * kept_per_token
-    desc = (f"gating+Algorithm 1 for 1 group of {cfg.S} tokens ({t_gate:.2f} s) + eq.(2)-(3) for {rows} "
+    s = 0
+    while rows < n_rows and s < cfg.S:
+        for g in range(n_groups):
+            for k in range(2):
+                if routings[g].slot[s, k] < 0 or rows >= n_rows:
+                    continue
+                wi_e, wo_e = experts[rows % len(experts)]
+                t1 = time.perf_counter()
+                orc.ffn_rows(x[g, s:s + 1], wi_e, wo_e)
+                t_ffn += time.perf_counter() - t1
+                rows += 1
+        s += 1
+    kept_per_token = kept / float(n_groups * cfg.S)
+    per_token = t_gate / (n_groups * cfg.S) + (t_ffn / max(rows, 1)) * kept_per_token
+    desc = (f"gating+Algorithm 1 for {n_groups} groups of {cfg.S} tokens ({t_gate:.2f} s) + eq.(2)-(3) for {rows} "
             f"token-expert rows ({t_ffn:.2f} s); tokens/s extrapolated at {kept_per_token:.2f} kept choices/token")
     return 1.0 / per_token, desc, orc.num_threads()
 
@@ -126,7 +150,7 @@ def run_reference(args, cfg):
     vals = []
     desc, cores = "", 0
     for i in range(args.warmup + args.steps):
-        v, desc, cores = oracle_sample(cfg, n_tokens_ffn=8, seed_offset=i)
+        v, desc, cores = oracle_sample(cfg, n_groups=2, n_rows=64, seed_offset=i)
         if i >= args.warmup:
             vals.append(v)
     value = statistics.mean(vals)
@@ -144,7 +168,7 @@ def run_reference(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--config", default="c4_2048e")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -209,8 +233,6 @@ def main():
         ev[i + 1].record(stream)
     barrier()
     total_ms = ev[0].elapsed_time(ev[-1])
-    sampler.stop_flag.set()
-    sampler.join(timeout=2)
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -280,6 +302,7 @@ def main():
         v, desc, cores = oracle_sample(cfg)
         cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
 
+    sampler.stop()
     if rank == 0:
         stats = rt["stats"].cpu().tolist()
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

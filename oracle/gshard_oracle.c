@@ -259,10 +259,63 @@ double gso_forward(int G, int S, int M, int H, int E, int C, const float* x,
  * Expert path for a kept choice with weight w: dout = w dy_s,
  *   dh = (dout . wo_e^T) * 1[pre-activation > 0], dwo_e += relu(h)^T dout,
  *   dwi_e += x_s^T dh, dx_s += dh . wi_e^T.
- *
- * Inputs are the forward inputs plus the oracle's own routing (expert_idx,
- * slot, first_count).  Outputs: dx [G,S,M], dwg [M,E], dwi [E,M,H], dwo [E,H,M].
  */
+
+/* Expert path backward for `rows` rows of ONE expert (eq. (2) differentiated):
+ * xrows [rows,M] inputs, dout [rows,M] upstream gradient of FFN_e's output.
+ * ACCUMULATES into dxrows [rows,M], dwi_e [M,H], dwo_e [H,M]. */
+void gso_ffn_rows_backward(const float* xrows, const double* dout, int rows, const float* wi_e,
+                           const float* wo_e, int M, int H, double* dxrows, double* dwi_e,
+                           double* dwo_e) {
+  double* hpre = (double*)malloc(sizeof(double) * (size_t)H);
+  double* dh = (double*)malloc(sizeof(double) * (size_t)H);
+  double* o = (double*)malloc(sizeof(double) * (size_t)M);
+  for (int r = 0; r < rows; ++r) {
+    const float* xs = xrows + (size_t)r * M;
+    const double* dor = dout + (size_t)r * M;
+    gso_ffn_rows(xs, 1, wi_e, wo_e, M, H, o, hpre);
+#pragma omp parallel for schedule(static)
+    for (int j = 0; j < H; ++j) {
+      double acc = 0.0;
+      const double act = hpre[j] > 0.0 ? hpre[j] : 0.0;
+      for (int i = 0; i < M; ++i) {
+        acc += dor[i] * (double)wo_e[(size_t)j * M + i];
+        dwo_e[(size_t)j * M + i] += act * dor[i];
+      }
+      dh[j] = hpre[j] > 0.0 ? acc : 0.0;
+    }
+#pragma omp parallel for schedule(static)
+    for (int mm = 0; mm < M; ++mm) {
+      double acc = 0.0;
+      for (int j = 0; j < H; ++j) {
+        dwi_e[(size_t)mm * H + j] += (double)xs[mm] * dh[j];
+        acc += dh[j] * (double)wi_e[(size_t)mm * H + j];
+      }
+      dxrows[(size_t)r * M + mm] += acc;
+    }
+  }
+  free(hpre); free(dh); free(o);
+}
+
+/* Gate backward for ONE token: p [E] its softmax gates, (e1,e2) its top-2, dw1/dw2 the
+ * gradients of its two combine weights (0 for a dropped choice), first_count_g [E] the
+ * group's c_e.  Writes dlogit [E]. */
+void gso_gate_row_backward(const double* p, int E, int e1, int e2, double dw1, double dw2,
+                           const int32_t* first_count_g, int S, int G, double k_aux,
+                           double* dlogit) {
+  const double a = p[e1], b = p[e2], D = a + b;
+  for (int e = 0; e < E; ++e)
+    dlogit[e] = k_aux * (1.0 / G) * (1.0 / E) * ((double)first_count_g[e] / (double)S) * (1.0 / S);
+  dlogit[e1] += (b / (D * D)) * (dw1 - dw2);
+  dlogit[e2] += (a / (D * D)) * (dw2 - dw1);
+  double dot = 0.0;
+  for (int e = 0; e < E; ++e) dot += p[e] * dlogit[e];
+  for (int e = 0; e < E; ++e) dlogit[e] = p[e] * (dlogit[e] - dot);
+}
+
+/* Whole-layer backward.  Inputs are the forward inputs plus the frozen routing
+ * (expert_idx, slot, first_count).  Outputs: dx [G,S,M], dwg [M,E], dwi [E,M,H],
+ * dwo [E,H,M]. */
 void gso_backward(int G, int S, int M, int H, int E, int C, const float* x,
                   const float* wg, const float* wi, const float* wo,
                   const int32_t* expert_idx, const int32_t* slot,
@@ -275,10 +328,9 @@ void gso_backward(int G, int S, int M, int H, int E, int C, const float* x,
   memset(dwi, 0, sizeof(double) * (size_t)E * M * H);
   memset(dwo, 0, sizeof(double) * (size_t)E * H * M);
   double* p = (double*)malloc(sizeof(double) * (size_t)S * E);
-  double* dg = (double*)malloc(sizeof(double) * (size_t)E);
-  double* hpre = (double*)malloc(sizeof(double) * (size_t)H);
-  double* o = (double*)malloc(sizeof(double) * (size_t)M * 2);
-  double* dh = (double*)malloc(sizeof(double) * (size_t)H);
+  double* dlogit = (double*)malloc(sizeof(double) * (size_t)E);
+  double* o = (double*)malloc(sizeof(double) * (size_t)M);
+  double* dout = (double*)malloc(sizeof(double) * (size_t)M);
   for (int g = 0; g < G; ++g) {
     gso_gates(x + (size_t)g * S * M, wg, S, M, E, NULL, p);
     for (int s = 0; s < S; ++s) {
@@ -290,52 +342,26 @@ void gso_backward(int G, int S, int M, int H, int E, int C, const float* x,
       const double a = ps[ea], b = ps[eb], D = a + b;
       const double wgt[2] = {a / D, b / D};
       double dw[2] = {0.0, 0.0};
-      /* expert path, one kept choice at a time */
       for (int k = 0; k < 2; ++k) {
         if (slot[2 * t + k] < 0) continue;
         const int32_t e = k ? eb : ea;
         const float* wie = wi + (size_t)e * M * H;
         const float* woe = wo + (size_t)e * H * M;
-        gso_ffn_rows(xs, 1, wie, woe, M, H, o + (size_t)k * M, hpre);
-        for (int i = 0; i < M; ++i) dw[k] += (double)dys[i] * o[(size_t)k * M + i];
-        /* dout = w * dy ; dh = (dout . wo^T) masked ; dwo += relu(h)^T dout */
-        for (int j = 0; j < H; ++j) {
-          double acc = 0.0;
-          const double act = hpre[j] > 0.0 ? hpre[j] : 0.0;
-          for (int i = 0; i < M; ++i) {
-            const double dout = wgt[k] * (double)dys[i];
-            acc += dout * (double)woe[(size_t)j * M + i];
-            dwo[((size_t)e * H + j) * M + i] += act * dout;
-          }
-          dh[j] = hpre[j] > 0.0 ? acc : 0.0;
-        }
-        for (int mm = 0; mm < M; ++mm) {
-          double acc = 0.0;
-          for (int j = 0; j < H; ++j) {
-            dwi[((size_t)e * M + mm) * H + j] += (double)xs[mm] * dh[j];
-            acc += dh[j] * (double)wie[(size_t)mm * H + j];
-          }
-          dx[t * M + mm] += acc;
-        }
+        gso_ffn_rows(xs, 1, wie, woe, M, H, o, NULL);
+        for (int i = 0; i < M; ++i) { dw[k] += (double)dys[i] * o[i]; dout[i] = wgt[k] * (double)dys[i]; }
+        gso_ffn_rows_backward(xs, dout, 1, wie, woe, M, H, dx + t * M,
+                              dwi + (size_t)e * M * H, dwo + (size_t)e * H * M);
       }
-      /* gate gradient: combine weights + dense aux term */
-      for (int e = 0; e < E; ++e)
-        dg[e] = k_aux * (1.0 / G) * (1.0 / E) *
-                ((double)first_count[(size_t)g * E + e] / (double)S) * (1.0 / S);
-      dg[ea] += (b / (D * D)) * (dw[0] - dw[1]);
-      dg[eb] += (a / (D * D)) * (dw[1] - dw[0]);
-      double dot = 0.0;
-      for (int e = 0; e < E; ++e) dot += ps[e] * dg[e];
-      for (int e = 0; e < E; ++e) dg[e] = ps[e] * (dg[e] - dot);   /* now dlogit */
+      gso_gate_row_backward(ps, E, ea, eb, dw[0], dw[1], first_count + (size_t)g * E, S, G, k_aux, dlogit);
       for (int mm = 0; mm < M; ++mm) {
         double acc = 0.0;
         for (int e = 0; e < E; ++e) {
-          dwg[(size_t)mm * E + e] += (double)xs[mm] * dg[e];
-          acc += dg[e] * (double)wg[(size_t)mm * E + e];
+          dwg[(size_t)mm * E + e] += (double)xs[mm] * dlogit[e];
+          acc += dlogit[e] * (double)wg[(size_t)mm * E + e];
         }
         dx[t * M + mm] += acc;
       }
     }
   }
-  free(p); free(dg); free(hpre); free(o); free(dh);
+  free(p); free(dlogit); free(o); free(dout);
 }

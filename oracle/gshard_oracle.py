@@ -185,6 +185,31 @@ def forward(x, wg, wi, wo, u, C, variant_a=False, want_y=True) -> Forward:
     return Forward(y, float(la), ei, slot, weight, flags, fc, tc, st, m, lg)
 
 
+def ffn_rows_backward(xrows, dout, wi_e, wo_e):
+    """Expert path backward for the rows of one expert -> (dxrows, dwi_e, dwo_e) float64."""
+    xrows, wi_e, wo_e = _f32(xrows), _f32(wi_e), _f32(wo_e)
+    dout = np.ascontiguousarray(dout, np.float64)
+    R, M = xrows.shape
+    H = wi_e.shape[1]
+    dxr = np.zeros((R, M), np.float64)
+    dwi = np.zeros((M, H), np.float64)
+    dwo = np.zeros((H, M), np.float64)
+    lib().gso_ffn_rows_backward(_ptr(xrows, c_f), _ptr(dout, c_d), R, _ptr(wi_e, c_f), _ptr(wo_e, c_f), M, H,
+                                _ptr(dxr, c_d), _ptr(dwi, c_d), _ptr(dwo, c_d))
+    return dxr, dwi, dwo
+
+
+def gate_row_backward(p_row, e1, e2, dw1, dw2, first_count_g, S, G, k_aux):
+    """Softmax/aux-loss backward of one token -> dlogit [E] float64."""
+    p_row = np.ascontiguousarray(p_row, np.float64)
+    fc = np.ascontiguousarray(first_count_g, np.int32)
+    E = p_row.shape[0]
+    dl = np.empty(E, np.float64)
+    lib().gso_gate_row_backward(_ptr(p_row, c_d), E, int(e1), int(e2), ctypes.c_double(dw1), ctypes.c_double(dw2),
+                                _ptr(fc, c_i), int(S), int(G), ctypes.c_double(k_aux), _ptr(dl, c_d))
+    return dl
+
+
 def backward(x, wg, wi, wo, fwd: Forward, dy, k_aux):
     """Gradients of <dy,y> + k_aux*l_aux with fwd's routing frozen -> dx, dwg, dwi, dwo."""
     x, wg, wi, wo, dy = _f32(x), _f32(wg), _f32(wi), _f32(wo), _f32(dy)

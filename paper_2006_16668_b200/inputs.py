@@ -63,6 +63,9 @@ CONFIGS = {
     "c3_512e_skew": MoEConfig("c3_512e_skew", G=16, S=4096, M=1024, H=8192, E=512, C=16,
                               seed=20200633, skew=True),
     "c4_2048e": MoEConfig("c4_2048e", G=32, S=4096, M=1024, H=8192, E=2048, C=4, seed=20200634),
+    # a 64-expert slice of the MoE(2048E) layer (same per-expert shapes: 128 rows, M=1024, H=8192,
+    # C=4; 2.1 GB of expert weights) - the small case profiler captures run on
+    "p4_slice": MoEConfig("p4_slice", G=32, S=128, M=1024, H=8192, E=64, C=4, seed=20200636),
     # configs[4]: training step
     "c5_512e_train": MoEConfig("c5_512e_train", G=16, S=4096, M=1024, H=8192, E=512, C=16,
                                seed=20200635, backward=True),
