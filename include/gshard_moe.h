@@ -153,6 +153,28 @@ int gshard_moe_capacity(const gshard_moe_shape* shape, const int32_t* expert_idx
                         const gshard_moe_routing* routing_out, float* l_aux, void* workspace,
                         size_t workspace_bytes, void* cuda_stream);
 
+/* gshard_moe_capacity for callers that cannot allocate device memory (the paper has no
+ * counterpart: this is an interface variant, not a different computation).
+ * Who needs it: code that runs where no device allocation is possible at call time - an operator
+ * inside a host runtime that owns the allocator and forbids allocating in its execute hook, a
+ * serving loop whose memory pool is frozen after start-up - and that therefore cannot hand over a
+ * workspace either.  The per-group statistics scratch of the capacity kernel then lives in a
+ * 128 KB array built into the library image (held by every GPU that loads the library until
+ * the process exits), which limits this variant to G <= 4096 groups: a larger G returns
+ * GSHARD_ERR_UNSUPPORTED_SHAPE and launches nothing.
+ * Arguments as gshard_moe_capacity, except that there is no workspace, so routing_out and its
+ * slot, weight, flags, first_count, total_count, slot_token and l_aux_group must all be given
+ * (stats and l_aux stay optional).  The call allocates nothing and calls no allocating routine.
+ * The first call on each device looks up the array's device address (the device must be
+ * current); make that first call before any stream capture begins.  All calls on a device share
+ * the one array: the kernel rewrites every entry it later reads, so nothing needs clearing
+ * between calls, but two calls whose kernels overlap on the GPU (different streams) race on it;
+ * keep them on one stream or order them yourself.  Results equal gshard_moe_capacity's. */
+int gshard_moe_capacity_static(const gshard_moe_shape* shape, const int32_t* expert_idx,
+                               const float* gate12, const float* u, const float* m,
+                               const gshard_moe_routing* routing_out, float* l_aux,
+                               void* cuda_stream);
+
 /* Algorithm 2 dispatch as an index gather: buf[e, g*C+c, :] = x[g, slot_token[e,g,c], :],
  * zero row for an empty slot.  buf [E, G*C, M] dtype. */
 int gshard_moe_dispatch(const gshard_moe_shape* shape, const void* x, const int32_t* slot_token,

@@ -56,6 +56,8 @@ EXPORTS = {
     "gshard_moe_gate": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6 + [c_size_t, c_void_p]),
     "gshard_moe_capacity": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 4 +
                             [POINTER(gshard_moe_routing), c_void_p, c_void_p, c_size_t, c_void_p]),
+    "gshard_moe_capacity_static": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 4 +
+                                   [POINTER(gshard_moe_routing), c_void_p, c_void_p]),
     "gshard_moe_dispatch": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 4),
     "gshard_moe_expert_ffn": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 5 + [c_size_t, c_void_p]),
     "gshard_moe_combine": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6),
@@ -203,6 +205,14 @@ def gshard_moe_capacity(shape, expert_idx, gate12, u, m, routing_out, l_aux, wor
     _check(load().gshard_moe_capacity(ctypes.byref(shape), _p(expert_idx), _p(gate12), _p(u), _p(m),
                                       ctypes.byref(routing_out), _p(l_aux), _p(workspace), workspace.numel(),
                                       _stream(stream)), "gshard_moe_capacity")
+
+
+def gshard_moe_capacity_static(shape, expert_idx, gate12, u, m, routing_out, l_aux, stream=None):
+    """Capacity assignment without a workspace: for callers that cannot allocate device memory
+    (scratch is a fixed array inside the library; G <= 4096; every routing output required)."""
+    _check(load().gshard_moe_capacity_static(ctypes.byref(shape), _p(expert_idx), _p(gate12), _p(u), _p(m),
+                                             ctypes.byref(routing_out), _p(l_aux), _stream(stream)),
+           "gshard_moe_capacity_static")
 
 
 def gshard_moe_dispatch(shape, x, slot_token, buf, stream=None):

@@ -8,6 +8,7 @@
 // exclusive scan over the warps' histograms (per expert, in warp order) gives each chunk's
 // offset.  Compact index lists are written; the dense [G,S,E,C] masks never exist.
 #include "kernels.cuh"
+#include "plan.cuh"
 
 namespace gshard {
 
@@ -226,3 +227,69 @@ int launch_capacity(const Dims& d, const int32_t* expert_idx, const float* gate1
 }
 
 }  // namespace gshard
+
+// ---------------------------------------------------------------------------------------------
+// Capacity assignment for callers that cannot allocate device memory.
+//
+// The regular entry point takes its scratch (the per-group statistics block, and any routing
+// output the caller left out) from a caller-supplied workspace.  Some callers have no way to
+// provide one: an operator plugged into a host runtime that owns the allocator and forbids
+// allocation inside its execute hook, or a serving loop whose memory pool is frozen after
+// start-up.  For them the scratch below is part of the library image itself: every GPU that
+// loads the library holds these 128 KB until the process exits.
+namespace gshard {
+constexpr int kStaticMaxGroups = 4096;                       // G limit of the static variant
+static __device__ __align__(256) int32_t g_static_stats_group[kStaticMaxGroups * 8];
+
+namespace {
+// In host code the array's name above is only a host-side stand-in, not a device address; the
+// address a kernel can use comes from cudaGetSymbolAddress, asked once per device with that
+// device current.
+int static_scratch_for_current_device(int32_t** out) {
+  constexpr int kMaxDevices = 64;
+  static int32_t* ptrs[kMaxDevices] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return GSHARD_ERR_CUDA; }
+  if (dev < 0 || dev >= kMaxDevices) return GSHARD_ERR_INTERNAL;
+  if (ptrs[dev] == nullptr) {
+    int32_t* p = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_stats_group) != cudaSuccess || p == nullptr) {
+      cudaGetLastError();
+      return GSHARD_ERR_CUDA;
+    }
+    ptrs[dev] = p;     // same value whichever thread stores it
+  }
+  *out = ptrs[dev];
+  return GSHARD_OK;
+}
+}  // namespace
+}  // namespace gshard
+
+extern "C" int gshard_moe_capacity_static(const gshard_moe_shape* shape, const int32_t* expert_idx,
+                                          const float* gate12, const float* u, const float* m,
+                                          const gshard_moe_routing* routing_out, float* l_aux,
+                                          void* cuda_stream) {
+  using namespace gshard;
+  launch_counter().n = 0;
+  const int rc = validate_shape(shape);
+  if (rc != GSHARD_OK) return rc;
+  if (shape->G > kStaticMaxGroups) return GSHARD_ERR_UNSUPPORTED_SHAPE;   // beyond the built-in scratch
+  auto bad = [](const void* p) { return p == nullptr || (reinterpret_cast<uintptr_t>(p) & 15u) != 0; };
+  if (bad(expert_idx) || bad(gate12) || bad(u) || bad(m) || routing_out == nullptr) return GSHARD_ERR_INVALID_ARG;
+  const gshard_moe_routing& r = *routing_out;
+  // no workspace to fall back on: every tensor the kernel writes must be the caller's
+  if (!r.slot || !r.weight || !r.flags || !r.first_count || !r.total_count || !r.slot_token || !r.l_aux_group)
+    return GSHARD_ERR_INVALID_ARG;
+  int major = 0, dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return GSHARD_ERR_CUDA; }
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return GSHARD_ERR_CUDA;
+  if (major != 10) return GSHARD_ERR_ARCH;
+  int32_t* stats_group = nullptr;
+  const int src = static_scratch_for_current_device(&stats_group);
+  if (src != GSHARD_OK) return src;
+  // The kernel overwrites all 8 statistics of each of its G groups before the finalize kernel
+  // reads them, so nothing in the shared array has to be cleared between calls.
+  return launch_capacity(make_dims(*shape), expert_idx, gate12, u, m, r.slot, r.weight, r.flags, r.first_count,
+                         r.total_count, r.slot_token, r.l_aux_group, stats_group, l_aux,
+                         reinterpret_cast<long long*>(r.stats), static_cast<cudaStream_t>(cuda_stream));
+}

@@ -1,0 +1,68 @@
+"""gshard_moe_capacity_static: the capacity stage for callers that cannot allocate device memory
+(an operator inside a runtime that forbids allocation in its execute hook, a serving loop with a
+frozen memory pool).  Its scratch is a fixed array inside the library, shared by every call, so
+the check runs the entry point twice in a row - on different inputs - and compares each result
+with the workspace-based gshard_moe_capacity.  Integer outputs must be identical; float outputs
+are held to the 1e-5 relative tolerance the other capacity tests use (they are in fact the same
+kernel on the same numbers).  This file is named to be collected last."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2006_16668_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+
+
+def _inputs(G, S, E, seed):
+    rng = np.random.default_rng(seed)
+    pop = rng.dirichlet(np.ones(E) * 0.5)
+    e1 = rng.choice(E, size=(G, S), p=pop)
+    e2 = (e1 + 1 + rng.integers(0, E - 1, size=(G, S))) % E
+    ga = rng.random((G, S), dtype=np.float32) * 0.5 + 1e-3
+    gb = np.maximum(ga * rng.random((G, S), dtype=np.float32), np.float32(1e-6))
+    t = lambda a, dt: torch.from_numpy(np.ascontiguousarray(a).astype(dt)).cuda()
+    return (t(np.stack([e1, e2], -1), np.int32), t(np.stack([ga, gb], -1), np.float32),
+            t(rng.random((G, S)), np.float32), t(rng.dirichlet(np.ones(E), size=G), np.float32))
+
+
+def _run(shape, inputs, static):
+    ei, g12, u, m = inputs
+    rt, rs = B.alloc_routing(shape)
+    l_aux = torch.zeros(1, device="cuda")
+    if static:
+        B.gshard_moe_capacity_static(shape, ei, g12, u, m, rs, l_aux)
+    else:
+        ws = B.alloc_workspace(shape)
+        B.gshard_moe_capacity(shape, ei, g12, u, m, rs, l_aux, ws)
+    torch.cuda.synchronize()
+    return rt, l_aux
+
+
+def test_static_capacity_matches_workspace_capacity_twice():
+    G, S, E, C = 6, 700, 96, 9
+    shape = B.make_shape(G=G, S=S, M=8, H=8, E=E, C=C, dtype="f32")
+    for call, seed in enumerate((101, 202)):          # two calls in a row share the static scratch
+        inputs = _inputs(G, S, E, seed)
+        ref, ref_aux = _run(shape, inputs, static=False)
+        got, got_aux = _run(shape, inputs, static=True)
+        for k in ("slot", "flags", "first_count", "total_count", "slot_token", "stats"):
+            assert torch.equal(got[k], ref[k]), (call, k)
+        for k in ("weight", "l_aux_group"):
+            torch.testing.assert_close(got[k], ref[k], rtol=1e-5, atol=0)
+        torch.testing.assert_close(got_aux, ref_aux, rtol=1e-5, atol=0)
+        assert int(got["stats"][4]) == int((got["slot"] >= 0).sum()) > 0
+
+
+def test_static_capacity_rejects_what_it_cannot_hold():
+    ok = B.make_shape(G=2, S=64, M=8, H=8, E=8, C=4, dtype="f32")
+    inputs = _inputs(2, 64, 8, 1)
+    big = B.make_shape(G=4097, S=64, M=8, H=8, E=8, C=4, dtype="f32")
+    rt, rs = B.alloc_routing(ok)
+    with pytest.raises(B.GshardError) as e:
+        B.gshard_moe_capacity_static(big, *inputs, rs, None)
+    assert e.value.code == B.GSHARD_ERR_UNSUPPORTED_SHAPE
+    rt.pop("slot")                                    # a required output is missing
+    with pytest.raises(B.GshardError) as e:
+        B.gshard_moe_capacity_static(ok, *inputs, B.routing_struct(rt), None)
+    assert e.value.code == B.GSHARD_ERR_INVALID_ARG
