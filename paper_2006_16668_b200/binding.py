@@ -28,6 +28,7 @@ GSHARD_BF16 = 1
 GSHARD_FLAG_SAVE_FOR_BACKWARD = 1
 GSHARD_FLAG_SECOND_SKIP_FREES_SLOT = 2
 GSHARD_FLAG_SIMT_CONTRACTIONS = 4
+GSHARD_FLAG_FUSED_FFN = 8
 
 
 class gshard_moe_shape(Structure):

@@ -41,6 +41,7 @@ struct Dims {
   bool bf16;
   bool simt;            // contractions on CUDA cores
   bool variant_a;
+  bool fused_ffn;       // experimental single-launch FFN with h in an L2-resident ring
 };
 
 inline Dims make_dims(const gshard_moe_shape& s) {
@@ -54,6 +55,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.esize = d.bf16 ? 2 : 4;
   d.simt = !d.bf16 || (s.flags & GSHARD_FLAG_SIMT_CONTRACTIONS);
   d.variant_a = (s.flags & GSHARD_FLAG_SECOND_SKIP_FREES_SLOT) != 0;
+  d.fused_ffn = (s.flags & GSHARD_FLAG_FUSED_FFN) != 0;
   return d;
 }
 

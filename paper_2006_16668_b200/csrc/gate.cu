@@ -108,16 +108,70 @@ __global__ void __launch_bounds__(128) gate_mean_kernel(const float* __restrict_
   m[(long long)g * E + e] = acc / (float)S;
 }
 
+// Same column sums with four experts per thread (16-byte loads, four rows in flight): the
+// bandwidth-bound form used whenever E is a multiple of 4.  Rows are added in ascending order.
+__global__ void __launch_bounds__(128) gate_colsum4_kernel(const float4* __restrict__ logits,
+                                                           const float* __restrict__ rowmax,
+                                                           const float* __restrict__ rowinv, int S,
+                                                           int E4, int tiles_per_group,
+                                                           float4* __restrict__ partial) {
+  const int e4 = blockIdx.x * blockDim.x + threadIdx.x;
+  const int tile = blockIdx.y;
+  const int g = tile / tiles_per_group;
+  const int s0 = (tile % tiles_per_group) * kGateTile;
+  const int n = min(S, s0 + kGateTile) - s0;
+  __shared__ float smax[kGateTile], sinv[kGateTile];
+  for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    smax[i] = rowmax[(long long)g * S + s0 + i];
+    sinv[i] = rowinv[(long long)g * S + s0 + i];
+  }
+  __syncthreads();
+  if (e4 >= E4) return;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  const float4* base = logits + ((long long)g * S + s0) * E4 + e4;
+  int i = 0;
+  for (; i + 4 <= n; i += 4) {
+    float4 v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = __ldcs(base + (long long)(i + j) * E4);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float mx = smax[i + j], iv = sinv[i + j];
+      acc.x += expf(v[j].x - mx) * iv; acc.y += expf(v[j].y - mx) * iv;
+      acc.z += expf(v[j].z - mx) * iv; acc.w += expf(v[j].w - mx) * iv;
+    }
+  }
+  for (; i < n; ++i) {
+    const float4 v = __ldcs(base + (long long)i * E4);
+    const float mx = smax[i], iv = sinv[i];
+    acc.x += expf(v.x - mx) * iv; acc.y += expf(v.y - mx) * iv;
+    acc.z += expf(v.z - mx) * iv; acc.w += expf(v.w - mx) * iv;
+  }
+  partial[(long long)tile * E4 + e4] = acc;
+}
+
 void launch_gate_rows(const Dims& d, const float* logits, int32_t* expert_idx, float* gate12,
-                      float* rowmax, float* rowinv, float* partial, float* m, cudaStream_t st) {
+                      float* rowmax, float* rowinv, cudaStream_t st) {
   const long long warps_needed = d.N;
   int blocks = (int)((warps_needed + 7) / 8);
   if (blocks > 148 * 16) blocks = 148 * 16;
   gate_rows_kernel<<<blocks, 256, 0, st>>>(logits, d.N, d.E, expert_idx, gate12, rowmax, rowinv);
-  dim3 grid(ceil_div(d.E, 128), d.G * d.tiles_per_group);
-  gate_colsum_kernel<<<grid, 128, 0, st>>>(logits, rowmax, rowinv, d.S, d.E, d.tiles_per_group, partial);
+  count_launch();
+}
+
+// m[g,e] from stored logits and row statistics (two launches).
+void launch_gate_means(const Dims& d, const float* logits, const float* rowmax, const float* rowinv,
+                       float* partial, float* m, cudaStream_t st) {
+  if (d.E % 4 == 0) {
+    dim3 grid(ceil_div(d.E / 4, 128), d.G * d.tiles_per_group);
+    gate_colsum4_kernel<<<grid, 128, 0, st>>>(reinterpret_cast<const float4*>(logits), rowmax, rowinv, d.S, d.E / 4,
+                                              d.tiles_per_group, reinterpret_cast<float4*>(partial));
+  } else {
+    dim3 grid(ceil_div(d.E, 128), d.G * d.tiles_per_group);
+    gate_colsum_kernel<<<grid, 128, 0, st>>>(logits, rowmax, rowinv, d.S, d.E, d.tiles_per_group, partial);
+  }
   gate_mean_kernel<<<dim3(ceil_div(d.E, 128), d.G), 128, 0, st>>>(partial, d.S, d.E, d.tiles_per_group, m);
-  count_launch(3);
+  count_launch(2);
 }
 
 }  // namespace gshard

@@ -1,0 +1,241 @@
+// Gating for the bf16 dtype in one tensor-core kernel (Algorithm 1: "g <- softmax(wg . x)" and
+// "top_2"): logits = x . wg on tcgen05 with fp32 accumulation, and in the epilogue - while the
+// accumulator is read out of tensor memory - the running row maximum, the running sum of
+// exponentials (online softmax) and the two largest logits with their expert indices (softmax is
+// monotone, so top-2 of the gates is top-2 of the logits; scanning experts in ascending order with
+// strict comparisons makes the lowest index win ties).
+//
+// A persistent CTA owns a tile of 128 tokens and walks all expert-column tiles of that row tile,
+// so x is streamed from HBM once (the 128 x M panel is re-read from L2 per column tile) and the
+// per-token state lives in the registers of the epilogue thread that owns the token's TMEM lane.
+// The fp32 logits are also stored: the mean gates m_e need the final row normaliser and are
+// summed by a second, bandwidth-bound pass (gate.cu).
+#include <cuda.h>
+
+#include "kernels.cuh"
+#include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
+
+namespace gshard {
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int kThreads = 192;
+constexpr int kABytes = BM * BK * 2;
+constexpr int kBBytes = BN * BK * 2;
+constexpr int kBoxBytes = 64 * 64 * 2;
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kStages = 4;
+constexpr int kTmemCols = 2 * BN;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+
+struct GateParams {
+  long long N;          // tokens
+  int E, M;
+  int row_tiles, n_tiles, k_blocks;
+  float* logits;        // [N,E] fp32
+  int32_t* expert_idx;  // [N,2]
+  float* gate12;        // [N,2] raw softmax values of the two picks
+  float* rowmax;        // [N]
+  float* rowinv;        // [N] 1 / sum exp(logit - rowmax)
+  int* status;
+};
+
+__device__ __forceinline__ int tile_cols(const GateParams& p, int nt) {   // multiple of 16, <= BN
+  const int left = p.E - nt * BN;
+  const int c = left < BN ? left : BN;
+  return (c + 15) & ~15;
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_wg,
+                  const GateParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * kStageBytes);
+  uint64_t* full = bars;
+  uint64_t* empty = bars + kStages;
+  uint64_t* acc_full = bars + 2 * kStages;
+  uint64_t* acc_empty = acc_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(full + s, 1); ptx::mbar_init(empty + s, 1); }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full + a, 1); ptx::mbar_init(acc_empty + a, 4); }
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&map_x);
+    ptx::prefetch_tensormap(&map_wg);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  bool ok = true;
+  if (warp == 0) {
+    if (lane == 0) {
+      const uint64_t pol_x = ptx::policy_evict_first();    // each row panel is used by one CTA only
+      const uint64_t pol_w = ptx::policy_evict_last();     // wg is shared by every CTA
+      int stage = 0; uint32_t phase = 0;
+      for (int rt = blockIdx.x; rt < p.row_tiles && ok; rt += gridDim.x) {
+        for (int nt = 0; nt < p.n_tiles && ok; ++nt) {
+          const int boxes = (tile_cols(p, nt) + 63) / 64;
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            if (!ptx::mbar_wait(empty + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+            unsigned char* sa = smem + stage * kStageBytes;
+            unsigned char* sb = sa + kABytes;
+            ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)(kABytes + boxes * kBoxBytes));
+            ptx::tma_load_3d(sa, &map_x, full + stage, kb * BK, rt * BM, 0, pol_x);
+            for (int j = 0; j < boxes; ++j)
+              ptx::tma_load_3d(sb + j * kBoxBytes, &map_wg, full + stage, nt * BN + j * 64, kb * BK, 0, pol_w);
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      for (int rt = blockIdx.x; rt < p.row_tiles && ok; rt += gridDim.x) {
+        for (int nt = 0; nt < p.n_tiles && ok; ++nt) {
+          const uint32_t idesc = ptx::make_idesc_bf16(BM, tile_cols(p, nt), false, true);
+          if (!ptx::mbar_wait(acc_empty + acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after_sync();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            if (!ptx::mbar_wait(full + stage, phase, abort_flag)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            const uint32_t sa = ptx::smem_u32(smem + stage * kStageBytes);
+            const uint32_t sb = sa + kABytes;
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k) {
+              const uint64_t da = ptx::make_smem_desc(sa + k * 32, 16, 1024);
+              const uint64_t db = ptx::make_smem_desc(sb + k * 2048, kBoxBytes, 1024);
+              ptx::umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            ptx::umma_commit(empty + stage);
+            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          }
+          if (!ok) break;
+          ptx::umma_commit(acc_full + acc);
+          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // epilogue: thread = token (TMEM lane); state carried across the column tiles of a row tile
+    const int q = warp & 3;
+    int acc = 0; uint32_t acc_phase = 0;
+    const float ninf = __int_as_float(0xff800000);
+    for (int rt = blockIdx.x; rt < p.row_tiles && ok; rt += gridDim.x) {
+      const long long row = (long long)rt * BM + q * 32 + lane;
+      const bool row_ok = row < p.N;
+      float m = ninf, s = 0.f;               // running max and sum of exp(logit - m)
+      float v1 = ninf, v2 = ninf;            // two largest logits
+      int i1 = 0, i2 = 0;
+      for (int nt = 0; nt < p.n_tiles; ++nt) {
+        if (!ptx::mbar_wait(acc_full + acc, acc_phase, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after_sync();
+        const int ncols = min(BN, p.E - nt * BN);       // valid columns of this tile
+#pragma unroll 1
+        for (int c = 0; c * 32 < ncols; ++c) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32(tmem_base + (uint32_t)(acc * BN + c * 32) + ((uint32_t)(q * 32) << 16), r);
+          ptx::tmem_ld_wait();
+          if (!row_ok) continue;
+          const int col0 = nt * BN + c * 32;
+          const int nv = min(32, p.E - col0);
+          float v[32];
+          float cmax = ninf;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            v[i] = i < nv ? __uint_as_float(r[i]) : ninf;
+            cmax = fmaxf(cmax, v[i]);
+          }
+          if (cmax > m) { s *= expf(m - cmax); m = cmax; }
+          float part = 0.f;
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            part += expf(v[i] - m);                      // exp(-inf) = 0 for the padded columns
+            if (v[i] > v1) { v2 = v1; i2 = i1; v1 = v[i]; i1 = col0 + i; }
+            else if (v[i] > v2) { v2 = v[i]; i2 = col0 + i; }
+          }
+          s += part;
+          float* dst = p.logits + row * p.E + col0;
+          if (nv == 32) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              reinterpret_cast<float4*>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) if (i < nv) dst[i] = v[i];
+          }
+        }
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+      if (!ok) break;
+      if (row_ok) {
+        const float inv = 1.0f / s;
+        p.expert_idx[2 * row] = i1;
+        p.expert_idx[2 * row + 1] = i2;
+        p.gate12[2 * row] = expf(v1 - m) * inv;          // v1 == m
+        p.gate12[2 * row + 1] = expf(v2 - m) * inv;
+        p.rowmax[row] = m;
+        p.rowinv[row] = inv;
+      }
+    }
+  }
+
+  if (!ok) {
+    *abort_flag = 1;
+    set_device_status(p.status, GSHARD_ERR_TIMEOUT);
+    const uint64_t t0 = ptx::globaltimer_ns();
+    while (ptx::globaltimer_ns() - t0 < 2000000ull) { __nanosleep(1000); }
+  }
+  __syncwarp();
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace
+
+int launch_gate_fused(const Dims& d, const void* x, const void* wg, float* logits, int32_t* expert_idx,
+                      float* gate12, float* rowmax, float* rowinv, int* status, cudaStream_t st) {
+  GateParams p;
+  p.N = d.N; p.E = d.E; p.M = d.M;
+  p.row_tiles = (int)((d.N + BM - 1) / BM);
+  p.n_tiles = ceil_div(d.E, BN);
+  p.k_blocks = ceil_div(d.M, BK);
+  p.logits = logits; p.expert_idx = expert_idx; p.gate12 = gate12; p.rowmax = rowmax; p.rowinv = rowinv;
+  p.status = status;
+  CUtensorMap mx, mw;
+  bool okm = make_map(&mx, x, d.M, d.N, 1, d.M, 0, BK, BM);
+  okm = okm && make_map(&mw, wg, d.E, d.M, 1, d.E, 0, 64, BK);
+  if (!okm) return GSHARD_ERR_CUDA;
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int grid = p.row_tiles < sms ? p.row_tiles : sms;
+  if (cudaFuncSetAttribute(gate_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+    return GSHARD_ERR_CUDA;
+  gate_fused_kernel<<<grid, kThreads, kSmemBytes, st>>>(mx, mw, p);
+  count_launch();
+  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+}  // namespace gshard

@@ -6,7 +6,13 @@ namespace gshard {
 
 // gate.cu: row statistics + top-2 on stored logits, tile column sums, mean gates.
 void launch_gate_rows(const Dims& d, const float* logits, int32_t* expert_idx, float* gate12, float* rowmax,
-                      float* rowinv, float* partial, float* m, cudaStream_t st);
+                      float* rowinv, cudaStream_t st);
+void launch_gate_means(const Dims& d, const float* logits, const float* rowmax, const float* rowinv,
+                       float* partial, float* m, cudaStream_t st);
+
+// gate_fused.cu: bf16 logits GEMM on tcgen05 with row statistics and top-2 in the epilogue.
+int launch_gate_fused(const Dims& d, const void* x, const void* wg, float* logits, int32_t* expert_idx,
+                      float* gate12, float* rowmax, float* rowinv, int* status, cudaStream_t st);
 
 // capacity.cu
 int launch_capacity(const Dims& d, const int32_t* expert_idx, const float* gate12, const float* u, const float* m,
@@ -35,5 +41,10 @@ struct UmmaGemm {
   int a_stream, b_stream;    // operand is read once: load with an evict-first L2 hint
 };
 int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st);
+
+// ffn_fused.cu: both expert GEMMs in one persistent launch, h in an L2-resident ring.
+void ffn_fused_schedule(int rows, int H, int E, int* lag, int* ring);
+int launch_ffn_fused(const Dims& d, const void* buf, const void* wi, const void* wo, void* h_ring, int ring,
+                     void* out, int* flags, int* status, cudaStream_t st);
 
 }  // namespace gshard

@@ -17,6 +17,7 @@
 
 #include "kernels.cuh"
 #include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
 
 namespace gshard {
 
@@ -43,6 +44,7 @@ struct Params {
   int m_tiles, n_tiles, total_tiles, k_blocks;
   int out_f32, relu;
   int a_stream, b_stream;
+  int n_fastest;   // tile order: column tiles fastest (A is the large operand) instead of row tiles
   int* status;
 };
 
@@ -88,8 +90,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       const uint64_t pol_b = p.b_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
       int stage = 0; uint32_t phase = 0;
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-        const int mt = tile % p.m_tiles;
-        const int nt = (tile / p.m_tiles) % p.n_tiles;
+        const int mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
+        const int nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
         const int b = tile / (p.m_tiles * p.n_tiles);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!ptx::mbar_wait(empty + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -150,8 +152,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int q = warp & 3;                          // TMEM lane quarter this warp may access
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-      const int mt = tile % p.m_tiles;
-      const int nt = (tile / p.m_tiles) % p.n_tiles;
+      const int mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
+      const int nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
       const int b = tile / (p.m_tiles * p.n_tiles);
       if (!ptx::mbar_wait(acc_full + acc, acc_phase, abort_flag)) { ok = false; break; }
       ptx::tc_fence_after_sync();
@@ -233,36 +235,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
 // ---- host side ------------------------------------------------------------------------------
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = [] {
-    void* f = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-      f = nullptr;
-    return reinterpret_cast<EncodeTiledFn>(f);
-  }();
-  return fn;
-}
-
-// 3-D bf16 tensor map {inner, outer, batch} with a {box_inner, box_outer, 1} box, 128-byte swizzle.
-bool make_map(CUtensorMap* map, const void* base, long long inner, long long outer, long long batch,
-              long long ld_elems, long long bs_elems, int box_inner, int box_outer) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)batch};
-  cuuint64_t strides[2] = {(cuuint64_t)ld_elems * 2, (cuuint64_t)(batch > 1 ? bs_elems : ld_elems * outer) * 2};
-  cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <bool A_K, bool B_K, int BN>
 int launch_t(const UmmaGemm& g, const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int grid,
              cudaStream_t st) {
@@ -297,6 +269,8 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   p.total_tiles = p.m_tiles * p.n_tiles * g.batch;
   p.k_blocks = ceil_div(g.K, BK);
   p.out_f32 = g.out_f32; p.relu = g.relu; p.a_stream = g.a_stream; p.b_stream = g.b_stream;
+  // stream the larger operand once: walk the tiles that share it back to back
+  p.n_fastest = ((long long)g.rows * g.K > (long long)g.cols * g.K) ? 1 : 0;
   p.status = status;
   int sms = 148;
   int dev = 0;

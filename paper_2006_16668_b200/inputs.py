@@ -66,6 +66,10 @@ CONFIGS = {
     # a 64-expert slice of the MoE(2048E) layer (same per-expert shapes: 128 rows, M=1024, H=8192,
     # C=4; 2.1 GB of expert weights) - the small case profiler captures run on
     "p4_slice": MoEConfig("p4_slice", G=32, S=128, M=1024, H=8192, E=64, C=4, seed=20200636),
+    # the MoE(2048E) layer with a thin expert hidden dimension: gating, capacity, dispatch and combine
+    # see exactly the c4 sizes (131072 tokens, 2048 experts) while the expert weights shrink to
+    # 0.5 GB - the small case for profiler captures of those kernels
+    "p4_routing": MoEConfig("p4_routing", G=32, S=4096, M=1024, H=64, E=2048, C=4, seed=20200637),
     # configs[4]: training step
     "c5_512e_train": MoEConfig("c5_512e_train", G=16, S=4096, M=1024, H=8192, E=512, C=16,
                                seed=20200635, backward=True),

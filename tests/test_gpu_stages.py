@@ -122,13 +122,17 @@ FFN_CASES = [
     (2, 2, 100, 1024, 2048, "bf16", 0),          # 200 rows: ragged second row tile
     (3, 1, 24, 192, 448, "bf16", 0),             # fewer rows than a tile, ragged column tile
     (1, 4, 96, 512, 1024, "bf16", 0),            # 384 rows
+    # the experimental single-launch FFN (h in an L2-resident ring, cross-CTA dependencies)
+    (40, 1, 128, 512, 2048, "bf16", B.GSHARD_FLAG_FUSED_FFN),
+    (6, 2, 100, 256, 512, "bf16", B.GSHARD_FLAG_FUSED_FFN),
 ]
 
 
 @pytest.mark.parametrize("E,G,C,M,H,dtype,flags", FFN_CASES)
 def test_expert_ffn_against_oracle(E, G, C, M, H, dtype, flags):
     tdt = torch.float32 if dtype == "f32" else torch.bfloat16
-    shape = _shape(G, 4 * C, M, H, max(E, 16) if dtype == "bf16" and not flags else max(E, 2), C, dtype, flags)
+    umma = dtype == "bf16" and not (flags & B.GSHARD_FLAG_SIMT_CONTRACTIONS)
+    shape = _shape(G, 4 * C, M, H, -(-max(E, 16) // 16) * 16 if umma else max(E, 2), C, dtype, flags)
     E_run = shape.E
     gen = torch.Generator(device="cuda").manual_seed(E * 100 + C)
     buf = torch.randn(E_run, G * C, M, generator=gen, device="cuda").to(tdt)
