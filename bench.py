@@ -209,9 +209,28 @@ def main():
     rt, rs = B.alloc_routing(shape, device=dev)
     stream = torch.cuda.current_stream()
 
+    train = cfg.backward            # the training-step configuration times forward + backward
+    if train:
+        shape_t = B.make_shape(cfg, flags=shape.flags | B.GSHARD_FLAG_SAVE_FOR_BACKWARD)
+        ctx = torch.empty(B.gshard_moe_top2_context_bytes(shape_t), dtype=torch.uint8, device=dev)
+        wsb = B.alloc_workspace(shape_t, for_backward=True, device=dev)
+        dx = torch.empty_like(inp["x"])
+        dwg = torch.empty(cfg.M, cfg.E, dtype=torch.float32, device=dev)
+        dwi = torch.empty_like(inp["wi"])
+        dwo = torch.empty_like(inp["wo"])
+    bwd_launches = [0]
+
     def step():
-        B.gshard_moe_top2_forward(shape, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l_aux, rs,
-                                  None, ws, stream)
+        if not train:
+            B.gshard_moe_top2_forward(shape, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l_aux, rs,
+                                      None, ws, stream)
+            return
+        B.gshard_moe_top2_forward(shape_t, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l_aux, rs,
+                                  ctx, ws, stream)
+        fwd_launches = B.gshard_moe_last_launch_count()
+        B.gshard_moe_top2_backward(shape_t, inp["x"], inp["wg"], inp["wi"], inp["wo"], ctx, inp["dy"], cfg.k_aux,
+                                   dx, dwg, dwi, dwo, wsb, stream)
+        bwd_launches[0] = fwd_launches + B.gshard_moe_last_launch_count()
 
     def barrier():
         if world > 1:
@@ -223,7 +242,7 @@ def main():
     barrier()
     if B.gshard_moe_last_device_status(ws) != B.GSHARD_OK:
         raise SystemExit("device status is not OK after warm-up")
-    launches_per_step = B.gshard_moe_last_launch_count()
+    launches_per_step = bwd_launches[0] if train else B.gshard_moe_last_launch_count()
 
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -272,13 +291,18 @@ def main():
     # whole-layer roofline: slower of FLOPs at the tensor peak and bytes at the HBM peak
     layer_flops = 2.0 * cfg.N * cfg.M * cfg.E + ffn_flops
     layer_bytes = 2 * cfg.E * cfg.M * cfg.H * es + 2 * cfg.N * cfg.M * es + cfg.M * cfg.E * es + cfg.N * 4
+    if train:
+        # backward: four more FFN-sized GEMMs and two more gating-sized ones (plus the recomputed
+        # logits); weights are read once more and their gradients written once
+        layer_flops = 3 * 2.0 * cfg.N * cfg.M * cfg.E + 2.0 * cfg.N * cfg.M * cfg.E + 3 * ffn_flops
+        layer_bytes = 2 * layer_bytes + 2 * cfg.E * cfg.M * cfg.H * es + 2 * cfg.N * cfg.M * es
     t_roof = max(layer_flops / (peaks["bf16_tflops"] * 1e12), layer_bytes / (peaks["hbm_gbs"] * 1e9))
     layer = {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_per_step, "flops": layer_flops,
              "bytes": layer_bytes, "peak_source": peaks["source"]}
 
     # ---- end to end through the host-buffer entry point -------------------------------------
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not train:
         xh = inp["x"].cpu().pin_memory()
         uh = inp["u"].cpu().pin_memory()
         yh = torch.empty_like(xh).pin_memory()

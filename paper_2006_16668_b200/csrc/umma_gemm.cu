@@ -33,8 +33,10 @@ template <int BN> struct Cfg {
   static constexpr int stage_bytes = kABytes + b_bytes;
   static constexpr int stages = (BN == 256) ? 4 : 6;
   static constexpr int tmem_cols = 2 * BN;   // two accumulators
-  static constexpr int smem_bytes = stages * stage_bytes + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr int smem_bytes = stages * stage_bytes + 1024 /*align*/ + 256 /*barriers*/ + 4 * 32 * 256 /*epilogue staging*/;
 };
+
+constexpr int kStageRowBytes = 256;          // epilogue staging: 32 rows x 256 bytes per warp
 
 struct Params {
   void* C;
@@ -47,6 +49,27 @@ struct Params {
   int n_fastest;   // tile order: column tiles fastest (A is the large operand) instead of row tiles
   int* status;
 };
+
+// Writes a warp's staged 32 rows x 256 bytes to C: lane l handles 16-byte piece (l & 15) of rows
+// 2*i + (l >> 4); pieces beyond the matrix edge are skipped (cols is a multiple of the piece width).
+__device__ __forceinline__ void flush_rows(const unsigned char* stg, const Params& p, int b, int row0, int col0,
+                                           int lane) {
+  __syncwarp();
+  const int esz = p.out_f32 ? 4 : 2;
+  const int piece = lane & 15;
+  const int col = col0 + piece * (16 / esz);
+  unsigned char* cbase = reinterpret_cast<unsigned char*>(p.C) + ((long long)b * p.c_bs + col) * esz;
+#pragma unroll 4
+  for (int i = 0; i < 16; ++i) {
+    const int r = 2 * i + (lane >> 4);
+    const int row = row0 + r;
+    if (row < p.rows && col < p.cols) {
+      const uint4 val = *reinterpret_cast<const uint4*>(stg + r * kStageRowBytes + ((piece ^ (r & 15)) * 16));
+      *reinterpret_cast<uint4*>(cbase + (long long)row * p.c_ld * esz) = val;
+    }
+  }
+  __syncwarp();
+}
 
 template <bool A_K, bool B_K, int BN>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -150,6 +173,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   } else {
     // ------------------------------ epilogue ----------------------------------------------
     const int q = warp & 3;                          // TMEM lane quarter this warp may access
+    unsigned char* stg = smem + C_::stages * C_::stage_bytes + 256 + (warp - 2) * kStageRowBytes * 32;
+    const int cols_per_flush = p.out_f32 ? 64 : 128;  // 256 bytes of a row
+    const int chunks_per_flush = cols_per_flush / 32;
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
       const int mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
@@ -160,6 +186,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       const int row = mt * BM + q * 32 + lane;
       const bool row_ok = row < p.rows;
       const long long row_off = (long long)b * p.c_bs + (long long)row * p.c_ld;
+      bool pending = false;
+      int pending_col0 = 0;
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
         const int col0 = nt * BN + c * 32;
@@ -167,7 +195,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         uint32_t r[32];
         ptx::tmem_ld_32x32(tmem_base + (uint32_t)(acc * BN + c * 32) + ((uint32_t)(q * 32) << 16), r);
         ptx::tmem_ld_wait();
-        if (!row_ok) continue;
         float v[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
@@ -175,39 +202,59 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
           if (p.relu) v[i] = fmaxf(v[i], 0.f);
         }
         const bool full_chunk = col0 + 32 <= p.cols;
-        if (p.mask) {
+        if (p.mask && row_ok) {
           const __nv_bfloat16* mk = reinterpret_cast<const __nv_bfloat16*>(p.mask) + row_off + col0;
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (col0 + i < p.cols && !(__bfloat162float(mk[i]) > 0.f)) v[i] = 0.f;
-        }
-        if (p.out_f32) {
-          float* dst = reinterpret_cast<float*>(p.C) + row_off + col0;
-          if (full_chunk) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-              reinterpret_cast<float4*>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-          } else {
-            for (int i = 0; i < 32; ++i) if (col0 + i < p.cols) dst[i] = v[i];
-          }
-        } else {
-          __nv_bfloat16* dst = reinterpret_cast<__nv_bfloat16*>(p.C) + row_off + col0;
           if (full_chunk) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-              uint32_t w[4];
+              const uint4 mv = __ldg(reinterpret_cast<const uint4*>(mk) + i);
+              const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                const __nv_bfloat162 pr = __floats2bfloat162_rn(v[8 * i + 2 * j], v[8 * i + 2 * j + 1]);
-                w[j] = *reinterpret_cast<const uint32_t*>(&pr);
+                // bf16 > 0  <=>  sign bit clear and magnitude bits non-zero
+                const uint32_t lo = w[j] & 0xffffu, hi = w[j] >> 16;
+                if (!(lo != 0u && lo < 0x8000u)) v[8 * i + 2 * j] = 0.f;
+                if (!(hi != 0u && hi < 0x8000u)) v[8 * i + 2 * j + 1] = 0.f;
               }
-              reinterpret_cast<uint4*>(dst)[i] = make_uint4(w[0], w[1], w[2], w[3]);
             }
           } else {
-            for (int i = 0; i < 32; ++i) if (col0 + i < p.cols) dst[i] = __float2bfloat16_rn(v[i]);
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (col0 + i < p.cols && !(__bfloat162float(mk[i]) > 0.f)) v[i] = 0.f;
           }
         }
+        // stage the 32 values of this thread's row in shared memory (16-byte pieces, XOR-swizzled by
+        // row so that neither the row-wise writes nor the piece-wise reads conflict) ...
+        const int slot_in_flush = c % chunks_per_flush;
+        unsigned char* srow = stg + lane * 256;
+        if (p.out_f32) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int piece = (slot_in_flush * 8 + i) ^ (lane & 15);
+            *reinterpret_cast<float4*>(srow + piece * 16) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint32_t w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const __nv_bfloat162 pr = __floats2bfloat162_rn(v[8 * i + 2 * j], v[8 * i + 2 * j + 1]);
+              w[j] = *reinterpret_cast<const uint32_t*>(&pr);
+            }
+            const int piece = (slot_in_flush * 4 + i) ^ (lane & 15);
+            *reinterpret_cast<uint4*>(srow + piece * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+        pending_col0 = nt * BN + (c / chunks_per_flush) * cols_per_flush;
+        pending = true;
+        // ... and write whole 256-byte row segments: 16 lanes cover one row, 2 rows per instruction
+        if (slot_in_flush == chunks_per_flush - 1) {
+          flush_rows(stg, p, b, mt * BM + q * 32, pending_col0, lane);
+          pending = false;
+        }
       }
+      if (pending) flush_rows(stg, p, b, mt * BM + q * 32, pending_col0, lane);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
