@@ -6,13 +6,16 @@
 //               ring of 128-byte-swizzled shared-memory stages, completion on mbarriers
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=BN, K=16) from shared-memory
 //               descriptors into one of two TMEM accumulators; tcgen05.commit frees the stage
-//   warps 2..5  epilogue: tcgen05.ld the finished accumulator (thread = row), apply ReLU / mask,
-//               convert and store; overlaps the next tile's MMAs through the second accumulator
+//   warps 2..9  epilogue: two warps per TMEM lane quarter, each taking half of the tile's columns.
+//               tcgen05.ld the finished accumulator (thread = row, two 32-column loads in flight),
+//               apply ReLU / mask, convert, stage in swizzled shared memory and write 128-byte row
+//               segments; overlaps the next tile's MMAs through the second accumulator
 // Operands may be K-major or MN-major in global memory (the expert weights wi [M,H] and wo [H,M]
 // are contiguous along the non-contracted dimension); the layout goes into the tensor map, the
 // shared-memory descriptor and the instruction descriptor - nothing is transposed in memory.
-// Tile order: row tiles fastest, then column tiles, then batch, so CTAs that run together share
-// the same weight tile through L2 and each weight byte leaves HBM once.
+// Tile order: the tiles that share the larger operand run back to back (row tiles fastest when B
+// is larger, column tiles fastest when A is), then batch, so that operand leaves HBM once and the
+// other is re-read from L2.
 #include <cuda.h>
 
 #include "kernels.cuh"
@@ -24,19 +27,22 @@ namespace gshard {
 namespace {
 
 constexpr int BM = 128, BK = 64;
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kABytes = BM * BK * 2;        // 16 KB
 constexpr int kBoxBytes = 64 * 64 * 2;      // one 64x64 box of an MN-major operand
+constexpr int kStgRowBytes = 128;           // epilogue staging: 32 rows x 128 bytes per warp
+constexpr int kStgWarpBytes = 32 * kStgRowBytes;
 
 template <int BN> struct Cfg {
   static constexpr int b_bytes = BN * BK * 2;
   static constexpr int stage_bytes = kABytes + b_bytes;
   static constexpr int stages = (BN == 256) ? 4 : 6;
   static constexpr int tmem_cols = 2 * BN;   // two accumulators
-  static constexpr int smem_bytes = stages * stage_bytes + 1024 /*align*/ + 256 /*barriers*/ + 4 * 32 * 256 /*epilogue staging*/;
+  static constexpr int bar_off = stages * stage_bytes;
+  static constexpr int stg_off = bar_off + 256;
+  static constexpr int smem_bytes = stg_off + kEpiWarps * kStgWarpBytes + 1024 /*alignment slack*/;
 };
-
-constexpr int kStageRowBytes = 256;          // epilogue staging: 32 rows x 256 bytes per warp
 
 struct Params {
   void* C;
@@ -46,29 +52,89 @@ struct Params {
   int m_tiles, n_tiles, total_tiles, k_blocks;
   int out_f32, relu;
   int a_stream, b_stream;
-  int n_fastest;   // tile order: column tiles fastest (A is the large operand) instead of row tiles
+  int n_fastest;   // tile order: column tiles fastest (A is the larger operand) instead of row tiles
   int* status;
 };
 
-// Writes a warp's staged 32 rows x 256 bytes to C: lane l handles 16-byte piece (l & 15) of rows
-// 2*i + (l >> 4); pieces beyond the matrix edge are skipped (cols is a multiple of the piece width).
+struct TileCoord { int mt, nt, b; };
+
+__device__ __forceinline__ TileCoord decode(const Params& p, int tile) {
+  TileCoord t;
+  t.mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
+  t.nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
+  t.b = tile / (p.m_tiles * p.n_tiles);
+  return t;
+}
+
+// Writes a warp's staged 32 rows x 128 bytes to C: lane l handles 16-byte piece (l & 7) of rows
+// 4*i + (l >> 3); pieces beyond the matrix edge are skipped (cols is a multiple of the piece width).
 __device__ __forceinline__ void flush_rows(const unsigned char* stg, const Params& p, int b, int row0, int col0,
                                            int lane) {
   __syncwarp();
   const int esz = p.out_f32 ? 4 : 2;
-  const int piece = lane & 15;
+  const int piece = lane & 7;
   const int col = col0 + piece * (16 / esz);
   unsigned char* cbase = reinterpret_cast<unsigned char*>(p.C) + ((long long)b * p.c_bs + col) * esz;
-#pragma unroll 4
-  for (int i = 0; i < 16; ++i) {
-    const int r = 2 * i + (lane >> 4);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = 4 * i + (lane >> 3);
     const int row = row0 + r;
     if (row < p.rows && col < p.cols) {
-      const uint4 val = *reinterpret_cast<const uint4*>(stg + r * kStageRowBytes + ((piece ^ (r & 15)) * 16));
+      const uint4 val = *reinterpret_cast<const uint4*>(stg + r * kStgRowBytes + ((piece ^ (r & 7)) * 16));
       *reinterpret_cast<uint4*>(cbase + (long long)row * p.c_ld * esz) = val;
     }
   }
   __syncwarp();
+}
+
+// ReLU / mask on one 32-column chunk of this thread's row, then into the staging row (XOR-swizzled
+// 16-byte pieces: conflict-free for the row-wise writes here and the piece-wise reads of the flush).
+__device__ __forceinline__ void process_chunk(const uint32_t* r, const Params& p, unsigned char* srow, int lane,
+                                              int piece0, bool row_ok, long long row_off, int col0) {
+  float v[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    v[i] = __uint_as_float(r[i]);
+    if (p.relu) v[i] = fmaxf(v[i], 0.f);
+  }
+  if (p.mask && row_ok) {
+    const __nv_bfloat16* mk = reinterpret_cast<const __nv_bfloat16*>(p.mask) + row_off + col0;
+    if (col0 + 32 <= p.cols) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint4 mv = __ldg(reinterpret_cast<const uint4*>(mk) + i);
+        const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          // bf16 > 0  <=>  sign bit clear and magnitude bits non-zero
+          const uint32_t lo = w[j] & 0xffffu, hi = w[j] >> 16;
+          if (!(lo != 0u && lo < 0x8000u)) v[8 * i + 2 * j] = 0.f;
+          if (!(hi != 0u && hi < 0x8000u)) v[8 * i + 2 * j + 1] = 0.f;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i)
+        if (col0 + i < p.cols && !(__bfloat162float(mk[i]) > 0.f)) v[i] = 0.f;
+    }
+  }
+  if (p.out_f32) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      *reinterpret_cast<float4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16)) =
+          make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t w[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const __nv_bfloat162 pr = __floats2bfloat162_rn(v[8 * i + 2 * j], v[8 * i + 2 * j + 1]);
+        w[j] = *reinterpret_cast<const uint32_t*>(&pr);
+      }
+      *reinterpret_cast<uint4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
 }
 
 template <bool A_K, bool B_K, int BN>
@@ -78,7 +144,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   using C_ = Cfg<BN>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C_::stages * C_::stage_bytes);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C_::bar_off);
   uint64_t* full = bars;                       // [stages]
   uint64_t* empty = bars + C_::stages;         // [stages]
   uint64_t* acc_full = bars + 2 * C_::stages;  // [2]
@@ -90,7 +156,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C_::stages; ++s) { ptx::mbar_init(full + s, 1); ptx::mbar_init(empty + s, 1); }
-    for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full + a, 1); ptx::mbar_init(acc_empty + a, 4); }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full + a, 1); ptx::mbar_init(acc_empty + a, kEpiWarps); }
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&map_a);
@@ -113,27 +179,25 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       const uint64_t pol_b = p.b_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
       int stage = 0; uint32_t phase = 0;
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-        const int mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
-        const int nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
-        const int b = tile / (p.m_tiles * p.n_tiles);
+        const TileCoord t = decode(p, tile);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!ptx::mbar_wait(empty + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
           unsigned char* sa = smem + stage * C_::stage_bytes;
           unsigned char* sb = sa + kABytes;
           ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)C_::stage_bytes);
           if (A_K) {
-            ptx::tma_load_3d(sa, &map_a, full + stage, kb * BK, mt * BM, b, pol_a);
+            ptx::tma_load_3d(sa, &map_a, full + stage, kb * BK, t.mt * BM, t.b, pol_a);
           } else {
 #pragma unroll
             for (int j = 0; j < BM / 64; ++j)
-              ptx::tma_load_3d(sa + j * kBoxBytes, &map_a, full + stage, mt * BM + j * 64, kb * BK, b, pol_a);
+              ptx::tma_load_3d(sa + j * kBoxBytes, &map_a, full + stage, t.mt * BM + j * 64, kb * BK, t.b, pol_a);
           }
           if (B_K) {
-            ptx::tma_load_3d(sb, &map_b, full + stage, kb * BK, nt * BN, b, pol_b);
+            ptx::tma_load_3d(sb, &map_b, full + stage, kb * BK, t.nt * BN, t.b, pol_b);
           } else {
 #pragma unroll
             for (int j = 0; j < BN / 64; ++j)
-              ptx::tma_load_3d(sb + j * kBoxBytes, &map_b, full + stage, nt * BN + j * 64, kb * BK, b, pol_b);
+              ptx::tma_load_3d(sb + j * kBoxBytes, &map_b, full + stage, t.nt * BN + j * 64, kb * BK, t.b, pol_b);
           }
           if (++stage == C_::stages) { stage = 0; phase ^= 1u; }
         }
@@ -172,89 +236,40 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
   } else {
     // ------------------------------ epilogue ----------------------------------------------
+    const int ew = warp - 2;
     const int q = warp & 3;                          // TMEM lane quarter this warp may access
-    unsigned char* stg = smem + C_::stages * C_::stage_bytes + 256 + (warp - 2) * kStageRowBytes * 32;
-    const int cols_per_flush = p.out_f32 ? 64 : 128;  // 256 bytes of a row
-    const int chunks_per_flush = cols_per_flush / 32;
+    const int half = ew >> 2;                        // which half of the tile's columns
+    constexpr int kHalfCols = BN / 2;
+    unsigned char* stg = smem + C_::stg_off + ew * kStgWarpBytes;
+    unsigned char* srow = stg + lane * kStgRowBytes;
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-      const int mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
-      const int nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
-      const int b = tile / (p.m_tiles * p.n_tiles);
+      const TileCoord t = decode(p, tile);
       if (!ptx::mbar_wait(acc_full + acc, acc_phase, abort_flag)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      const int row = mt * BM + q * 32 + lane;
-      const bool row_ok = row < p.rows;
-      const long long row_off = (long long)b * p.c_bs + (long long)row * p.c_ld;
-      bool pending = false;
-      int pending_col0 = 0;
+      const int row0 = t.mt * BM + q * 32;
+      const bool row_ok = row0 + lane < p.rows;
+      const long long row_off = (long long)t.b * p.c_bs + (long long)(row0 + lane) * p.c_ld;
+      const uint32_t t_acc = tmem_base + (uint32_t)(acc * BN + half * kHalfCols) + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-      for (int c = 0; c < BN / 32; ++c) {
-        const int col0 = nt * BN + c * 32;
+      for (int c = 0; c < kHalfCols / 64; ++c) {     // 64 columns per round: two TMEM loads in flight
+        const int col0 = t.nt * BN + half * kHalfCols + c * 64;
         if (col0 >= p.cols) break;                   // uniform over the warp
-        uint32_t r[32];
-        ptx::tmem_ld_32x32(tmem_base + (uint32_t)(acc * BN + c * 32) + ((uint32_t)(q * 32) << 16), r);
+        uint32_t r0[32], r1[32];
+        ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r0);
+        ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r1);
         ptx::tmem_ld_wait();
-        float v[32];
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          v[i] = __uint_as_float(r[i]);
-          if (p.relu) v[i] = fmaxf(v[i], 0.f);
-        }
-        const bool full_chunk = col0 + 32 <= p.cols;
-        if (p.mask && row_ok) {
-          const __nv_bfloat16* mk = reinterpret_cast<const __nv_bfloat16*>(p.mask) + row_off + col0;
-          if (full_chunk) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const uint4 mv = __ldg(reinterpret_cast<const uint4*>(mk) + i);
-              const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                // bf16 > 0  <=>  sign bit clear and magnitude bits non-zero
-                const uint32_t lo = w[j] & 0xffffu, hi = w[j] >> 16;
-                if (!(lo != 0u && lo < 0x8000u)) v[8 * i + 2 * j] = 0.f;
-                if (!(hi != 0u && hi < 0x8000u)) v[8 * i + 2 * j + 1] = 0.f;
-              }
-            }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (col0 + i < p.cols && !(__bfloat162float(mk[i]) > 0.f)) v[i] = 0.f;
-          }
-        }
-        // stage the 32 values of this thread's row in shared memory (16-byte pieces, XOR-swizzled by
-        // row so that neither the row-wise writes nor the piece-wise reads conflict) ...
-        const int slot_in_flush = c % chunks_per_flush;
-        unsigned char* srow = stg + lane * 256;
-        if (p.out_f32) {
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int piece = (slot_in_flush * 8 + i) ^ (lane & 15);
-            *reinterpret_cast<float4*>(srow + piece * 16) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint32_t w[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const __nv_bfloat162 pr = __floats2bfloat162_rn(v[8 * i + 2 * j], v[8 * i + 2 * j + 1]);
-              w[j] = *reinterpret_cast<const uint32_t*>(&pr);
-            }
-            const int piece = (slot_in_flush * 4 + i) ^ (lane & 15);
-            *reinterpret_cast<uint4*>(srow + piece * 16) = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
-        pending_col0 = nt * BN + (c / chunks_per_flush) * cols_per_flush;
-        pending = true;
-        // ... and write whole 256-byte row segments: 16 lanes cover one row, 2 rows per instruction
-        if (slot_in_flush == chunks_per_flush - 1) {
-          flush_rows(stg, p, b, mt * BM + q * 32, pending_col0, lane);
-          pending = false;
+        if (p.out_f32) {                             // 32 fp32 columns = one 128-byte staging row
+          process_chunk(r0, p, srow, lane, 0, row_ok, row_off, col0);
+          flush_rows(stg, p, t.b, row0, col0, lane);
+          process_chunk(r1, p, srow, lane, 0, row_ok, row_off, col0 + 32);
+          flush_rows(stg, p, t.b, row0, col0 + 32, lane);
+        } else {                                     // 64 bf16 columns = one 128-byte staging row
+          process_chunk(r0, p, srow, lane, 0, row_ok, row_off, col0);
+          process_chunk(r1, p, srow, lane, 4, row_ok, row_off, col0 + 32);
+          flush_rows(stg, p, t.b, row0, col0, lane);
         }
       }
-      if (pending) flush_rows(stg, p, b, mt * BM + q * 32, pending_col0, lane);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
@@ -283,15 +298,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 // ---- host side ------------------------------------------------------------------------------
 
 template <bool A_K, bool B_K, int BN>
-int launch_t(const UmmaGemm& g, const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int grid,
-             cudaStream_t st) {
+int launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int grid, cudaStream_t st) {
   auto kern = umma_gemm_kernel<A_K, B_K, BN>;
-  static bool attr_done = false;
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::smem_bytes) != cudaSuccess)
-      return GSHARD_ERR_CUDA;
-    attr_done = true;
-  }
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::smem_bytes) != cudaSuccess)
+    return GSHARD_ERR_CUDA;
   kern<<<grid, kThreads, Cfg<BN>::smem_bytes, st>>>(ma, mb, p);
   count_launch();
   return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
@@ -317,14 +327,14 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   p.k_blocks = ceil_div(g.K, BK);
   p.out_f32 = g.out_f32; p.relu = g.relu; p.a_stream = g.a_stream; p.b_stream = g.b_stream;
   // stream the larger operand once: walk the tiles that share it back to back
-  p.n_fastest = ((long long)g.rows * g.K > (long long)g.cols * g.K) ? 1 : 0;
+  p.n_fastest = (g.rows > g.cols) ? 1 : 0;
   p.status = status;
   int sms = 148;
   int dev = 0;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int grid = p.total_tiles < sms ? p.total_tiles : sms;
-#define GSHARD_DISPATCH(AK, BKM)                                                         \
-  (BN == 256 ? launch_t<AK, BKM, 256>(g, ma, mb, p, grid, st) : launch_t<AK, BKM, 128>(g, ma, mb, p, grid, st))
+#define GSHARD_DISPATCH(AK, BKM) \
+  (BN == 256 ? launch_t<AK, BKM, 256>(ma, mb, p, grid, st) : launch_t<AK, BKM, 128>(ma, mb, p, grid, st))
   if (g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH(true, true);
   if (g.a_kmajor && !g.b_kmajor) return GSHARD_DISPATCH(true, false);
   if (!g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH(false, true);
