@@ -82,7 +82,7 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   bool ok = true;
   if (warp == 0) {
     if (lane == 0) {
-      const uint64_t pol_x = ptx::policy_evict_first();    // each row panel is used by one CTA only
+      const uint64_t pol_x = ptx::policy_evict_last();     // a row panel is re-read for every column tile
       const uint64_t pol_w = ptx::policy_evict_last();     // wg is shared by every CTA
       int stage = 0; uint32_t phase = 0;
       for (int rt = blockIdx.x; rt < p.row_tiles && ok; rt += gridDim.x) {
@@ -132,52 +132,76 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       }
     }
   } else {
-    // epilogue: thread = token (TMEM lane); state carried across the column tiles of a row tile
+    // epilogue: thread = token (TMEM lane); state carried across the column tiles of a row tile.
+    // The running top-2 and the exp-sum are kept as four independent chains (columns i mod 4) so
+    // that the per-element updates overlap instead of forming one long dependency chain; each
+    // chain scans its columns in ascending order with strict comparisons, and the chains are
+    // merged at the end of the row with an explicit lowest-index tie rule.
     const int q = warp & 3;
     int acc = 0; uint32_t acc_phase = 0;
     const float ninf = __int_as_float(0xff800000);
+    constexpr float kLog2e = 1.4426950408889634f;
     for (int rt = blockIdx.x; rt < p.row_tiles && ok; rt += gridDim.x) {
       const long long row = (long long)rt * BM + q * 32 + lane;
       const bool row_ok = row < p.N;
-      float m = ninf, s = 0.f;               // running max and sum of exp(logit - m)
-      float v1 = ninf, v2 = ninf;            // two largest logits
-      int i1 = 0, i2 = 0;
+      float m = ninf;                        // running row maximum
+      float s4[4] = {0.f, 0.f, 0.f, 0.f};    // partial sums of exp(logit - m)
+      float a1[4], a2[4];                    // per chain: two largest logits ...
+      int j1[4], j2[4];                      // ... and their expert indices
+#pragma unroll
+      for (int k = 0; k < 4; ++k) { a1[k] = ninf; a2[k] = ninf; j1[k] = 0x7fffffff; j2[k] = 0x7fffffff; }
       for (int nt = 0; nt < p.n_tiles; ++nt) {
         if (!ptx::mbar_wait(acc_full + acc, acc_phase, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const int ncols = min(BN, p.E - nt * BN);       // valid columns of this tile
+        const uint32_t t_acc = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-        for (int c = 0; c * 32 < ncols; ++c) {
-          uint32_t r[32];
-          ptx::tmem_ld_32x32(tmem_base + (uint32_t)(acc * BN + c * 32) + ((uint32_t)(q * 32) << 16), r);
+        for (int c = 0; c * 64 < ncols; ++c) {          // 64 columns per round: two TMEM loads in flight
+          uint32_t r[2][32];
+          ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r[0]);
+          ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r[1]);
           ptx::tmem_ld_wait();
           if (!row_ok) continue;
-          const int col0 = nt * BN + c * 32;
-          const int nv = min(32, p.E - col0);
-          float v[32];
-          float cmax = ninf;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            v[i] = i < nv ? __uint_as_float(r[i]) : ninf;
-            cmax = fmaxf(cmax, v[i]);
-          }
-          if (cmax > m) { s *= expf(m - cmax); m = cmax; }
-          float part = 0.f;
+          for (int hh = 0; hh < 2; ++hh) {
+            const int col0 = nt * BN + c * 64 + hh * 32;
+            const int nv = min(32, p.E - col0);
+            if (nv <= 0) break;
+            float v[32];
+            float cm[4] = {ninf, ninf, ninf, ninf};
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            part += expf(v[i] - m);                      // exp(-inf) = 0 for the padded columns
-            if (v[i] > v1) { v2 = v1; i2 = i1; v1 = v[i]; i1 = col0 + i; }
-            else if (v[i] > v2) { v2 = v[i]; i2 = col0 + i; }
-          }
-          s += part;
-          float* dst = p.logits + row * p.E + col0;
-          if (nv == 32) {
+            for (int i = 0; i < 32; ++i) {
+              v[i] = i < nv ? __uint_as_float(r[hh][i]) : ninf;
+              cm[i & 3] = fmaxf(cm[i & 3], v[i]);
+            }
+            const float cmax = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
+            if (cmax > m) {
+              const float sc = __expf(m - cmax);        // exp(-inf) = 0 on the first chunk
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-              reinterpret_cast<float4*>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-          } else {
+              for (int k = 0; k < 4; ++k) s4[k] *= sc;
+              m = cmax;
+            }
+            const float ml = m * kLog2e;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) if (i < nv) dst[i] = v[i];
+            for (int i = 0; i < 32; ++i) {
+              const int k = i & 3;
+              s4[k] += exp2f(fmaf(v[i], kLog2e, -ml));  // exp(v - m); 0 for the padded columns
+              const bool gt1 = v[i] > a1[k];
+              const bool gt2 = v[i] > a2[k];
+              a2[k] = gt1 ? a1[k] : (gt2 ? v[i] : a2[k]);
+              j2[k] = gt1 ? j1[k] : (gt2 ? col0 + i : j2[k]);
+              a1[k] = gt1 ? v[i] : a1[k];
+              j1[k] = gt1 ? col0 + i : j1[k];
+            }
+            float* dst = p.logits + row * p.E + col0;
+            if (nv == 32) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                __stcs(reinterpret_cast<float4*>(dst) + i, make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) if (i < nv) dst[i] = v[i];
+            }
           }
         }
         ptx::tc_fence_before_sync();
@@ -187,10 +211,28 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       }
       if (!ok) break;
       if (row_ok) {
-        const float inv = 1.0f / s;
+        // merge the four chains: larger value first, lower index on equal values
+        float v1 = a1[0], v2 = a2[0];
+        int i1 = j1[0], i2 = j2[0];
+#pragma unroll
+        for (int k = 1; k < 4; ++k) {
+          const bool b1 = a1[k] > v1 || (a1[k] == v1 && j1[k] < i1);       // chain's best beats v1
+          // candidates for the new second place: loser of the first comparison and the winner's second
+          const float l_v = b1 ? v1 : a1[k];
+          const int l_i = b1 ? i1 : j1[k];
+          const float w2_v = b1 ? a2[k] : v2;
+          const int w2_i = b1 ? j2[k] : i2;
+          v1 = b1 ? a1[k] : v1;
+          i1 = b1 ? j1[k] : i1;
+          const bool b2 = l_v > w2_v || (l_v == w2_v && l_i < w2_i);
+          v2 = b2 ? l_v : w2_v;
+          i2 = b2 ? l_i : w2_i;
+        }
+        const float ssum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+        const float inv = 1.0f / ssum;
         p.expert_idx[2 * row] = i1;
         p.expert_idx[2 * row + 1] = i2;
-        p.gate12[2 * row] = expf(v1 - m) * inv;          // v1 == m
+        p.gate12[2 * row] = inv;                          // exp(v1 - m) = 1
         p.gate12[2 * row + 1] = expf(v2 - m) * inv;
         p.rowmax[row] = m;
         p.rowinv[row] = inv;
