@@ -57,10 +57,12 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  the counter of its second expert */
 #define GSHARD_FLAG_SIMT_CONTRACTIONS 4u   /* bf16 only: run every contraction on CUDA cores
                                               (fp32 FMA) instead of tcgen05; for debugging */
-#define GSHARD_FLAG_FUSED_FFN 8u           /* bf16 tensor-core path only, experimental: run the expert
-                                              FFN as one persistent launch that keeps the hidden
-                                              activations in an L2-resident ring (measured slower
-                                              than the default two grouped-GEMM launches) */
+#define GSHARD_FLAG_FUSED_FFN 8u           /* bf16 tensor-core path: force the single-launch expert FFN
+                                              (hidden activations handed over through L2, never
+                                              written to HBM) where the shape allows it; by default
+                                              it is used when an expert has at most 128 rows */
+#define GSHARD_FLAG_UNFUSED_FFN 16u        /* force the two grouped-GEMM launches instead (hidden
+                                              activations make a round trip through HBM) */
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

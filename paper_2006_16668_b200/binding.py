@@ -29,6 +29,7 @@ GSHARD_FLAG_SAVE_FOR_BACKWARD = 1
 GSHARD_FLAG_SECOND_SKIP_FREES_SLOT = 2
 GSHARD_FLAG_SIMT_CONTRACTIONS = 4
 GSHARD_FLAG_FUSED_FFN = 8
+GSHARD_FLAG_UNFUSED_FFN = 16
 
 
 class gshard_moe_shape(Structure):

@@ -65,15 +65,16 @@ int gate_stage(const Dims& d, const FwdPlan& pl, unsigned char* ws, const void* 
 }
 
 // h = relu(buf . wi), out = h . wo for every expert (eq. (2)); weights are read once.
-int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool h_is_full, void* out,
-              int* flags, int* status, cudaStream_t st) {
+int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
+              void* fused_scratch, int* status, cudaStream_t st) {
   const long long rows = d.rows;
-  if (!d.simt && d.fused_ffn) {
-    // one persistent launch; h lives in a ring of a few experts unless the caller keeps all of it
-    int lag = 0, ring = 0;
-    ffn_fused_schedule(d.rows, d.H, d.E, &lag, &ring);
-    return launch_ffn_fused(d, buf, wi, wo, h, h_is_full ? d.E : ring, out, flags, status, st);
-  }
+  // One persistent launch in which the hidden activations never leave L2: the faster form when
+  // the FFN is bound by streaming the expert weights (at most one 128-row tile per expert); with
+  // more rows per expert the two grouped-GEMM launches keep the tensor pipe busier.  Not available
+  // when the caller keeps h for the backward pass.
+  const bool want_fused = d.fused_ffn || (!d.unfused_ffn && d.rows <= 128);
+  if (!d.simt && want_fused && !keep_h && ffn_fused_supported(d))
+    return launch_ffn_fused(d, buf, wi, wo, fused_scratch, out, status, st);
   UmmaGemm g{};
   g.A = buf; g.B = wi; g.C = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;
   g.a_kmajor = true; g.b_kmajor = false;
@@ -98,7 +99,8 @@ int validate_shape(const gshard_moe_shape* s) {
   if (!s) return GSHARD_ERR_INVALID_ARG;
   if (s->G <= 0 || s->S <= 0 || s->M <= 0 || s->H <= 0 || s->E <= 0 || s->C <= 0) return GSHARD_ERR_INVALID_ARG;
   if (s->dtype != GSHARD_F32 && s->dtype != GSHARD_BF16) return GSHARD_ERR_INVALID_ARG;
-  if (s->flags & ~15u) return GSHARD_ERR_INVALID_ARG;
+  if (s->flags & ~31u) return GSHARD_ERR_INVALID_ARG;
+  if ((s->flags & GSHARD_FLAG_FUSED_FFN) && (s->flags & GSHARD_FLAG_UNFUSED_FFN)) return GSHARD_ERR_INVALID_ARG;
   if (s->E < 2) return GSHARD_ERR_INVALID_ARG;
   if (s->M % 8 || s->H % 8) return GSHARD_ERR_UNSUPPORTED_SHAPE;
   if (s->S > 32767 || s->E > 16384 || s->C > 32767) return GSHARD_ERR_UNSUPPORTED_SHAPE;
@@ -148,7 +150,7 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
   GS_TRY(launch_capacity(d, expert_idx, gate12, u, m, slot, weight, flags, first_count, total_count, slot_token,
                          l_aux_group, stats_group, l_aux, reinterpret_cast<long long*>(r.stats), st));
   launch_dispatch(d, x, slot_token, buf, st);
-  GS_TRY(ffn_stage(d, buf, wi, wo, h, save, out, reinterpret_cast<int*>(ws + pl.ffn_flags), status, st));
+  GS_TRY(ffn_stage(d, buf, wi, wo, h, save, out, ws + pl.ffn_scratch, status, st));
   launch_combine(d, out, expert_idx, slot, weight, y, st);
 
   if (save) {   // hand the caller the routing tensors it asked for
@@ -331,7 +333,7 @@ int gshard_moe_expert_ffn(const gshard_moe_shape* shape, const void* buf, const 
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   if (cudaMemsetAsync(ws + pl.status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
-  GS_TRY(ffn_stage(d, buf, wi, wo, ws + pl.h, false, out, reinterpret_cast<int*>(ws + pl.ffn_flags),
+  GS_TRY(ffn_stage(d, buf, wi, wo, ws + pl.h, false, out, ws + pl.ffn_scratch,
                    reinterpret_cast<int*>(ws + pl.status), st));
   return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }

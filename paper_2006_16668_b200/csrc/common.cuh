@@ -41,7 +41,8 @@ struct Dims {
   bool bf16;
   bool simt;            // contractions on CUDA cores
   bool variant_a;
-  bool fused_ffn;       // experimental single-launch FFN with h in an L2-resident ring
+  bool fused_ffn;       // force the single-launch FFN (h handed over through L2)
+  bool unfused_ffn;     // force the two grouped-GEMM launches (h through HBM)
 };
 
 inline Dims make_dims(const gshard_moe_shape& s) {
@@ -56,6 +57,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.simt = !d.bf16 || (s.flags & GSHARD_FLAG_SIMT_CONTRACTIONS);
   d.variant_a = (s.flags & GSHARD_FLAG_SECOND_SKIP_FREES_SLOT) != 0;
   d.fused_ffn = (s.flags & GSHARD_FLAG_FUSED_FFN) != 0;
+  d.unfused_ffn = (s.flags & GSHARD_FLAG_UNFUSED_FFN) != 0;
   return d;
 }
 

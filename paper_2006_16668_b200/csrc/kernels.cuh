@@ -42,9 +42,11 @@ struct UmmaGemm {
 };
 int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st);
 
-// ffn_fused.cu: both expert GEMMs in one persistent launch, h in an L2-resident ring.
-void ffn_fused_schedule(int rows, int H, int E, int* lag, int* ring);
-int launch_ffn_fused(const Dims& d, const void* buf, const void* wi, const void* wo, void* h_ring, int ring,
-                     void* out, int* flags, int* status, cudaStream_t st);
+// ffn_fused.cu: both expert GEMMs in one persistent launch; groups of four CTAs exchange 256-column
+// chunks of the hidden activations through a small L2-resident scratch ring.
+bool ffn_fused_supported(const Dims& d);
+size_t ffn_fused_scratch_bytes(const Dims& d);
+int launch_ffn_fused(const Dims& d, const void* buf, const void* wi, const void* wo, void* scratch, void* out,
+                     int* status, cudaStream_t st);
 
 }  // namespace gshard

@@ -12,7 +12,7 @@ struct Carver {
 
 struct FwdPlan {
   size_t status, logits, rowmax, rowinv, partial, gate12, m, expert_idx, slot, weight, flags, first_count,
-      total_count, slot_token, l_aux_group, stats_group, ffn_flags, buf, h, out, total;
+      total_count, slot_token, l_aux_group, stats_group, ffn_scratch, buf, h, out, total;
 };
 
 inline FwdPlan plan_forward(const Dims& d) {
@@ -34,7 +34,7 @@ inline FwdPlan plan_forward(const Dims& d) {
   p.slot_token = c.take(R * 4);
   p.l_aux_group = c.take((size_t)d.G * 4);
   p.stats_group = c.take((size_t)d.G * 8 * 4);
-  p.ffn_flags = c.take((size_t)2 * d.E * ceil_div(d.rows, 128) * 4);
+  p.ffn_scratch = c.take(ffn_fused_scratch_bytes(d));
   p.buf = c.take(R * d.M * d.esize);
   p.h = c.take(R * d.H * d.esize);
   p.out = c.take(R * d.M * d.esize);

@@ -115,6 +115,9 @@ SMALL = [
     ("bf16_umma_ragged_rows", 3, 333, 192, 448, 48, 7, "bf16", 0),
     ("bf16_umma_variant_a", 2, 512, 256, 512, 32, 16, "bf16", B.GSHARD_FLAG_SECOND_SKIP_FREES_SLOT),
     ("bf16_capacity_one", 2, 128, 64, 128, 32, 1, "bf16", 0),
+    # <= 128 rows per expert and H a multiple of 1024: the single-launch FFN is chosen by default
+    ("bf16_fused_ffn_auto", 2, 256, 256, 1024, 32, 16, "bf16", 0),
+    ("bf16_unfused_forced", 2, 256, 256, 1024, 32, 16, "bf16", B.GSHARD_FLAG_UNFUSED_FFN),
 ]
 
 

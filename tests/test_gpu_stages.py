@@ -122,9 +122,10 @@ FFN_CASES = [
     (2, 2, 100, 1024, 2048, "bf16", 0),          # 200 rows: ragged second row tile
     (3, 1, 24, 192, 448, "bf16", 0),             # fewer rows than a tile, ragged column tile
     (1, 4, 96, 512, 1024, "bf16", 0),            # 384 rows
-    # the experimental single-launch FFN (h in an L2-resident ring, cross-CTA dependencies)
+    # the single-launch FFN (groups of four CTAs, h chunks handed over through an L2-resident ring)
     (40, 1, 128, 512, 2048, "bf16", B.GSHARD_FLAG_FUSED_FFN),
-    (6, 2, 100, 256, 512, "bf16", B.GSHARD_FLAG_FUSED_FFN),
+    (6, 2, 100, 256, 1024, "bf16", B.GSHARD_FLAG_FUSED_FFN),     # 200 rows: two row tiles per expert
+    (3, 1, 24, 192, 3072, "bf16", B.GSHARD_FLAG_FUSED_FFN),      # 48 output columns per rank
 ]
 
 
