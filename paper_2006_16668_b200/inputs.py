@@ -70,6 +70,8 @@ CONFIGS = {
     # see exactly the c4 sizes (131072 tokens, 2048 experts) while the expert weights shrink to
     # 0.5 GB - the small case for profiler captures of those kernels
     "p4_routing": MoEConfig("p4_routing", G=32, S=4096, M=1024, H=64, E=2048, C=4, seed=20200637),
+    # a 16-expert slice of the MoE(128E) layer (1024 rows per expert, tensor-bound expert GEMMs)
+    "p2_slice": MoEConfig("p2_slice", G=16, S=512, M=1024, H=8192, E=16, C=64, seed=20200638),
     # configs[4]: training step
     "c5_512e_train": MoEConfig("c5_512e_train", G=16, S=4096, M=1024, H=8192, E=512, C=16,
                                seed=20200635, backward=True),
