@@ -17,8 +17,11 @@
 // round T (epilogue -> scratch -> flag -> TMA load) hides behind GEMM-1 of round T+1.
 //   chunk hand-over  prod[group][rank] counts finished epilogue warps (release); the producers of
 //                    all four ranks acquire it, then fence the async proxy before the TMA load.
-//   ring reuse       safe without further flags: a rank can be four rounds ahead of another only
-//                    if that one has completed the GEMM-2 reads of the slot (see DESIGN notes).
+//   ring reuse       safe without further flags.  Rank r overwrites the slot of round T when its
+//                    epilogue of round T+4 runs, i.e. after its G1(T+4) completed; tcgen05 MMAs
+//                    complete in issue order, so its G2(T+2) completed, which needed the round
+//                    T+2 chunks of every rank r'; r' stored that chunk after its own G1(T+2)
+//                    completed, and r' issued G2(T) before G1(T+2): r' is done reading round T.
 // All CTAs are co-resident (grid <= SM count, one CTA per SM) and every wait is bounded in wall
 // time, reporting GSHARD_ERR_TIMEOUT through the status word instead of hanging.
 #include <cuda.h>
