@@ -126,6 +126,9 @@ FFN_CASES = [
     (40, 1, 128, 512, 2048, "bf16", B.GSHARD_FLAG_FUSED_FFN),
     (6, 2, 100, 256, 1024, "bf16", B.GSHARD_FLAG_FUSED_FFN),     # 200 rows: two row tiles per expert
     (3, 1, 24, 192, 3072, "bf16", B.GSHARD_FLAG_FUSED_FFN),      # 48 output columns per rank
+    (37, 1, 1, 64, 1024, "bf16", B.GSHARD_FLAG_FUSED_FFN),       # one row per expert, 16 columns per rank
+    (150, 1, 128, 1024, 1024, "bf16", B.GSHARD_FLAG_FUSED_FFN),  # more units than groups, uneven split
+    (2, 3, 128, 448, 2048, "bf16", B.GSHARD_FLAG_FUSED_FFN),     # three full row tiles, 112 columns per rank
 ]
 
 
