@@ -63,6 +63,9 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                               it is used when an expert has at most 128 rows */
 #define GSHARD_FLAG_UNFUSED_FFN 16u        /* force the two grouped-GEMM launches instead (hidden
                                               activations make a round trip through HBM) */
+#define GSHARD_FLAG_TWO_SM_MMA 32u         /* grouped GEMMs with more than 128 rows per problem run on
+                                              CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles) instead
+                                              of single CTAs (128 x 256 tiles) */
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

@@ -30,6 +30,7 @@ GSHARD_FLAG_SECOND_SKIP_FREES_SLOT = 2
 GSHARD_FLAG_SIMT_CONTRACTIONS = 4
 GSHARD_FLAG_FUSED_FFN = 8
 GSHARD_FLAG_UNFUSED_FFN = 16
+GSHARD_FLAG_TWO_SM_MMA = 32
 
 
 class gshard_moe_shape(Structure):

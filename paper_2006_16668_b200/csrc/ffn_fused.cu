@@ -271,7 +271,7 @@ ffn_group4_kernel(const __grid_constant__ CUtensorMap map_buf, const __grid_cons
     for (int T = 0; T <= total_T && ok; ++T) {
       if (T < total_T) {
         // h chunk of round T: TMEM -> relu -> bf16 -> scratch slot of this rank
-        if (!ptx::mbar_wait(g1_full, (uint32_t)T & 1u, abort_flag)) { ok = false; break; }
+        if (!ptx::mbar_wait_warp(g1_full, (uint32_t)T & 1u, abort_flag, lane)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const int slot = (group * kRing + (T % kRing)) * kGroup + rank;
         __nv_bfloat16* dst = p.scratch + ((size_t)slot * BM + q * 32) * KC;
@@ -300,7 +300,7 @@ ffn_group4_kernel(const __grid_constant__ CUtensorMap map_buf, const __grid_cons
         const int ui = (T - 1) / p.rounds;
         const int u = group + ui * p.groups;
         const int e = u / p.m_tiles, mt = u % p.m_tiles;
-        if (!ptx::mbar_wait(out_full, (uint32_t)ui & 1u, abort_flag)) { ok = false; break; }
+        if (!ptx::mbar_wait_warp(out_full, (uint32_t)ui & 1u, abort_flag, lane)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const int row0 = mt * BM + q * 32;
         __nv_bfloat16* dst = p.out + ((size_t)e * p.rows + row0) * p.M + rank * p.NW;

@@ -151,7 +151,7 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 #pragma unroll
       for (int k = 0; k < 4; ++k) { a1[k] = ninf; a2[k] = ninf; j1[k] = 0x7fffffff; j2[k] = 0x7fffffff; }
       for (int nt = 0; nt < p.n_tiles; ++nt) {
-        if (!ptx::mbar_wait(acc_full + acc, acc_phase, abort_flag)) { ok = false; break; }
+        if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const int ncols = min(BN, p.E - nt * BN);       // valid columns of this tile
         const uint32_t t_acc = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);

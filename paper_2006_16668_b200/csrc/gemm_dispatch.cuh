@@ -7,7 +7,14 @@ namespace gshard {
 
 // A and B hold the configuration dtype; C holds float when g.out_f32, else the dtype.
 inline int run_gemm(const Dims& d, const UmmaGemm& g, int* status, cudaStream_t st) {
-  if (!d.simt) return launch_umma_gemm(g, status, st);
+  if (!d.simt) {
+    // CTA pairs with the two-SM MMA load a third fewer operand bytes per SM and run the tensor pipe
+    // about 10 % busier in isolation, but under the board's sustained power cap they measured no
+    // faster than single CTAs (slower on the 1024-rows-per-expert shape), so they are opt-in.  A
+    // single row tile would leave the second CTA of a pair without rows.
+    if (g.rows > 128 && d.two_sm_mma) return launch_umma2_gemm(g, status, st);
+    return launch_umma_gemm(g, status, st);
+  }
   SimtGemm s{};
   s.A = g.A; s.B = g.B; s.C = g.C; s.mask = g.mask;
   s.rows = g.rows; s.cols = g.cols; s.K = g.K; s.batch = g.batch;

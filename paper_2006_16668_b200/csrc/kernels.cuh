@@ -41,6 +41,8 @@ struct UmmaGemm {
   int a_stream, b_stream;    // operand is read once: load with an evict-first L2 hint
 };
 int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st);
+// umma2_gemm.cu: the same contraction with the two-SM MMA (CTA pairs, 256 x 256 tiles).
+int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st);
 
 // ffn_fused.cu: both expert GEMMs in one persistent launch; groups of four CTAs exchange 256-column
 // chunks of the hidden activations through a small L2-resident scratch ring.

@@ -77,6 +77,29 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
   }
 }
 
+// Whole-warp wait: lane 0 polls (sleeping between polls, the waits of an epilogue warp last
+// microseconds) while the other lanes park at the shuffle instead of all 32 spinning on the
+// barrier; the shuffle also orders the other lanes' later reads after lane 0's acquire.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int lane,
+                                               uint64_t limit_ns = 2000000000ull) {
+  int done = 1;
+  if (lane == 0) {
+    done = 0;
+    if (mbar_try_wait(bar, parity)) {
+      done = 1;
+    } else {
+      const uint64_t t0 = globaltimer_ns();
+      uint32_t it = 0;
+      while (true) {
+        if (mbar_try_wait(bar, parity)) { done = 1; break; }
+        __nanosleep(100);
+        if ((++it & 63u) == 0 && (*abort_flag || globaltimer_ns() - t0 > limit_ns)) break;
+      }
+    }
+  }
+  return __shfl_sync(0xffffffffu, done, 0) != 0;
+}
+
 // ---- TMA -----------------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");

@@ -1,0 +1,410 @@
+// Grouped bf16 GEMM with the two-SM tensor-core instruction (tcgen05.mma.cta_group::2): a pair of
+// CTAs (a cluster of two) computes a 256 x 256 output tile, each CTA holding 128 rows of A, HALF
+// of the B tile (128 of its 256 columns) and the accumulator of its own 128 rows in its TMEM.
+// Per 64-deep k-block a CTA loads 32 KB instead of the 48 KB a lone 128 x 256 tile needs, which
+// takes the operand feed (about 91 B/clk per SM for the one-SM kernel) below what an SM can draw
+// from L2 - the limit of the one-SM kernel on shapes with many rows per expert.
+//
+// Roles per CTA as in the one-SM kernel (warp 0 TMA producer, warp 1 MMA, warps 2..9 epilogue),
+// with the pair protocol:
+//   * both producers issue cta_group::2 TMA loads into their own shared memory that complete on
+//     the LEADER's (cluster rank 0) full barrier; the leader's producer arms it with the bytes of
+//     both CTAs.  No load is multicast.
+//   * only the leader's MMA thread issues tcgen05.mma.cta_group::2; tcgen05.commit multicasts the
+//     "stage free" and "accumulator complete" arrivals to the same barrier in both CTAs.
+//   * the peer's epilogue warps release the accumulator on the leader's barrier (remote arrive).
+//   * TMEM is allocated and freed with the cta_group::2 forms by warp 1 of both CTAs; cluster
+//     barriers order barrier initialisation before, and teardown after, all cross-CTA traffic.
+// Every mbarrier wait is bounded in wall time and reports GSHARD_ERR_TIMEOUT; a CTA that gave up
+// still reaches the final cluster barrier, so its peer is not left waiting.
+#include <cuda.h>
+
+#include "kernels.cuh"
+#include "sm100_ptx.cuh"
+#include "tensor_map.cuh"
+
+namespace gshard {
+
+namespace {
+
+constexpr int BM = 128, BK = 64, BN = 256, BNH = BN / 2;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kABytes = BM * BK * 2;          // 16 KB
+constexpr int kBBytes = BNH * BK * 2;         // 16 KB: this CTA's half of the B tile
+constexpr int kBoxBytes = 64 * 64 * 2;
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kStages = 6;
+constexpr int kTmemCols = 2 * BN;
+constexpr int kBarOff = kStages * kStageBytes;
+constexpr int kStgOff = kBarOff + 256;
+constexpr int kStgRowBytes = 128;
+constexpr int kStgWarpBytes = 32 * kStgRowBytes;
+constexpr int kSmemBytes = kStgOff + kEpiWarps * kStgWarpBytes + 1024;
+
+struct Params2 {
+  void* C;
+  const void* mask;
+  int rows, cols, K, batch;
+  long long c_ld, c_bs;
+  int m_tiles, n_tiles, total_tiles, k_blocks;   // tiles of 256 x 256
+  int out_f32, relu;
+  int a_stream, b_stream;
+  int n_fastest;
+  int* status;
+};
+
+struct TileCoord { int mt, nt, b; };
+
+__device__ __forceinline__ TileCoord decode(const Params2& p, int tile) {
+  TileCoord t;
+  t.mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
+  t.nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
+  t.b = tile / (p.m_tiles * p.n_tiles);
+  return t;
+}
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// tiled load into this CTA's shared memory, completion counted on a barrier given by its
+// shared::cluster address (the leader's); not multicast
+__device__ __forceinline__ void tma_load_3d_pair(void* smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
+                                                 int c0, int c1, int c2, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      :
+      : "r"(ptx::smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1),
+        "r"(c2), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_u32(smem_dst)),
+               "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t"
+      ".reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      "}"
+      :
+      : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once the MMAs issued
+// so far have completed (a tcgen05.commit, not a load)
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(ptx::smem_u32(bar)), "h"((uint16_t)3)
+      : "memory");
+}
+
+__device__ __forceinline__ void flush_rows2(const unsigned char* stg, const Params2& p, int b, int row0, int col0,
+                                            int lane) {
+  __syncwarp();
+  const int esz = p.out_f32 ? 4 : 2;
+  const int piece = lane & 7;
+  const int col = col0 + piece * (16 / esz);
+  unsigned char* cbase = reinterpret_cast<unsigned char*>(p.C) + ((long long)b * p.c_bs + col) * esz;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = 4 * i + (lane >> 3);
+    const int row = row0 + r;
+    if (row < p.rows && col < p.cols) {
+      const uint4 val = *reinterpret_cast<const uint4*>(stg + r * kStgRowBytes + ((piece ^ (r & 7)) * 16));
+      *reinterpret_cast<uint4*>(cbase + (long long)row * p.c_ld * esz) = val;
+    }
+  }
+  __syncwarp();
+}
+
+__device__ __forceinline__ void process_chunk2(const uint32_t* r, const Params2& p, unsigned char* srow, int lane,
+                                               int piece0, bool row_ok, long long row_off, int col0) {
+  float v[32];
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    v[i] = __uint_as_float(r[i]);
+    if (p.relu) v[i] = fmaxf(v[i], 0.f);
+  }
+  if (p.mask && row_ok) {
+    const __nv_bfloat16* mk = reinterpret_cast<const __nv_bfloat16*>(p.mask) + row_off + col0;
+    if (col0 + 32 <= p.cols) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint4 mv = __ldg(reinterpret_cast<const uint4*>(mk) + i);
+        const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t lo = w[j] & 0xffffu, hi = w[j] >> 16;      // bf16 > 0: sign clear, magnitude non-zero
+          if (!(lo != 0u && lo < 0x8000u)) v[8 * i + 2 * j] = 0.f;
+          if (!(hi != 0u && hi < 0x8000u)) v[8 * i + 2 * j + 1] = 0.f;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 32; ++i)
+        if (col0 + i < p.cols && !(__bfloat162float(mk[i]) > 0.f)) v[i] = 0.f;
+    }
+  }
+  if (p.out_f32) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      *reinterpret_cast<float4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16)) =
+          make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t w[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const __nv_bfloat162 pr = __floats2bfloat162_rn(v[8 * i + 2 * j], v[8 * i + 2 * j + 1]);
+        w[j] = *reinterpret_cast<const uint32_t*>(&pr);
+      }
+      *reinterpret_cast<uint4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+}
+
+template <bool A_K, bool B_K>
+__global__ void __launch_bounds__(kThreads, 1)
+umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const Params2 p) {
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBarOff);
+  uint64_t* full = bars;                      // [kStages]  used in the leader
+  uint64_t* empty = bars + kStages;           // [kStages]  in each CTA
+  uint64_t* acc_full = bars + 2 * kStages;    // [2]        in each CTA
+  uint64_t* acc_empty = acc_full + 2;         // [2]        used in the leader (both epilogues arrive)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();          // 0 = leader
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { ptx::mbar_init(full + s, 1); ptx::mbar_init(empty + s, 1); }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full + a, 1); ptx::mbar_init(acc_empty + a, 2 * kEpiWarps); }
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&map_a);
+    ptx::prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_slot, kTmemCols);
+    tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();                               // barriers of both CTAs initialised before any remote use
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  bool ok = true;
+  if (warp == 0) {
+    // ------------------------------ TMA producer (both CTAs) -------------------------------
+    if (lane == 0) {
+      const uint64_t pol_a = p.a_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
+      const uint64_t pol_b = p.b_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
+      int stage = 0; uint32_t phase = 0;
+      for (int tile = pair; tile < p.total_tiles && ok; tile += n_pairs) {
+        const TileCoord t = decode(p, tile);
+        const int row0 = t.mt * 2 * BM + (int)rank * BM;      // this CTA's 128 rows of the 256-row tile
+        const int col0 = t.nt * BN + (int)rank * BNH;         // this CTA's half of the B columns
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!ptx::mbar_wait(empty + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+          unsigned char* sa = smem + stage * kStageBytes;
+          unsigned char* sb = sa + kABytes;
+          const uint32_t bar = map_to_cta(ptx::smem_u32(full + stage), 0);
+          if (rank == 0) ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)(2 * kStageBytes));
+          if (A_K) {
+            tma_load_3d_pair(sa, &map_a, bar, kb * BK, row0, t.b, pol_a);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j)
+              tma_load_3d_pair(sa + j * kBoxBytes, &map_a, bar, row0 + j * 64, kb * BK, t.b, pol_a);
+          }
+          if (B_K) {
+            tma_load_3d_pair(sb, &map_b, bar, kb * BK, col0, t.b, pol_b);
+          } else {
+#pragma unroll
+            for (int j = 0; j < BNH / 64; ++j)
+              tma_load_3d_pair(sb + j * kBoxBytes, &map_b, bar, col0 + j * 64, kb * BK, t.b, pol_b);
+          }
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer (leader only) -------------------------------
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_bf16(2 * BM, BN, !A_K, !B_K);
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      for (int tile = pair; tile < p.total_tiles && ok; tile += n_pairs) {
+        if (!ptx::mbar_wait(acc_empty + acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < p.k_blocks; ++kb) {
+          if (!ptx::mbar_wait(full + stage, phase, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after_sync();
+          const uint32_t sa = ptx::smem_u32(smem + stage * kStageBytes);
+          const uint32_t sb = sa + kABytes;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t da = A_K ? ptx::make_smem_desc(sa + k * 32, 16, 1024)
+                                    : ptx::make_smem_desc(sa + k * 2048, kBoxBytes, 1024);
+            const uint64_t db = B_K ? ptx::make_smem_desc(sb + k * 32, 16, 1024)
+                                    : ptx::make_smem_desc(sb + k * 2048, kBoxBytes, 1024);
+            umma_bf16_pair(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit_pair(empty + stage);             // stage free in both CTAs
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        umma_commit_pair(acc_full + acc);              // accumulator complete in both CTAs
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue (both CTAs, own 128 rows) ----------------------
+    const int ew = warp - 2;
+    const int q = warp & 3;
+    const int half = ew >> 2;
+    constexpr int kHalfCols = BN / 2;
+    unsigned char* stg = smem + kStgOff + ew * kStgWarpBytes;
+    unsigned char* srow = stg + lane * kStgRowBytes;
+    int acc = 0; uint32_t acc_phase = 0;
+    for (int tile = pair; tile < p.total_tiles && ok; tile += n_pairs) {
+      const TileCoord t = decode(p, tile);
+      if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
+      ptx::tc_fence_after_sync();
+      const int row0 = t.mt * 2 * BM + (int)rank * BM + q * 32;
+      const bool row_ok = row0 + lane < p.rows;
+      const long long row_off = (long long)t.b * p.c_bs + (long long)(row0 + lane) * p.c_ld;
+      const uint32_t t_acc = tmem_base + (uint32_t)(acc * BN + half * kHalfCols) + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < kHalfCols / 64; ++c) {
+        const int col0 = t.nt * BN + half * kHalfCols + c * 64;
+        if (col0 >= p.cols) break;
+        uint32_t r0[32], r1[32];
+        ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r0);
+        ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r1);
+        ptx::tmem_ld_wait();
+        if (p.out_f32) {
+          process_chunk2(r0, p, srow, lane, 0, row_ok, row_off, col0);
+          flush_rows2(stg, p, t.b, row0, col0, lane);
+          process_chunk2(r1, p, srow, lane, 0, row_ok, row_off, col0 + 32);
+          flush_rows2(stg, p, t.b, row0, col0 + 32, lane);
+        } else {
+          process_chunk2(r0, p, srow, lane, 0, row_ok, row_off, col0);
+          process_chunk2(r1, p, srow, lane, 4, row_ok, row_off, col0 + 32);
+          flush_rows2(stg, p, t.b, row0, col0, lane);
+        }
+      }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(map_to_cta(ptx::smem_u32(acc_empty + acc), 0));   // the leader's barrier
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // ------------------------------ teardown ---------------------------------------------------
+  if (!ok) {
+    *abort_flag = 1;
+    set_device_status(p.status, GSHARD_ERR_TIMEOUT);
+    const uint64_t t0 = ptx::globaltimer_ns();
+    while (ptx::globaltimer_ns() - t0 < 2000000ull) { __nanosleep(1000); }
+  }
+  __syncwarp();
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();                  // no CTA frees TMEM or exits while its peer may still use it
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, kTmemCols);
+  }
+}
+
+template <bool A_K, bool B_K>
+int launch2_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params2& p, int pairs, cudaStream_t st) {
+  auto kern = umma2_gemm_kernel<A_K, B_K>;
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+    return GSHARD_ERR_CUDA;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2 * pairs, 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, kern, ma, mb, p) != cudaSuccess) { cudaGetLastError(); return GSHARD_ERR_CUDA; }
+  count_launch();
+  return GSHARD_OK;
+}
+
+}  // namespace
+
+// C[b] = act(A[b] . B[b]) with 256 x 256 tiles on CTA pairs; same operand conventions as
+// launch_umma_gemm.  Worth it when a problem has more than one 128-row tile.
+int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
+  if (g.rows <= 0 || g.cols <= 0 || g.K <= 0 || g.batch <= 0) return GSHARD_OK;
+  CUtensorMap ma, mb;
+  bool okm;
+  if (g.a_kmajor) okm = make_map(&ma, g.A, g.K, g.rows, g.batch, g.a_ld, g.a_bs, BK, BM);
+  else            okm = make_map(&ma, g.A, g.rows, g.K, g.batch, g.a_ld, g.a_bs, 64, BK);
+  if (g.b_kmajor) okm = okm && make_map(&mb, g.B, g.K, g.cols, g.batch, g.b_ld, g.b_bs, BK, BNH);
+  else            okm = okm && make_map(&mb, g.B, g.cols, g.K, g.batch, g.b_ld, g.b_bs, 64, BK);
+  if (!okm) return GSHARD_ERR_CUDA;
+  Params2 p;
+  p.C = g.C; p.mask = g.mask; p.rows = g.rows; p.cols = g.cols; p.K = g.K; p.batch = g.batch;
+  p.c_ld = g.c_ld; p.c_bs = g.c_bs;
+  p.m_tiles = ceil_div(g.rows, 2 * BM); p.n_tiles = ceil_div(g.cols, BN);
+  p.total_tiles = p.m_tiles * p.n_tiles * g.batch;
+  p.k_blocks = ceil_div(g.K, BK);
+  p.out_f32 = g.out_f32; p.relu = g.relu; p.a_stream = g.a_stream; p.b_stream = g.b_stream;
+  p.n_fastest = (g.rows > g.cols) ? 1 : 0;
+  p.status = status;
+  int sms = 148, dev = 0;
+  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  int pairs = sms / 2;
+  if (pairs > p.total_tiles) pairs = p.total_tiles;
+  if (g.a_kmajor && g.b_kmajor) return launch2_t<true, true>(ma, mb, p, pairs, st);
+  if (g.a_kmajor && !g.b_kmajor) return launch2_t<true, false>(ma, mb, p, pairs, st);
+  if (!g.a_kmajor && g.b_kmajor) return launch2_t<false, true>(ma, mb, p, pairs, st);
+  return launch2_t<false, false>(ma, mb, p, pairs, st);
+}
+
+}  // namespace gshard

@@ -245,7 +245,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
       const TileCoord t = decode(p, tile);
-      if (!ptx::mbar_wait(acc_full + acc, acc_phase, abort_flag)) { ok = false; break; }
+      if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       const int row0 = t.mt * BM + q * 32;
       const bool row_ok = row0 + lane < p.rows;

@@ -55,6 +55,8 @@ BWD_CASES = [
     ("bf16_umma", 2, 256, 128, 256, 16, 24, "bf16", 0, GRAD_TOL),
     ("bf16_umma_ragged", 3, 200, 192, 320, 32, 5, "bf16", 0, GRAD_TOL),
     ("bf16_umma_variant_a", 2, 256, 128, 256, 16, 20, "bf16", B.GSHARD_FLAG_SECOND_SKIP_FREES_SLOT, GRAD_TOL),
+    # every grouped GEMM with more than 128 rows on CTA pairs (all four operand-layout variants)
+    ("bf16_two_sm", 2, 384, 256, 512, 16, 80, "bf16", B.GSHARD_FLAG_TWO_SM_MMA, GRAD_TOL),
 ]
 
 

@@ -129,6 +129,10 @@ FFN_CASES = [
     (37, 1, 1, 64, 1024, "bf16", B.GSHARD_FLAG_FUSED_FFN),       # one row per expert, 16 columns per rank
     (150, 1, 128, 1024, 1024, "bf16", B.GSHARD_FLAG_FUSED_FFN),  # more units than groups, uneven split
     (2, 3, 128, 448, 2048, "bf16", B.GSHARD_FLAG_FUSED_FFN),     # three full row tiles, 112 columns per rank
+    # grouped GEMMs on CTA pairs (two-SM MMA): ragged 256-row tiles, odd tile counts
+    (2, 2, 100, 1024, 2048, "bf16", B.GSHARD_FLAG_TWO_SM_MMA),   # 200 rows: second CTA of the pair ragged
+    (3, 4, 96, 512, 1024, "bf16", B.GSHARD_FLAG_TWO_SM_MMA),     # 384 rows: two pair tiles, second half empty
+    (5, 8, 128, 256, 1536, "bf16", B.GSHARD_FLAG_TWO_SM_MMA),    # 1024 rows, more tiles than pairs
 ]
 
 
