@@ -88,7 +88,7 @@ class ClockSampler(threading.Thread):
                 "reasons": reasons, "samples": len(self.samples), "samples_under_load": len(busy)}
 
 
-def oracle_sample(cfg, n_groups=8, n_rows=400, seed_offset=0):
+def oracle_sample(cfg, n_groups=16, n_rows=1200, seed_offset=0):
     """Times the CPU oracle on a bounded sample of the configuration: gating + Algorithm 1 for
     n_groups whole groups, eq. (2)-(3) for n_rows token-expert rows of those groups.  Returns
     (tokens/s of a full layer at that per-token cost, description, threads)."""
@@ -250,9 +250,16 @@ def main():
     sampler = ClockSampler(local_rank)
     sampler.start()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    # event pairs recorded by the library around the expert FFN of each timed step (the dominant
+    # kernel); recorded once here so that their handles exist before they are handed over
+    ffn_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in ffn_ev:
+        a.record(stream)
+        b.record(stream)
     barrier()
     ev[0].record(stream)
     for i in range(args.steps):
+        B.gshard_moe_time_expert_ffn(*ffn_ev[i])
         step()
         ev[i + 1].record(stream)
     barrier()
@@ -264,32 +271,28 @@ def main():
     ms_per_step = total_ms / args.steps
     value = world * cfg.N / (ms_per_step * 1e-3)
 
-    # ---- dominant kernel: the expert FFN's grouped GEMM (two launches per step) -----------------
+    # ---- dominant kernel: the expert FFN, timed inside the steps above --------------------------
     peaks = load_peaks()
-    buf = torch.empty(cfg.E, cfg.G * cfg.C, cfg.M, dtype=cfg.torch_dtype, device=dev)
-    B.gshard_moe_dispatch(shape, inp["x"], rt["slot_token"], buf, stream)
-    out = torch.empty_like(buf)
-    for _ in range(2):
-        B.gshard_moe_expert_ffn(shape, buf, inp["wi"], inp["wo"], out, ws, stream)
-    torch.cuda.synchronize()
-    k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    k0.record(stream)
-    for _ in range(args.steps):
-        B.gshard_moe_expert_ffn(shape, buf, inp["wi"], inp["wo"], out, ws, stream)
-    k1.record(stream)
-    torch.cuda.synchronize()
-    ffn_ms = k0.elapsed_time(k1) / args.steps
+    ffn_ms = sum(a.elapsed_time(b) for a, b in ffn_ev) / args.steps
     es = 2 if cfg.dtype == "bf16" else 4
     R = cfg.E * cfg.G * cfg.C
     ffn_bytes = 2 * cfg.E * cfg.M * cfg.H * es + 2 * R * cfg.M * es      # weights + buf in + out
     ffn_flops = 4.0 * R * cfg.M * cfg.H
-    fused = args.fused_ffn or (not args.unfused_ffn and cfg.G * cfg.C <= 128 and cfg.dtype == "bf16")
+    fused = (cfg.dtype == "bf16" and not train and
+             (args.fused_ffn or (not args.unfused_ffn and cfg.G * cfg.C <= 128)))
     n_launch = 1 if fused else 2                              # launches of the FFN per step
     launch_ms = ffn_ms / n_launch
     achieved = (ffn_bytes / n_launch) / (launch_ms * 1e-3) / 1e9
     kname = "ffn_group4_kernel (expert FFN, 1 launch)" if fused else "umma_gemm_kernel (expert FFN, 2 launches)"
+    # DRAM bytes per launch from the ncu capture of the 64-expert slice of this shape, scaled by the
+    # expert count (profiles/ffn_group4_p4_slice.md); only known for the single-launch kernel at the
+    # MoE(2048E) per-expert shape
+    traffic = None
+    if fused and (cfg.M, cfg.H, cfg.G * cfg.C) == (1024, 8192, 128):
+        traffic = cfg.E / 64.0 * (2.164371e9 + 33.554432e6)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "kernel": kname,
+                "frac": achieved / peaks["hbm_gbs"], "traffic": traffic, "traffic_unit": "bytes per launch",
+                "algorithmic_bytes": ffn_bytes / n_launch, "kernel": kname,
                 "peak_source": peaks["source"], "launch_ms": launch_ms,
                 "ffn_tflops": ffn_flops / (ffn_ms * 1e-3) / 1e12}
     # whole-layer roofline: slower of FLOPs at the tensor peak and bytes at the HBM peak

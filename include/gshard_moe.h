@@ -207,6 +207,13 @@ int gshard_moe_last_device_status(void* workspace, void* cuda_stream);
 /* Number of kernels the last forward/backward/stage call on this thread launched. */
 int gshard_moe_last_launch_count(void);
 
+/* Measurement hook: the NEXT gshard_moe_top2_forward call on this thread records start_event
+ * before and stop_event after its expert-FFN launches (eq. (2)) on the call's stream
+ * (cudaEvent_t handles passed as void*, created with timing enabled, owned by the caller).  The
+ * pair is used once; pass two NULLs to disarm.  Lets a benchmark time the dominant kernel inside
+ * its timed region instead of in a loop of its own. */
+int gshard_moe_time_expert_ffn(void* start_event, void* stop_event);
+
 #ifdef __cplusplus
 }
 #endif

@@ -66,6 +66,7 @@ EXPORTS = {
     "gshard_moe_combine": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6),
     "gshard_moe_last_device_status": (c_int, [c_void_p, c_void_p]),
     "gshard_moe_last_launch_count": (c_int, []),
+    "gshard_moe_time_expert_ffn": (c_int, [c_void_p, c_void_p]),
 }
 
 _lib = None
@@ -239,3 +240,11 @@ def gshard_moe_last_device_status(workspace, stream=None) -> int:
 
 def gshard_moe_last_launch_count() -> int:
     return int(load().gshard_moe_last_launch_count())
+
+
+def gshard_moe_time_expert_ffn(start_event, stop_event):
+    """Arm torch.cuda.Event pair (enable_timing=True, already recorded once so that their handles
+    exist) around the expert FFN of the next forward call; (None, None) disarms."""
+    s = None if start_event is None else start_event.cuda_event
+    e = None if stop_event is None else stop_event.cuda_event
+    _check(load().gshard_moe_time_expert_ffn(s, e), "gshard_moe_time_expert_ffn")

@@ -13,6 +13,12 @@ LaunchCounter& launch_counter() {
   return c;
 }
 
+struct FfnTiming { void* start = nullptr; void* stop = nullptr; };
+static FfnTiming& ffn_timing() {
+  static thread_local FfnTiming t;
+  return t;
+}
+
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -150,7 +156,13 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
   GS_TRY(launch_capacity(d, expert_idx, gate12, u, m, slot, weight, flags, first_count, total_count, slot_token,
                          l_aux_group, stats_group, l_aux, reinterpret_cast<long long*>(r.stats), st));
   launch_dispatch(d, x, slot_token, buf, st);
+  // optional event pair around the expert FFN, armed for one call by gshard_moe_time_expert_ffn
+  FfnTiming& ft = ffn_timing();
+  const bool timed = ft.start != nullptr && ft.stop != nullptr;
+  if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.start), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   GS_TRY(ffn_stage(d, buf, wi, wo, h, save, out, ws + pl.ffn_scratch, status, st));
+  if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.stop), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  ft.start = ft.stop = nullptr;
   launch_combine(d, out, expert_idx, slot, weight, y, st);
 
   if (save) {   // hand the caller the routing tensors it asked for
@@ -358,5 +370,12 @@ int gshard_moe_last_device_status(void* workspace, void* cuda_stream) {
 }
 
 int gshard_moe_last_launch_count(void) { return launch_counter().n; }
+
+int gshard_moe_time_expert_ffn(void* start_event, void* stop_event) {
+  if ((start_event == nullptr) != (stop_event == nullptr)) return GSHARD_ERR_INVALID_ARG;
+  ffn_timing().start = start_event;
+  ffn_timing().stop = stop_event;
+  return GSHARD_OK;
+}
 
 }  // extern "C"
