@@ -55,7 +55,9 @@ __device__ __forceinline__ void rank_chunk(const CapacityArgs& a, int g, int k, 
     const int s = base + lane;
     const bool valid = s < hi;
     const long long t = (long long)g * a.S + (valid ? s : lo);
-    int key = valid ? a.expert_idx[2 * t + k] : -1 - lane;
+    // expert ids index shared-memory histograms: ids outside [0,E) (possible only through the
+    // stage entry point, which takes them from the caller) are clamped instead of trusted
+    int key = valid ? min(max(a.expert_idx[2 * t + k], 0), a.E - 1) : -1 - lane;
     bool counts = valid;
     if (second_pass && a.variant_a && valid) counts = (a.flags[t] & 2u) != 0;
     if (!counts) key = -1 - lane;           // unique key: matches nobody
@@ -113,7 +115,7 @@ __global__ void __launch_bounds__(kCapThreads) capacity_kernel(CapacityArgs a) {
   int n_first_dropped = 0, n_rnd_skipped = 0, n_cap_dropped = 0, n_overflowed = 0, n_filled = 0;
   for (int s = lo + (tid & 31); s < hi; s += 32) {
     const long long t = (long long)g * a.S + s;
-    const int e1 = a.expert_idx[2 * t];
+    const int e1 = min(max(a.expert_idx[2 * t], 0), a.E - 1);
     const float g1 = a.gate12[2 * t], g2 = a.gate12[2 * t + 1];
     const float den = g1 + g2;
     const float w1 = g1 / den, w2 = g2 / den;
@@ -152,7 +154,7 @@ __global__ void __launch_bounds__(kCapThreads) capacity_kernel(CapacityArgs a) {
   __syncthreads();
   for (int s = lo + (tid & 31); s < hi; s += 32) {
     const long long t = (long long)g * a.S + s;
-    const int e2 = a.expert_idx[2 * t + 1];
+    const int e2 = min(max(a.expert_idx[2 * t + 1], 0), a.E - 1);
     unsigned f = a.flags[t];
     const bool pass = (f & 2u) != 0;
     const int pos = (int)hist[(size_t)w * a.E + e2] + a.slot[2 * t + 1];

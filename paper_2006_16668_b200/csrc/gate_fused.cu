@@ -21,14 +21,19 @@ namespace gshard {
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kABytes = BM * BK * 2;
 constexpr int kBBytes = BN * BK * 2;
 constexpr int kBoxBytes = 64 * 64 * 2;
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kStages = 4;
 constexpr int kTmemCols = 2 * BN;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 + 256;
+constexpr int kBarOff = kStages * kStageBytes;
+constexpr int kStgOff = kBarOff + 256;
+constexpr int kStgRowBytes = 128;
+constexpr int kStgWarpBytes = 32 * kStgRowBytes;
+constexpr int kSmemBytes = kStgOff + kEpiWarps * kStgWarpBytes + 1024;
 
 struct GateParams {
   long long N;          // tokens
@@ -41,6 +46,22 @@ struct GateParams {
   float* rowinv;        // [N] 1 / sum exp(logit - rowmax)
   int* status;
 };
+
+// (v1,i1),(v2,i2) <- top-2 of the union with (b1,k1),(b2,k2); larger value first, lower expert
+// index on equal values.
+__device__ __forceinline__ void top2_merge(float& v1, int& i1, float& v2, int& i2, float b1, int k1, float b2, int k2) {
+  const bool first = b1 > v1 || (b1 == v1 && k1 < i1);          // the other set's best beats v1
+  // candidates for second place: the loser of that comparison and the winner's own second
+  const float l_v = first ? v1 : b1;
+  const int l_i = first ? i1 : k1;
+  const float w_v = first ? b2 : v2;
+  const int w_i = first ? k2 : i2;
+  v1 = first ? b1 : v1;
+  i1 = first ? k1 : i1;
+  const bool second = l_v > w_v || (l_v == w_v && l_i < w_i);
+  v2 = second ? l_v : w_v;
+  i2 = second ? l_i : w_i;
+}
 
 __device__ __forceinline__ int tile_cols(const GateParams& p, int nt) {   // multiple of 16, <= BN
   const int left = p.E - nt * BN;
@@ -58,13 +79,17 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
   uint64_t* empty = bars + kStages;
   uint64_t* acc_full = bars + 2 * kStages;
   uint64_t* acc_empty = acc_full + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* x_full = acc_empty + 2;            // upper-half results of a row tile written
+  uint64_t* x_empty = x_full + 1;              // ... and read
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(x_empty + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { ptx::mbar_init(full + s, 1); ptx::mbar_init(empty + s, 1); }
-    for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full + a, 1); ptx::mbar_init(acc_empty + a, 4); }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full + a, 1); ptx::mbar_init(acc_empty + a, kEpiWarps); }
+    ptx::mbar_init(x_full, kEpiWarps / 2);
+    ptx::mbar_init(x_empty, kEpiWarps / 2);
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&map_x);
@@ -132,19 +157,31 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       }
     }
   } else {
-    // epilogue: thread = token (TMEM lane); state carried across the column tiles of a row tile.
-    // The running top-2 and the exp-sum are kept as four independent chains (columns i mod 4) so
-    // that the per-element updates overlap instead of forming one long dependency chain; each
-    // chain scans its columns in ascending order with strict comparisons, and the chains are
-    // merged at the end of the row with an explicit lowest-index tie rule.
+    // epilogue: two warps per TMEM lane quarter; a thread owns one token (lane) and one half of
+    // each column tile, and carries its state across the column tiles of the row tile.  The
+    // running top-2 and the exp-sum are kept as four independent chains (columns i mod 4) so that
+    // the per-element updates overlap instead of forming one long dependency chain; each chain
+    // scans its columns in ascending order with strict comparisons, and chains (and then the two
+    // halves, through shared memory) are merged with an explicit lowest-index tie rule.
+    const int ew = warp - 2;
     const int q = warp & 3;
-    int acc = 0; uint32_t acc_phase = 0;
+    const int half = ew >> 2;
+    constexpr int kHalfCols = BN / 2;
+    unsigned char* stg = smem + kStgOff + ew * kStgWarpBytes;       // 32 rows x 128 B staging
+    unsigned char* srow = stg + lane * kStgRowBytes;
+    // exchange slot of this token: the staging row of the half-1 warp of the same lane quarter
+    float* xchg = reinterpret_cast<float*>(smem + kStgOff + ((4 + (ew & 3)) * kStgWarpBytes) + lane * kStgRowBytes);
+    int acc = 0; uint32_t acc_phase = 0, x_phase = 0;
     const float ninf = __int_as_float(0xff800000);
     constexpr float kLog2e = 1.4426950408889634f;
     for (int rt = blockIdx.x; rt < p.row_tiles && ok; rt += gridDim.x) {
-      const long long row = (long long)rt * BM + q * 32 + lane;
+      // the exchange slots alias the upper-half warps' staging rows: those warps may not stage
+      // logits of this row tile before the previous tile's results have been read
+      if (half == 1 && !ptx::mbar_wait_warp(x_empty, x_phase ^ 1u, abort_flag, lane)) { ok = false; break; }
+      const long long row0 = (long long)rt * BM + q * 32;
+      const long long row = row0 + lane;
       const bool row_ok = row < p.N;
-      float m = ninf;                        // running row maximum
+      float m = ninf;                        // running maximum of this thread's columns
       float s4[4] = {0.f, 0.f, 0.f, 0.f};    // partial sums of exp(logit - m)
       float a1[4], a2[4];                    // per chain: two largest logits ...
       int j1[4], j2[4];                      // ... and their expert indices
@@ -153,20 +190,20 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
       for (int nt = 0; nt < p.n_tiles; ++nt) {
         if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
         ptx::tc_fence_after_sync();
-        const int ncols = min(BN, p.E - nt * BN);       // valid columns of this tile
-        const uint32_t t_acc = tmem_base + (uint32_t)(acc * BN) + ((uint32_t)(q * 32) << 16);
+        const uint32_t t_acc = tmem_base + (uint32_t)(acc * BN + half * kHalfCols) + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
-        for (int c = 0; c * 64 < ncols; ++c) {          // 64 columns per round: two TMEM loads in flight
+        for (int c = 0; c < kHalfCols / 64; ++c) {      // 64 columns per round: two TMEM loads in flight
+          const int cbase = nt * BN + half * kHalfCols + c * 64;
+          if (cbase >= p.E) break;                       // uniform over the warp
           uint32_t r[2][32];
           ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r[0]);
           ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r[1]);
           ptx::tmem_ld_wait();
-          if (!row_ok) continue;
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
-            const int col0 = nt * BN + c * 64 + hh * 32;
+            const int col0 = cbase + hh * 32;
             const int nv = min(32, p.E - col0);
-            if (nv <= 0) break;
+            if (nv <= 0) break;                          // uniform over the warp
             float v[32];
             float cm[4] = {ninf, ninf, ninf, ninf};
 #pragma unroll
@@ -193,15 +230,26 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
               a1[k] = gt1 ? v[i] : a1[k];
               j1[k] = gt1 ? col0 + i : j1[k];
             }
-            float* dst = p.logits + row * p.E + col0;
-            if (nv == 32) {
+            // logits: stage the 32 fp32 of this row (one 128-byte staging row, XOR-swizzled pieces),
+            // then write 128-byte row segments: 8 lanes per row, 4 rows per instruction
 #pragma unroll
-              for (int i = 0; i < 8; ++i)
-                __stcs(reinterpret_cast<float4*>(dst) + i, make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
-            } else {
+            for (int i = 0; i < 8; ++i)
+              *reinterpret_cast<float4*>(srow + ((i ^ (lane & 7)) * 16)) =
+                  make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            __syncwarp();
+            {
+              const int piece = lane & 7;
+              const int col = col0 + piece * 4;
 #pragma unroll
-              for (int i = 0; i < 32; ++i) if (i < nv) dst[i] = v[i];
+              for (int i = 0; i < 8; ++i) {
+                const int rr = 4 * i + (lane >> 3);
+                if (row0 + rr < p.N && col < p.E) {
+                  const float4 val = *reinterpret_cast<const float4*>(stg + rr * kStgRowBytes + ((piece ^ (rr & 7)) * 16));
+                  __stcs(reinterpret_cast<float4*>(p.logits + (row0 + rr) * p.E + col), val);
+                }
+              }
             }
+            __syncwarp();
           }
         }
         ptx::tc_fence_before_sync();
@@ -210,33 +258,42 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
       if (!ok) break;
-      if (row_ok) {
-        // merge the four chains: larger value first, lower index on equal values
-        float v1 = a1[0], v2 = a2[0];
-        int i1 = j1[0], i2 = j2[0];
+      // merge this thread's four chains: larger value first, lower index on equal values
+      float v1 = a1[0], v2 = a2[0];
+      int i1 = j1[0], i2 = j2[0];
 #pragma unroll
-        for (int k = 1; k < 4; ++k) {
-          const bool b1 = a1[k] > v1 || (a1[k] == v1 && j1[k] < i1);       // chain's best beats v1
-          // candidates for the new second place: loser of the first comparison and the winner's second
-          const float l_v = b1 ? v1 : a1[k];
-          const int l_i = b1 ? i1 : j1[k];
-          const float w2_v = b1 ? a2[k] : v2;
-          const int w2_i = b1 ? j2[k] : i2;
-          v1 = b1 ? a1[k] : v1;
-          i1 = b1 ? j1[k] : i1;
-          const bool b2 = l_v > w2_v || (l_v == w2_v && l_i < w2_i);
-          v2 = b2 ? l_v : w2_v;
-          i2 = b2 ? l_i : w2_i;
-        }
-        const float ssum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+      for (int k = 1; k < 4; ++k) top2_merge(v1, i1, v2, i2, a1[k], j1[k], a2[k], j2[k]);
+      float ssum = (s4[0] + s4[1]) + (s4[2] + s4[3]);
+      // hand the upper half's result to the thread that owns the lower half of the same token
+      // (bounded mbarrier hand-shake instead of a CTA barrier, so that a warp that gave up on a
+      // wait cannot leave the others stuck)
+      if (half == 1) {
+        xchg[0] = m; xchg[1] = ssum; xchg[2] = v1; xchg[3] = v2;
+        reinterpret_cast<int*>(xchg)[4] = i1; reinterpret_cast<int*>(xchg)[5] = i2;
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(x_full);
+      } else {
+        if (!ptx::mbar_wait_warp(x_full, x_phase, abort_flag, lane)) { ok = false; break; }
+      }
+      if (half == 0 && row_ok) {
+        const float m1 = xchg[0], s1 = xchg[1];
+        top2_merge(v1, i1, v2, i2, xchg[2], reinterpret_cast<const int*>(xchg)[4], xchg[3],
+                   reinterpret_cast<const int*>(xchg)[5]);
+        const float mm = fmaxf(m, m1);
+        ssum = ssum * expf(m - mm) + s1 * expf(m1 - mm);   // exp(-inf) = 0 when a half had no columns
         const float inv = 1.0f / ssum;
         p.expert_idx[2 * row] = i1;
         p.expert_idx[2 * row + 1] = i2;
-        p.gate12[2 * row] = inv;                          // exp(v1 - m) = 1
-        p.gate12[2 * row + 1] = expf(v2 - m) * inv;
-        p.rowmax[row] = m;
+        p.gate12[2 * row] = inv;                          // exp(v1 - mm) = 1
+        p.gate12[2 * row + 1] = expf(v2 - mm) * inv;
+        p.rowmax[row] = mm;
         p.rowinv[row] = inv;
       }
+      if (half == 0) {
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(x_empty);          // exchange slots free again
+      }
+      x_phase ^= 1u;
     }
   }
 
