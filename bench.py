@@ -45,6 +45,22 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Device time of the slowest rank (every rank calls this; one all-reduce when world > 1)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job tokens/s: every rank (replica) processes tokens_per_rank per step (weak scaling)."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons with one looping nvidia-smi while timed regions run."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -263,13 +279,9 @@ def main():
         step()
         ev[i + 1].record(stream)
     barrier()
-    total_ms = ev[0].elapsed_time(ev[-1])
-    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(ev[0].elapsed_time(ev[-1]), world, dev)
     ms_per_step = total_ms / args.steps
-    value = world * cfg.N / (ms_per_step * 1e-3)
+    value = aggregate_throughput(cfg.N, world, ms_per_step)
 
     # ---- dominant kernel: the expert FFN, timed inside the steps above --------------------------
     peaks = load_peaks()
@@ -323,11 +335,8 @@ def main():
             B.gshard_moe_top2_forward_host(shape, xh, inp["wg"], inp["wi"], inp["wo"], uh, yh, lh, None, ws, stream)
         h1.record(stream)
         barrier()
-        tt = torch.tensor([h0.elapsed_time(h1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tt.item()) / args.steps
-        e2e = {"value": world * cfg.N / (e2e_ms * 1e-3), "unit": UNIT,
+        e2e_ms = max_over_ranks(h0.elapsed_time(h1), world, dev) / args.steps
+        e2e = {"value": aggregate_throughput(cfg.N, world, e2e_ms), "unit": UNIT,
                "h2d_bytes_per_step": xh.numel() * xh.element_size() + uh.numel() * 4,
                "d2h_bytes_per_step": yh.numel() * yh.element_size() + 4, "ms_per_step": e2e_ms,
                "note": "expert and gating weights stay resident on the device (model state)"}
