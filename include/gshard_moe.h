@@ -69,7 +69,7 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,
- * E >= 2, S < 65536, E <= 16384; dtype BF16 without SIMT flag also needs M % 64 == 0,
+ * E >= 2, S <= 32767, C <= 32767, E <= 16384; dtype BF16 without SIMT flag also needs M % 64 == 0,
  * H % 64 == 0, E % 16 == 0. */
 typedef struct {
   int32_t G, S, M, H, E, C;

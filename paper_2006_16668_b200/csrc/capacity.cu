@@ -216,12 +216,9 @@ int launch_capacity(const Dims& d, const int32_t* expert_idx, const float* gate1
   a.total_count = total_count; a.slot_token = slot_token; a.l_aux_group = l_aux_group;
   a.stats_group = stats_group;
   const size_t smem = capacity_smem_bytes(d.E, a.warps_used);
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(capacity_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-      return GSHARD_ERR_CUDA;
-    attr_set = true;
-  }
+  // set on every launch: the attribute is per device, and the call is cheap
+  if (cudaFuncSetAttribute(capacity_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+    return GSHARD_ERR_CUDA;
   capacity_kernel<<<d.G, kCapThreads, smem, st>>>(a);
   capacity_finalize_kernel<<<1, 32, 0, st>>>(l_aux_group, stats_group, d.G, l_aux, stats);
   count_launch(2);

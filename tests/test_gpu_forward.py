@@ -147,6 +147,31 @@ def test_umma_matches_simt_contractions():
     assert same > 0.999
 
 
+def test_expert_ffn_timing_hook():
+    # the event pair armed by gshard_moe_time_expert_ffn brackets the expert FFN of the next
+    # forward call only
+    cfg = MoEConfig("hook", G=2, S=512, M=256, H=1024, E=32, C=40, dtype="bf16", seed=78)
+    inp = make_inputs(cfg, "cuda")
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(); b.record()                         # materialise the handles
+    torch.cuda.synchronize()
+    B.gshard_moe_time_expert_ffn(a, b)
+    s0.record()
+    run_forward(cfg, inp)
+    s1.record()
+    torch.cuda.synchronize()
+    ffn_ms, all_ms = a.elapsed_time(b), s0.elapsed_time(s1)
+    assert 0.0 < ffn_ms < all_ms
+    # a second call is not timed: the events keep their values
+    run_forward(cfg, inp)
+    torch.cuda.synchronize()
+    assert a.elapsed_time(b) == ffn_ms
+    with pytest.raises(B.GshardError):
+        B.load().gshard_moe_time_expert_ffn.restype = B.c_int
+        B._check(B.load().gshard_moe_time_expert_ffn(a.cuda_event, None), "one-sided event pair")
+
+
 FULL = [("c2_128e", [0, 9], 6), ("c3_512e_skew", [3, 15], 6), ("c4_2048e", [0, 17, 31], 5)]
 
 
