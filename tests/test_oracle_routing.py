@@ -4,6 +4,8 @@ closed forms.  None of these retypes the oracle's loops: the expected values com
 from hand arithmetic, from counting definitions evaluated by brute force, or from
 special cases with a known answer.
 """
+import json
+import os
 from fractions import Fraction as Fr
 
 import numpy as np
@@ -52,36 +54,49 @@ def _example_inputs():
     return x, wg, wi, wo, U.reshape(1, S)
 
 
+GOLDEN = json.load(open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "alg1_worked_example.json")))
+
+
+def _fr(v):
+    return float(Fr(v))
+
+
+def test_golden_file_matches_the_inputs_used_here():
+    assert np.array_equal(np.array(GOLDEN["gate_probabilities"]), P)
+    assert np.allclose(np.array(GOLDEN["u"], np.float32), U)
+    assert GOLDEN["token_tag"] == TAG.astype(int).tolist()
+
+
 def test_worked_example_default_reading():
     x, wg, wi, wo, u = _example_inputs()
-    f = orc.forward(x, wg, wi, wo, u, C=2)
-    assert f.expert_idx[0].tolist() == [[0, 1], [0, 2], [0, 1], [1, 2], [2, 1]]
-    assert f.slot[0].tolist() == [[0, 1], [1, -1], [-1, -1], [0, -1], [0, -1]]
-    w_exp = [[Fr(2, 3), Fr(1, 3)], [Fr(5, 9), Fr(4, 9)], [Fr(7, 9), Fr(2, 9)],
-             [Fr(5, 8), Fr(3, 8)], [Fr(2, 3), Fr(1, 3)]]
+    f = orc.forward(x, wg, wi, wo, u, C=GOLDEN["C"])
+    g = GOLDEN["default_reading"]
+    assert f.expert_idx[0].tolist() == GOLDEN["expert_idx"]
+    assert f.slot[0].tolist() == g["slot"]
+    w_exp = [[_fr(a), _fr(b)] for a, b in GOLDEN["weight_fractions"]]
     np.testing.assert_allclose(f.weight[0], np.array(w_exp, dtype=np.float64), rtol=1e-6)
     # flags: bit0 first kept, bit1 random test passed, bit2 second kept
-    assert f.flags[0].tolist() == [1 | 2 | 4, 1, 2, 1 | 2, 1]
-    assert f.first_count[0].tolist() == [3, 1, 1]
-    assert f.total_count[0].tolist() == [3, 4, 3]
-    np.testing.assert_allclose(f.m[0], [0.42, 0.28, 0.30], rtol=1e-6)
-    assert f.l_aux == pytest.approx(46 / 375, rel=1e-6)
-    assert f.l_aux_group[0] == pytest.approx(46 / 375, rel=1e-6)
+    assert f.flags[0].tolist() == g["flags"]
+    assert f.first_count[0].tolist() == GOLDEN["first_count"]
+    assert f.total_count[0].tolist() == g["total_count"]
+    np.testing.assert_allclose(f.m[0], [_fr(v) for v in GOLDEN["mean_gates_fractions"]], rtol=1e-6)
+    assert f.l_aux == pytest.approx(_fr(GOLDEN["l_aux_fraction"]), rel=1e-6)
+    assert f.l_aux_group[0] == pytest.approx(_fr(GOLDEN["l_aux_fraction"]), rel=1e-6)
     # slot_token [E,G,C]: e0 <- s0,s1 ; e1 <- s3,s0 ; e2 <- s4,empty
-    assert f.slot_token[:, 0, :].tolist() == [[0, 1], [3, 0], [4, -1]]
-    y3 = [float(Fr(4, 3)), float(Fr(10, 9)), 0.0, 5.0, 10.0]
-    np.testing.assert_allclose(f.y[0, :, 3], y3, rtol=1e-6)
+    assert f.slot_token[:, 0, :].tolist() == g["slot_token"]
+    np.testing.assert_allclose(f.y[0, :, 3], [_fr(v) for v in g["y_tag_component_fractions"]], rtol=1e-6)
     assert np.all(f.y[0, :, :3] == 0.0)
 
 
 def test_worked_example_other_reading():
     x, wg, wi, wo, u = _example_inputs()
-    f = orc.forward(x, wg, wi, wo, u, C=2, variant_a=True)
-    assert f.slot[0].tolist() == [[0, 1], [1, -1], [-1, -1], [0, 1], [0, -1]]
-    assert f.total_count[0].tolist() == [3, 3, 2]
-    assert f.first_count[0].tolist() == [3, 1, 1]
-    np.testing.assert_allclose(f.y[0, :, 3], [4 / 3, 10 / 9, 0.0, 9.5, 10.0], rtol=1e-6)
-    assert f.l_aux == pytest.approx(46 / 375, rel=1e-6)
+    f = orc.forward(x, wg, wi, wo, u, C=GOLDEN["C"], variant_a=True)
+    g = GOLDEN["other_reading"]
+    assert f.slot[0].tolist() == g["slot"]
+    assert f.total_count[0].tolist() == g["total_count"]
+    assert f.first_count[0].tolist() == GOLDEN["first_count"]
+    np.testing.assert_allclose(f.y[0, :, 3], [_fr(v) for v in g["y_tag_component_fractions"]], rtol=1e-6)
+    assert f.l_aux == pytest.approx(_fr(GOLDEN["l_aux_fraction"]), rel=1e-6)
 
 
 def test_tie_lowest_index_wins():
