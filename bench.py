@@ -316,8 +316,11 @@ def main():
         layer_flops = 3 * 2.0 * cfg.N * cfg.M * cfg.E + 2.0 * cfg.N * cfg.M * cfg.E + 3 * ffn_flops
         layer_bytes = 2 * layer_bytes + 2 * cfg.E * cfg.M * cfg.H * es + 2 * cfg.N * cfg.M * es
     t_roof = max(layer_flops / (peaks["bf16_tflops"] * 1e12), layer_bytes / (peaks["hbm_gbs"] * 1e9))
+    # the same with the tensor peak a seconds-long cuBLAS loop sustains under the power cap
+    t_roof_s = max(layer_flops / (peaks["bf16_tflops_sustained"] * 1e12), layer_bytes / (peaks["hbm_gbs"] * 1e9))
     layer = {"t_roof_ms": t_roof * 1e3, "frac": t_roof * 1e3 / ms_per_step, "flops": layer_flops,
-             "bytes": layer_bytes, "peak_source": peaks["source"]}
+             "bytes": layer_bytes, "peak_source": peaks["source"],
+             "frac_at_sustained_tensor_peak": t_roof_s * 1e3 / ms_per_step}
 
     # ---- end to end through the host-buffer entry point -------------------------------------
     e2e = None

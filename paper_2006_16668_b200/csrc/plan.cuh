@@ -2,6 +2,7 @@
 // 256-byte aligned; the status word is the first word of the workspace.
 #pragma once
 #include "common.cuh"
+#include "kernels.cuh"
 
 namespace gshard {
 

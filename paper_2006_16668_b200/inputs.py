@@ -72,6 +72,8 @@ CONFIGS = {
     "p4_routing": MoEConfig("p4_routing", G=32, S=4096, M=1024, H=64, E=2048, C=4, seed=20200637),
     # a 16-expert slice of the MoE(128E) layer (1024 rows per expert, tensor-bound expert GEMMs)
     "p2_slice": MoEConfig("p2_slice", G=16, S=512, M=1024, H=8192, E=16, C=64, seed=20200638),
+    # a 32-expert slice of the MoE(512E) training step (256 rows per expert; 1.1 GB of expert weights)
+    "p5_slice": MoEConfig("p5_slice", G=16, S=256, M=1024, H=8192, E=32, C=16, seed=20200639, backward=True),
     # configs[4]: training step
     "c5_512e_train": MoEConfig("c5_512e_train", G=16, S=4096, M=1024, H=8192, E=512, C=16,
                                seed=20200635, backward=True),
