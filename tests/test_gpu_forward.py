@@ -172,7 +172,7 @@ def test_expert_ffn_timing_hook():
         B._check(B.load().gshard_moe_time_expert_ffn(a.cuda_event, None), "one-sided event pair")
 
 
-FULL = [("c2_128e", [0, 9], 6), ("c3_512e_skew", [3, 15], 6), ("c4_2048e", [0, 17, 31], 5)]
+FULL = [("c2_128e", [0, 9], 10), ("c3_512e_skew", [3, 15], 10), ("c4_2048e", [0, 17, 31], 10)]
 
 
 @pytest.mark.parametrize("name,groups,tokens", FULL, ids=[c[0] for c in FULL])
@@ -197,3 +197,7 @@ def test_full_size_sampled(name, groups, tokens):
     assert not bool(y[dropped].any())
     if cfg.skew:
         assert int(rt["stats"][0]) > 0.1 * cfg.N       # experts 0..7 overflow by construction
+    # bit-reproducible at full size (no atomics, fixed reduction orders, fixed hand-over order)
+    y2, l_aux2, rt2 = run_forward(cfg, inp)
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16)) and torch.equal(l_aux, l_aux2)
+    assert torch.equal(rt["slot"], rt2["slot"]) and torch.equal(rt["m"], rt2["m"])
