@@ -131,6 +131,29 @@ int gshard_moe_top2_forward_host(const gshard_moe_shape* shape, const void* x_ho
                                  const gshard_moe_routing* routing_out, void* workspace,
                                  size_t workspace_bytes, void* cuda_stream);
 
+/* Pipelined form of the host-buffer forward for callers that stream batches: nothing is
+ * synchronised, the three phases of a step go to three streams so that the host-to-device copy of
+ * the next batch, the layer of the current one and the device-to-host copy of the previous one
+ * overlap (eq. (1)-(3) / Algorithm 1-2 as in gshard_moe_top2_forward).
+ *   staging: device buffer of gshard_moe_top2_host_staging_bytes(shape) bytes holding this SLOT's
+ *   copies of x, u, y, l_aux; use two or more slots (staging buffers with their own three events)
+ *   in rotation.  workspace: gshard_moe_top2_workspace_bytes(shape, 0) bytes, shared by all slots
+ *   (forwards are serialised on compute_stream).  ev_in / ev_done / ev_out: the slot's
+ *   cudaEvent_t handles (as void*), created by the caller; the call waits on them where the slot's
+ *   previous use must have finished and re-records them, so the same three events are passed every
+ *   time the slot is used.  Host buffers must be pinned and stay untouched until ev_out (or
+ *   copy_out_stream) has completed; routing_out, if given, must be per slot.  Not for
+ *   SAVE_FOR_BACKWARD shapes.  Device-side status: gshard_moe_last_device_status(workspace,
+ *   compute_stream). */
+int gshard_moe_top2_forward_host_async(const gshard_moe_shape* shape, const void* x_host,
+                                       const void* wg, const void* wi, const void* wo,
+                                       const float* u_host, void* y_host, float* l_aux_host,
+                                       const gshard_moe_routing* routing_out, void* workspace,
+                                       size_t workspace_bytes, void* staging, size_t staging_bytes,
+                                       void* copy_in_stream, void* compute_stream,
+                                       void* copy_out_stream, void* ev_in, void* ev_done,
+                                       void* ev_out);
+
 /* Backward of L = <dy, y> + l_aux_weight * l_aux with the routing of the forward call held
  * constant (the paper leaves the backward to automatic differentiation and states that the
  * counts c_e are not differentiable; section 2.2, auxiliary-loss paragraph).

@@ -54,6 +54,9 @@ EXPORTS = {
                                 [POINTER(gshard_moe_routing), c_void_p, c_void_p, c_size_t, c_void_p]),
     "gshard_moe_top2_forward_host": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 7 +
                                      [POINTER(gshard_moe_routing), c_void_p, c_size_t, c_void_p]),
+    "gshard_moe_top2_forward_host_async": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 7 +
+                                           [POINTER(gshard_moe_routing), c_void_p, c_size_t, c_void_p, c_size_t] +
+                                           [c_void_p] * 6),
     "gshard_moe_top2_backward": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6 + [c_float] +
                                  [c_void_p] * 5 + [c_size_t, c_void_p]),
     "gshard_moe_gate": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6 + [c_size_t, c_void_p]),
@@ -190,6 +193,19 @@ def gshard_moe_top2_forward_host(shape, x_host, wg, wi, wo, u_host, y_host, l_au
                                                _p(u_host), _p(y_host), _p(l_aux_host), rp, _p(workspace),
                                                workspace.numel(), _stream(stream)),
            "gshard_moe_top2_forward_host")
+
+
+def gshard_moe_top2_forward_host_async(shape, x_host, wg, wi, wo, u_host, y_host, l_aux_host, routing_out,
+                                       workspace, staging, copy_in_stream, compute_stream, copy_out_stream,
+                                       ev_in, ev_done, ev_out):
+    """Pipelined host-buffer forward: streams are torch.cuda.Stream, events torch.cuda.Event that
+    have been recorded once (so that their handles exist).  Nothing is synchronised."""
+    rp = ctypes.byref(routing_out) if routing_out is not None else None
+    _check(load().gshard_moe_top2_forward_host_async(
+        ctypes.byref(shape), _p(x_host), _p(wg), _p(wi), _p(wo), _p(u_host), _p(y_host), _p(l_aux_host), rp,
+        _p(workspace), workspace.numel(), _p(staging), staging.numel(), copy_in_stream.cuda_stream,
+        compute_stream.cuda_stream, copy_out_stream.cuda_stream, ev_in.cuda_event, ev_done.cuda_event,
+        ev_out.cuda_event), "gshard_moe_top2_forward_host_async")
 
 
 def gshard_moe_top2_backward(shape, x, wg, wi, wo, context, dy, l_aux_weight, dx, dwg, dwi, dwo,

@@ -265,6 +265,52 @@ int gshard_moe_top2_forward_host(const gshard_moe_shape* shape, const void* x_ho
   return status;
 }
 
+int gshard_moe_top2_forward_host_async(const gshard_moe_shape* shape, const void* x_host, const void* wg,
+                                       const void* wi, const void* wo, const float* u_host, void* y_host,
+                                       float* l_aux_host, const gshard_moe_routing* routing_out, void* workspace,
+                                       size_t workspace_bytes, void* staging, size_t staging_bytes,
+                                       void* copy_in_stream, void* compute_stream, void* copy_out_stream,
+                                       void* ev_in, void* ev_done, void* ev_out) {
+  launch_counter().n = 0;
+  GS_TRY(validate_shape(shape));
+  if (!x_host || !u_host || !y_host || !l_aux_host || !ev_in || !ev_done || !ev_out) return GSHARD_ERR_INVALID_ARG;
+  GS_REQUIRE_PTR(wg); GS_REQUIRE_PTR(wi); GS_REQUIRE_PTR(wo); GS_REQUIRE_PTR(workspace); GS_REQUIRE_PTR(staging);
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign || reinterpret_cast<uintptr_t>(staging) % kAlign)
+    return GSHARD_ERR_INVALID_ARG;
+  if (shape->flags & GSHARD_FLAG_SAVE_FOR_BACKWARD) return GSHARD_ERR_INVALID_ARG;
+  const Dims d = make_dims(*shape);
+  const size_t fwd = plan_forward(d).total;
+  const StagePlan sp = plan_staging(d);
+  if (workspace_bytes < fwd || staging_bytes < sp.total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  GS_TRY(check_device());
+  cudaStream_t s_in = static_cast<cudaStream_t>(copy_in_stream);
+  cudaStream_t s_cmp = static_cast<cudaStream_t>(compute_stream);
+  cudaStream_t s_out = static_cast<cudaStream_t>(copy_out_stream);
+  cudaEvent_t e_in = static_cast<cudaEvent_t>(ev_in), e_done = static_cast<cudaEvent_t>(ev_done),
+              e_out = static_cast<cudaEvent_t>(ev_out);
+  unsigned char* stg = static_cast<unsigned char*>(staging);
+  void* xd = stg + sp.x; float* ud = reinterpret_cast<float*>(stg + sp.u);
+  void* yd = stg + sp.y; float* ld = reinterpret_cast<float*>(stg + sp.l_aux);
+  const size_t act_bytes = (size_t)d.N * d.M * d.esize;
+#define GS_CUDA(call) do { if ((call) != cudaSuccess) return GSHARD_ERR_CUDA; } while (0)
+  // inputs of this slot may be overwritten once the previous forward that used the slot has run
+  GS_CUDA(cudaStreamWaitEvent(s_in, e_done, 0));
+  GS_CUDA(cudaMemcpyAsync(xd, x_host, act_bytes, cudaMemcpyHostToDevice, s_in));
+  GS_CUDA(cudaMemcpyAsync(ud, u_host, (size_t)d.N * 4, cudaMemcpyHostToDevice, s_in));
+  GS_CUDA(cudaEventRecord(e_in, s_in));
+  // the forward needs this slot's inputs, and its previous outputs must have left the device
+  GS_CUDA(cudaStreamWaitEvent(s_cmp, e_in, 0));
+  GS_CUDA(cudaStreamWaitEvent(s_cmp, e_out, 0));
+  GS_TRY(forward_device(shape, xd, wg, wi, wo, ud, yd, ld, routing_out, nullptr, workspace, fwd, s_cmp));
+  GS_CUDA(cudaEventRecord(e_done, s_cmp));
+  GS_CUDA(cudaStreamWaitEvent(s_out, e_done, 0));
+  GS_CUDA(cudaMemcpyAsync(y_host, yd, act_bytes, cudaMemcpyDeviceToHost, s_out));
+  GS_CUDA(cudaMemcpyAsync(l_aux_host, ld, 4, cudaMemcpyDeviceToHost, s_out));
+  GS_CUDA(cudaEventRecord(e_out, s_out));
+#undef GS_CUDA
+  return GSHARD_OK;
+}
+
 int gshard_moe_top2_backward(const gshard_moe_shape* shape, const void* x, const void* wg, const void* wi,
                              const void* wo, const void* context, const void* dy, float l_aux_weight, void* dx,
                              float* dwg, void* dwi, void* dwo, void* workspace, size_t workspace_bytes,
