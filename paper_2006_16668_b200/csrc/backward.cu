@@ -194,6 +194,19 @@ __global__ void __launch_bounds__(256) dx_kernel(const float4* __restrict__ dxg,
   }
 }
 
+// out[i] = part[0][i] + part[1][i] + ... (fixed order), float4 elements.
+__global__ void __launch_bounds__(256) sum_partials_kernel(const float4* __restrict__ part, float4* __restrict__ out,
+                                                           long long n4, int splits) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n4) return;
+  float4 acc = part[i];
+  for (int s = 1; s < splits; ++s) {
+    const float4 v = part[(long long)s * n4 + i];
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+  }
+  out[i] = acc;
+}
+
 int grid_rows(long long rows) {
   long long blocks = (rows + 7) / 8;
   const long long cap = 148LL * 32;
@@ -281,8 +294,31 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   g = UmmaGemm{};
   g.A = x; g.B = dlogits; g.C = dwg; g.rows = d.M; g.cols = d.E; g.K = (int)d.N; g.batch = 1;
   g.a_kmajor = false; g.b_kmajor = false; g.a_ld = d.M; g.b_ld = d.E; g.c_ld = d.E; g.out_f32 = 1;
+  // Few output tiles, very long contraction: split the token dimension over the batch index so that
+  // every SM gets a share, then add the partial sums in a fixed order.  The partials live in the dxg
+  // region, which is not written before the next GEMM.
+  int splits = 1;
+  if (!d.simt) {
+    const long long tiles = (long long)ceil_div(d.M, 128) * ceil_div(d.E, d.E > 128 ? 256 : 128);
+    for (int sp = (int)(148 / tiles); sp > 1; --sp)
+      if (d.N % ((long long)sp * 64) == 0 && (long long)sp * d.E <= d.N && ((long long)d.M * d.E) % 4 == 0) {
+        splits = sp;
+        break;
+      }
+  }
+  if (splits > 1) {
+    const long long kn = d.N / splits;
+    g.C = dxg; g.K = (int)kn; g.batch = splits;
+    g.a_bs = kn * d.M; g.b_bs = kn * d.E; g.c_bs = (long long)d.M * d.E;
+  }
   rc = run_gemm(d, g, status, st);
   if (rc) return rc;
+  if (splits > 1) {
+    const long long n4 = (long long)d.M * d.E / 4;
+    sum_partials_kernel<<<(int)((n4 + 255) / 256), 256, 0, st>>>(reinterpret_cast<const float4*>(dxg),
+                                                                 reinterpret_cast<float4*>(dwg), n4, splits);
+    count_launch();
+  }
   // dxg = dlogits . wg^T   [N x M] fp32
   g = UmmaGemm{};
   g.A = dlogits; g.B = wg; g.C = dxg; g.rows = (int)d.N; g.cols = d.M; g.K = d.E; g.batch = 1;

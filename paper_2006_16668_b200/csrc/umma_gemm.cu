@@ -137,6 +137,37 @@ __device__ __forceinline__ void process_chunk(const uint32_t* r, const Params& p
   }
 }
 
+// One epilogue warp's share of a finished 128 x BN accumulator: lane quarter q, column half `half`.
+template <int BN>
+__device__ __forceinline__ void epilogue_tile(const Params& p, const TileCoord& t, uint32_t tmem_acc, int q, int half,
+                                              unsigned char* stg, int lane) {
+  constexpr int kHalfCols = BN / 2;
+  unsigned char* srow = stg + lane * kStgRowBytes;
+  const int row0 = t.mt * BM + q * 32;
+  const bool row_ok = row0 + lane < p.rows;
+  const long long row_off = (long long)t.b * p.c_bs + (long long)(row0 + lane) * p.c_ld;
+  const uint32_t t_acc = tmem_acc + (uint32_t)(half * kHalfCols) + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+  for (int c = 0; c < kHalfCols / 64; ++c) {     // 64 columns per round: two TMEM loads in flight
+    const int col0 = t.nt * BN + half * kHalfCols + c * 64;
+    if (col0 >= p.cols) break;                   // uniform over the warp
+    uint32_t r0[32], r1[32];
+    ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r0);
+    ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r1);
+    ptx::tmem_ld_wait();
+    if (p.out_f32) {                             // 32 fp32 columns = one 128-byte staging row
+      process_chunk(r0, p, srow, lane, 0, row_ok, row_off, col0);
+      flush_rows(stg, p, t.b, row0, col0, lane);
+      process_chunk(r1, p, srow, lane, 0, row_ok, row_off, col0 + 32);
+      flush_rows(stg, p, t.b, row0, col0 + 32, lane);
+    } else {                                     // 64 bf16 columns = one 128-byte staging row
+      process_chunk(r0, p, srow, lane, 0, row_ok, row_off, col0);
+      process_chunk(r1, p, srow, lane, 4, row_ok, row_off, col0 + 32);
+      flush_rows(stg, p, t.b, row0, col0, lane);
+    }
+  }
+}
+
 template <bool A_K, bool B_K, int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -239,37 +270,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int ew = warp - 2;
     const int q = warp & 3;                          // TMEM lane quarter this warp may access
     const int half = ew >> 2;                        // which half of the tile's columns
-    constexpr int kHalfCols = BN / 2;
     unsigned char* stg = smem + C_::stg_off + ew * kStgWarpBytes;
-    unsigned char* srow = stg + lane * kStgRowBytes;
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
       const TileCoord t = decode(p, tile);
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      const int row0 = t.mt * BM + q * 32;
-      const bool row_ok = row0 + lane < p.rows;
-      const long long row_off = (long long)t.b * p.c_bs + (long long)(row0 + lane) * p.c_ld;
-      const uint32_t t_acc = tmem_base + (uint32_t)(acc * BN + half * kHalfCols) + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
-      for (int c = 0; c < kHalfCols / 64; ++c) {     // 64 columns per round: two TMEM loads in flight
-        const int col0 = t.nt * BN + half * kHalfCols + c * 64;
-        if (col0 >= p.cols) break;                   // uniform over the warp
-        uint32_t r0[32], r1[32];
-        ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r0);
-        ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r1);
-        ptx::tmem_ld_wait();
-        if (p.out_f32) {                             // 32 fp32 columns = one 128-byte staging row
-          process_chunk(r0, p, srow, lane, 0, row_ok, row_off, col0);
-          flush_rows(stg, p, t.b, row0, col0, lane);
-          process_chunk(r1, p, srow, lane, 0, row_ok, row_off, col0 + 32);
-          flush_rows(stg, p, t.b, row0, col0 + 32, lane);
-        } else {                                     // 64 bf16 columns = one 128-byte staging row
-          process_chunk(r0, p, srow, lane, 0, row_ok, row_off, col0);
-          process_chunk(r1, p, srow, lane, 4, row_ok, row_off, col0 + 32);
-          flush_rows(stg, p, t.b, row0, col0, lane);
-        }
-      }
+      epilogue_tile<BN>(p, t, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
@@ -292,6 +299,166 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc(tmem_base, C_::tmem_cols);
+  }
+}
+
+
+// ---- short-contraction variant: B tile resident in shared memory -------------------------------
+//
+// For C[b] = A[b]^T-like products with both operands MN-major and a contraction of at most 256 (the
+// expert weight gradients dwo = h^T.dout and dwi = buf^T.dh, contraction = rows per expert) a
+// 128 x 256 tile needs only 16 MMAs but 192 KB of operands, so the general kernel is bound by the
+// L2 -> shared-memory feed.  Here a CTA takes a whole column block of one problem (fixed batch and
+// 256-column tile) and walks its row tiles: the 256-column slice of B (up to 256 x 256, 128 KB) is
+// loaded once and stays, only the 64 KB A tile changes, which cuts the operand feed to a third.
+// Each of B's four k-blocks has its own full/empty barrier pair, so that the next column block's B
+// arrives k-block by k-block behind the last row tile's MMAs.
+namespace resb {
+constexpr int BN = 256;
+constexpr int kMaxKBlocks = 4;
+constexpr int kBBlockBytes = BN * BK * 2;                        // 32 KB per k-block
+constexpr int kAStages = 4;
+constexpr int a_off = kMaxKBlocks * kBBlockBytes;                // 128 KB
+constexpr int bar_off = a_off + kAStages * kABytes;              // + 64 KB
+constexpr int stg_off = bar_off + 256;
+constexpr int smem_bytes = stg_off + kEpiWarps * kStgWarpBytes + 1024;
+constexpr int tmem_cols = 2 * BN;
+}  // namespace resb
+
+__global__ void __launch_bounds__(kThreads, 1)
+umma_gemm_resident_b_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                            const Params p) {
+  using namespace resb;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + bar_off);
+  uint64_t* full = bars;                         // [kAStages]   A k-block landed
+  uint64_t* empty = full + kAStages;             // [kAStages]   A k-block consumed
+  uint64_t* b_full = empty + kAStages;           // [kMaxKBlocks] B k-block landed
+  uint64_t* b_empty = b_full + kMaxKBlocks;      // [kMaxKBlocks] B k-block no longer needed by this column block
+  uint64_t* acc_full = b_empty + kMaxKBlocks;    // [2]
+  uint64_t* acc_empty = acc_full + 2;            // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_groups = p.n_tiles * p.batch;      // column blocks
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kAStages; ++s) { ptx::mbar_init(full + s, 1); ptx::mbar_init(empty + s, 1); }
+    for (int s = 0; s < kMaxKBlocks; ++s) { ptx::mbar_init(b_full + s, 1); ptx::mbar_init(b_empty + s, 1); }
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(acc_full + a, 1); ptx::mbar_init(acc_empty + a, kEpiWarps); }
+    *abort_flag = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&map_a);
+    ptx::prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, tmem_cols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  bool ok = true;
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (lane == 0) {
+      const uint64_t pol_a = p.a_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
+      const uint64_t pol_b = p.b_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
+      int stage = 0; uint32_t phase = 0, b_phase = 0;
+      for (int grp = blockIdx.x; grp < n_groups && ok; grp += gridDim.x, b_phase ^= 1u) {
+        const int nt = grp % p.n_tiles, b = grp / p.n_tiles;
+        for (int mt = 0; mt < p.m_tiles && ok; ++mt) {
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            if (mt == 0) {
+              if (!ptx::mbar_wait(b_empty + kb, b_phase ^ 1u, abort_flag)) { ok = false; break; }
+              unsigned char* sb = smem + kb * kBBlockBytes;
+              ptx::mbar_arrive_expect_tx(b_full + kb, (uint32_t)kBBlockBytes);
+#pragma unroll
+              for (int j = 0; j < BN / 64; ++j)
+                ptx::tma_load_3d(sb + j * kBoxBytes, &map_b, b_full + kb, nt * BN + j * 64, kb * BK, b, pol_b);
+            }
+            if (!ptx::mbar_wait(empty + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+            unsigned char* sa = smem + a_off + stage * kABytes;
+            ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)kABytes);
+#pragma unroll
+            for (int j = 0; j < BM / 64; ++j)
+              ptx::tma_load_3d(sa + j * kBoxBytes, &map_a, full + stage, mt * BM + j * 64, kb * BK, b, pol_a);
+            if (++stage == kAStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer --------------------------------------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_bf16(BM, BN, true, true);
+      int stage = 0; uint32_t phase = 0, b_phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      for (int grp = blockIdx.x; grp < n_groups && ok; grp += gridDim.x, b_phase ^= 1u) {
+        for (int mt = 0; mt < p.m_tiles && ok; ++mt) {
+          if (!ptx::mbar_wait(acc_empty + acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after_sync();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+          for (int kb = 0; kb < p.k_blocks; ++kb) {
+            if (mt == 0 && !ptx::mbar_wait(b_full + kb, b_phase, abort_flag)) { ok = false; break; }
+            if (!ptx::mbar_wait(full + stage, phase, abort_flag)) { ok = false; break; }
+            ptx::tc_fence_after_sync();
+            const uint32_t sa = ptx::smem_u32(smem + a_off + stage * kABytes);
+            const uint32_t sb = ptx::smem_u32(smem + kb * kBBlockBytes);
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k) {
+              const uint64_t da = ptx::make_smem_desc(sa + k * 2048, kBoxBytes, 1024);
+              const uint64_t db = ptx::make_smem_desc(sb + k * 2048, kBoxBytes, 1024);
+              ptx::umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            ptx::umma_commit(empty + stage);
+            if (mt == p.m_tiles - 1) ptx::umma_commit(b_empty + kb);   // last use of this B k-block
+            if (++stage == kAStages) { stage = 0; phase ^= 1u; }
+          }
+          if (!ok) break;
+          ptx::umma_commit(acc_full + acc);
+          if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue ----------------------------------------------
+    const int ew = warp - 2;
+    const int q = warp & 3;
+    const int half = ew >> 2;
+    unsigned char* stg = smem + stg_off + ew * kStgWarpBytes;
+    int acc = 0; uint32_t acc_phase = 0;
+    for (int grp = blockIdx.x; grp < n_groups && ok; grp += gridDim.x) {
+      TileCoord t;
+      t.nt = grp % p.n_tiles; t.b = grp / p.n_tiles;
+      for (t.mt = 0; t.mt < p.m_tiles; ++t.mt) {
+        if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
+        ptx::tc_fence_after_sync();
+        epilogue_tile<BN>(p, t, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane);
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  }
+
+  if (!ok) {
+    *abort_flag = 1;
+    set_device_status(p.status, GSHARD_ERR_TIMEOUT);
+    const uint64_t t0 = ptx::globaltimer_ns();
+    while (ptx::globaltimer_ns() - t0 < 2000000ull) { __nanosleep(1000); }
+  }
+  __syncwarp();
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, tmem_cols);
   }
 }
 
@@ -332,6 +499,16 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   int sms = 148;
   int dev = 0;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  if (!g.a_kmajor && !g.b_kmajor && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
+    // short contraction, several row tiles per column block: keep the B tile resident
+    const int n_groups = p.n_tiles * g.batch;
+    if (cudaFuncSetAttribute(umma_gemm_resident_b_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             resb::smem_bytes) != cudaSuccess)
+      return GSHARD_ERR_CUDA;
+    umma_gemm_resident_b_kernel<<<n_groups < sms ? n_groups : sms, kThreads, resb::smem_bytes, st>>>(ma, mb, p);
+    count_launch();
+    return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+  }
   const int grid = p.total_tiles < sms ? p.total_tiles : sms;
 #define GSHARD_DISPATCH(AK, BKM) \
   (BN == 256 ? launch_t<AK, BKM, 256>(ma, mb, p, grid, st) : launch_t<AK, BKM, 128>(ma, mb, p, grid, st))

@@ -57,6 +57,11 @@ BWD_CASES = [
     ("bf16_umma_variant_a", 2, 256, 128, 256, 16, 20, "bf16", B.GSHARD_FLAG_SECOND_SKIP_FREES_SLOT, GRAD_TOL),
     # every grouped GEMM with more than 128 rows on CTA pairs (all four operand-layout variants)
     ("bf16_two_sm", 2, 384, 256, 512, 16, 80, "bf16", B.GSHARD_FLAG_TWO_SM_MMA, GRAD_TOL),
+    # weight-gradient GEMMs on the resident-B kernel (contraction = rows per expert <= 256, at least
+    # four row tiles): a ragged contraction (80 = 64 + 16) with a ragged last column block, and the
+    # full four k-blocks
+    ("bf16_wgrad_resident_ragged", 2, 256, 512, 640, 16, 40, "bf16", 0, GRAD_TOL),
+    ("bf16_wgrad_resident_k256", 2, 1024, 512, 512, 16, 128, "bf16", 0, GRAD_TOL),
 ]
 
 
