@@ -87,35 +87,54 @@ __device__ __forceinline__ void flush_rows(const unsigned char* stg, const Param
   __syncwarp();
 }
 
+// Coalesced load of a warp's 32 x 64 block of the bf16 mask (128 bytes per row): lane l takes piece
+// (l & 7) of rows 4*i + (l >> 3), the pattern of flush_rows.  Pieces outside the matrix read as zero.
+__device__ __forceinline__ void load_mask_block(const Params& p, int b, int row0, int col0, int lane, uint4* m) {
+  const int piece = lane & 7;
+  const int col = col0 + piece * 8;
+  const unsigned char* base = reinterpret_cast<const unsigned char*>(p.mask) + ((long long)b * p.c_bs + col) * 2;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int row = row0 + 4 * i + (lane >> 3);
+    m[i] = (row < p.rows && col < p.cols) ? __ldg(reinterpret_cast<const uint4*>(base + (long long)row * p.c_ld * 2))
+                                          : make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+
+__device__ __forceinline__ void stage_mask_block(unsigned char* stg, int lane, const uint4* m) {
+  const int piece = lane & 7;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = 4 * i + (lane >> 3);
+    *reinterpret_cast<uint4*>(stg + r * kStgRowBytes + ((piece ^ (r & 7)) * 16)) = m[i];
+  }
+  __syncwarp();
+}
+
 // ReLU / mask on one 32-column chunk of this thread's row, then into the staging row (XOR-swizzled
 // 16-byte pieces: conflict-free for the row-wise writes here and the piece-wise reads of the flush).
+template <bool MASK>
 __device__ __forceinline__ void process_chunk(const uint32_t* r, const Params& p, unsigned char* srow, int lane,
-                                              int piece0, bool row_ok, long long row_off, int col0) {
+                                              int piece0) {
   float v[32];
 #pragma unroll
   for (int i = 0; i < 32; ++i) {
     v[i] = __uint_as_float(r[i]);
     if (p.relu) v[i] = fmaxf(v[i], 0.f);
   }
-  if (p.mask && row_ok) {
-    const __nv_bfloat16* mk = reinterpret_cast<const __nv_bfloat16*>(p.mask) + row_off + col0;
-    if (col0 + 32 <= p.cols) {
+  if (MASK) {
+    // the mask block was staged into this row's pieces (same swizzle as the output written below)
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint4 mv = __ldg(reinterpret_cast<const uint4*>(mk) + i);
-        const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
+    for (int i = 0; i < 4; ++i) {
+      const uint4 mv = *reinterpret_cast<const uint4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16));
+      const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          // bf16 > 0  <=>  sign bit clear and magnitude bits non-zero
-          const uint32_t lo = w[j] & 0xffffu, hi = w[j] >> 16;
-          if (!(lo != 0u && lo < 0x8000u)) v[8 * i + 2 * j] = 0.f;
-          if (!(hi != 0u && hi < 0x8000u)) v[8 * i + 2 * j + 1] = 0.f;
-        }
+      for (int j = 0; j < 4; ++j) {
+        // bf16 > 0  <=>  sign bit clear and magnitude bits non-zero
+        const uint32_t lo = w[j] & 0xffffu, hi = w[j] >> 16;
+        if (!(lo != 0u && lo < 0x8000u)) v[8 * i + 2 * j] = 0.f;
+        if (!(hi != 0u && hi < 0x8000u)) v[8 * i + 2 * j + 1] = 0.f;
       }
-    } else {
-#pragma unroll
-      for (int i = 0; i < 32; ++i)
-        if (col0 + i < p.cols && !(__bfloat162float(mk[i]) > 0.f)) v[i] = 0.f;
     }
   }
   if (p.out_f32) {
@@ -137,38 +156,49 @@ __device__ __forceinline__ void process_chunk(const uint32_t* r, const Params& p
   }
 }
 
-// One epilogue warp's share of a finished 128 x BN accumulator: lane quarter q, column half `half`.
+// First column of round c of this warp's half of the tile.
 template <int BN>
+__device__ __forceinline__ int round_col0(const TileCoord& t, int half, int c) {
+  return t.nt * BN + half * (BN / 2) + c * 64;
+}
+
+// One epilogue warp's share of a finished 128 x BN accumulator: lane quarter q, column half `half`.
+// With a mask (bf16 output only) `mreg` holds the mask block of round 0, loaded by the caller
+// before it waited for the accumulator; the block of round c + 1 is fetched while round c is
+// processed, so the mask's global-memory latency stays off the accumulator's critical path.
+template <int BN, bool MASK>
 __device__ __forceinline__ void epilogue_tile(const Params& p, const TileCoord& t, uint32_t tmem_acc, int q, int half,
-                                              unsigned char* stg, int lane) {
+                                              unsigned char* stg, int lane, uint4* mreg) {
   constexpr int kHalfCols = BN / 2;
   unsigned char* srow = stg + lane * kStgRowBytes;
   const int row0 = t.mt * BM + q * 32;
-  const bool row_ok = row0 + lane < p.rows;
-  const long long row_off = (long long)t.b * p.c_bs + (long long)(row0 + lane) * p.c_ld;
   const uint32_t t_acc = tmem_acc + (uint32_t)(half * kHalfCols) + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
   for (int c = 0; c < kHalfCols / 64; ++c) {     // 64 columns per round: two TMEM loads in flight
-    const int col0 = t.nt * BN + half * kHalfCols + c * 64;
+    const int col0 = round_col0<BN>(t, half, c);
     if (col0 >= p.cols) break;                   // uniform over the warp
     uint32_t r0[32], r1[32];
     ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r0);
     ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r1);
+    if (MASK) {
+      stage_mask_block(stg, lane, mreg);
+      if (c + 1 < kHalfCols / 64) load_mask_block(p, t.b, row0, col0 + 64, lane, mreg);
+    }
     ptx::tmem_ld_wait();
     if (p.out_f32) {                             // 32 fp32 columns = one 128-byte staging row
-      process_chunk(r0, p, srow, lane, 0, row_ok, row_off, col0);
+      process_chunk<MASK>(r0, p, srow, lane, 0);
       flush_rows(stg, p, t.b, row0, col0, lane);
-      process_chunk(r1, p, srow, lane, 0, row_ok, row_off, col0 + 32);
+      process_chunk<MASK>(r1, p, srow, lane, 0);
       flush_rows(stg, p, t.b, row0, col0 + 32, lane);
     } else {                                     // 64 bf16 columns = one 128-byte staging row
-      process_chunk(r0, p, srow, lane, 0, row_ok, row_off, col0);
-      process_chunk(r1, p, srow, lane, 4, row_ok, row_off, col0 + 32);
+      process_chunk<MASK>(r0, p, srow, lane, 0);
+      process_chunk<MASK>(r1, p, srow, lane, 4);
       flush_rows(stg, p, t.b, row0, col0, lane);
     }
   }
 }
 
-template <bool A_K, bool B_K, int BN>
+template <bool A_K, bool B_K, int BN, bool MASK>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const Params p) {
@@ -274,9 +304,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
       const TileCoord t = decode(p, tile);
+      uint4 mreg[MASK ? 8 : 1];
+      if (MASK) load_mask_block(p, t.b, t.mt * BM + q * 32, round_col0<BN>(t, half, 0), lane, mreg);
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      epilogue_tile<BN>(p, t, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane);
+      epilogue_tile<BN, MASK>(p, t, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, mreg);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
@@ -438,7 +470,7 @@ umma_gemm_resident_b_kernel(const __grid_constant__ CUtensorMap map_a, const __g
       for (t.mt = 0; t.mt < p.m_tiles; ++t.mt) {
         if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
         ptx::tc_fence_after_sync();
-        epilogue_tile<BN>(p, t, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane);
+        epilogue_tile<BN, false>(p, t, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, nullptr);
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
@@ -464,9 +496,9 @@ umma_gemm_resident_b_kernel(const __grid_constant__ CUtensorMap map_a, const __g
 
 // ---- host side ------------------------------------------------------------------------------
 
-template <bool A_K, bool B_K, int BN>
+template <bool A_K, bool B_K, int BN, bool MASK>
 int launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int grid, cudaStream_t st) {
-  auto kern = umma_gemm_kernel<A_K, B_K, BN>;
+  auto kern = umma_gemm_kernel<A_K, B_K, BN, MASK>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::smem_bytes) != cudaSuccess)
     return GSHARD_ERR_CUDA;
   kern<<<grid, kThreads, Cfg<BN>::smem_bytes, st>>>(ma, mb, p);
@@ -478,6 +510,7 @@ int launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int 
 
 int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (g.rows <= 0 || g.cols <= 0 || g.K <= 0 || g.batch <= 0) return GSHARD_OK;
+  if (g.mask && g.out_f32) return GSHARD_ERR_INTERNAL;   // the mask is staged as bf16 rows
   const int BN = g.cols > 128 ? 256 : 128;
   CUtensorMap ma, mb;
   bool okm;
@@ -499,7 +532,7 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   int sms = 148;
   int dev = 0;
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  if (!g.a_kmajor && !g.b_kmajor && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
+  if (!g.a_kmajor && !g.b_kmajor && !g.mask && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
     // short contraction, several row tiles per column block: keep the B tile resident
     const int n_groups = p.n_tiles * g.batch;
     if (cudaFuncSetAttribute(umma_gemm_resident_b_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -510,8 +543,11 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
     return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
   }
   const int grid = p.total_tiles < sms ? p.total_tiles : sms;
-#define GSHARD_DISPATCH(AK, BKM) \
-  (BN == 256 ? launch_t<AK, BKM, 256>(ma, mb, p, grid, st) : launch_t<AK, BKM, 128>(ma, mb, p, grid, st))
+#define GSHARD_DISPATCH(AK, BKM)                                                                    \
+  (p.mask ? (BN == 256 ? launch_t<AK, BKM, 256, true>(ma, mb, p, grid, st)                          \
+                       : launch_t<AK, BKM, 128, true>(ma, mb, p, grid, st))                         \
+          : (BN == 256 ? launch_t<AK, BKM, 256, false>(ma, mb, p, grid, st)                         \
+                       : launch_t<AK, BKM, 128, false>(ma, mb, p, grid, st)))
   if (g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH(true, true);
   if (g.a_kmajor && !g.b_kmajor) return GSHARD_DISPATCH(true, false);
   if (!g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH(false, true);
