@@ -190,6 +190,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--gather-dispatch", action="store_true",
+                    help="single-launch FFN gathers its rows from x (no dispatch buffer)")
     ap.add_argument("--fused-ffn", action="store_true", help="ablation: force the single-launch expert FFN")
     ap.add_argument("--unfused-ffn", action="store_true", help="ablation: force the two grouped-GEMM launches")
     ap.add_argument("--two-sm-mma", action="store_true", help="ablation: grouped GEMMs on CTA pairs (cta_group::2)")
@@ -221,7 +223,8 @@ def main():
     inp = make_inputs(rcfg, dev)
     shape = B.make_shape(cfg, flags=(B.GSHARD_FLAG_FUSED_FFN if args.fused_ffn else 0) |
                          (B.GSHARD_FLAG_UNFUSED_FFN if args.unfused_ffn else 0) |
-                         (B.GSHARD_FLAG_TWO_SM_MMA if args.two_sm_mma else 0))
+                         (B.GSHARD_FLAG_TWO_SM_MMA if args.two_sm_mma else 0) |
+                         (B.GSHARD_FLAG_GATHER_DISPATCH if args.gather_dispatch else 0))
     ws = B.alloc_workspace(shape, host_staging=True, device=dev)
     y = torch.empty_like(inp["x"])
     l_aux = torch.zeros(1, dtype=torch.float32, device=dev)

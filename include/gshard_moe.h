@@ -66,6 +66,11 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
 #define GSHARD_FLAG_TWO_SM_MMA 32u         /* grouped GEMMs with more than 128 rows per problem run on
                                               CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles) instead
                                               of single CTAs (128 x 256 tiles) */
+#define GSHARD_FLAG_GATHER_DISPATCH 64u    /* forward with the single-launch expert FFN: the token rows
+                                              of an expert are gathered straight from x by the slot
+                                              index list (TMA row gather) while GEMM-1 runs, and the
+                                              [E, G*C, M] dispatch buffer of Algorithm 2 is not
+                                              written; ignored where that FFN form is not in use */
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

@@ -71,16 +71,21 @@ int gate_stage(const Dims& d, const FwdPlan& pl, unsigned char* ws, const void* 
 }
 
 // h = relu(buf . wi), out = h . wo for every expert (eq. (2)); weights are read once.
+bool ffn_runs_fused(const Dims& d, bool keep_h) {
+  const bool want_fused = d.fused_ffn || (!d.unfused_ffn && d.rows <= 128);
+  return !d.simt && want_fused && !keep_h && ffn_fused_supported(d);
+}
+
+// With x / slot_token (only where ffn_runs_fused) the rows are gathered from x and buf is not read.
 int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
-              void* fused_scratch, int* status, cudaStream_t st) {
+              void* fused_scratch, int* status, cudaStream_t st, const void* x = nullptr,
+              const int32_t* slot_token = nullptr) {
   const long long rows = d.rows;
   // One persistent launch in which the hidden activations never leave L2: the faster form when
   // the FFN is bound by streaming the expert weights (at most one 128-row tile per expert); with
   // more rows per expert the two grouped-GEMM launches keep the tensor pipe busier.  Not available
   // when the caller keeps h for the backward pass.
-  const bool want_fused = d.fused_ffn || (!d.unfused_ffn && d.rows <= 128);
-  if (!d.simt && want_fused && !keep_h && ffn_fused_supported(d))
-    return launch_ffn_fused(d, buf, wi, wo, fused_scratch, out, status, st);
+  if (ffn_runs_fused(d, keep_h)) return launch_ffn_fused(d, buf, wi, wo, fused_scratch, out, status, st, x, slot_token);
   UmmaGemm g{};
   g.A = buf; g.B = wi; g.C = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;
   g.a_kmajor = true; g.b_kmajor = false;
@@ -105,7 +110,7 @@ int validate_shape(const gshard_moe_shape* s) {
   if (!s) return GSHARD_ERR_INVALID_ARG;
   if (s->G <= 0 || s->S <= 0 || s->M <= 0 || s->H <= 0 || s->E <= 0 || s->C <= 0) return GSHARD_ERR_INVALID_ARG;
   if (s->dtype != GSHARD_F32 && s->dtype != GSHARD_BF16) return GSHARD_ERR_INVALID_ARG;
-  if (s->flags & ~63u) return GSHARD_ERR_INVALID_ARG;
+  if (s->flags & ~127u) return GSHARD_ERR_INVALID_ARG;
   if ((s->flags & GSHARD_FLAG_FUSED_FFN) && (s->flags & GSHARD_FLAG_UNFUSED_FFN)) return GSHARD_ERR_INVALID_ARG;
   if (s->E < 2) return GSHARD_ERR_INVALID_ARG;
   if (s->M % 8 || s->H % 8) return GSHARD_ERR_UNSUPPORTED_SHAPE;
@@ -155,12 +160,13 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
   GS_TRY(gate_stage(d, pl, ws, x, wg, expert_idx, gate12, m, rowmax, rowinv, st));
   GS_TRY(launch_capacity(d, expert_idx, gate12, u, m, slot, weight, flags, first_count, total_count, slot_token,
                          l_aux_group, stats_group, l_aux, reinterpret_cast<long long*>(r.stats), st));
-  launch_dispatch(d, x, slot_token, buf, st);
+  const bool gather = d.gather_dispatch && ffn_runs_fused(d, save);
+  if (!gather) launch_dispatch(d, x, slot_token, buf, st);
   // optional event pair around the expert FFN, armed for one call by gshard_moe_time_expert_ffn
   FfnTiming& ft = ffn_timing();
   const bool timed = ft.start != nullptr && ft.stop != nullptr;
   if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.start), st) != cudaSuccess) return GSHARD_ERR_CUDA;
-  GS_TRY(ffn_stage(d, buf, wi, wo, h, save, out, ws + pl.ffn_scratch, status, st));
+  GS_TRY(ffn_stage(d, buf, wi, wo, h, save, out, ws + pl.ffn_scratch, status, st, gather ? x : nullptr, slot_token));
   if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.stop), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   ft.start = ft.stop = nullptr;
   launch_combine(d, out, expert_idx, slot, weight, y, st);

@@ -22,6 +22,15 @@
 //                    complete in issue order, so its G2(T+2) completed, which needed the round
 //                    T+2 chunks of every rank r'; r' stored that chunk after its own G1(T+2)
 //                    completed, and r' issued G2(T) before G1(T+2): r' is done reading round T.
+//   row gather       optional (Algorithm 2's dispatch fused into this launch): a seventh warp of
+//                    every rank copies a quarter of the NEXT units' token rows from x, through
+//                    the slot index list, into a per-group, two-unit-deep A-slot in the scratch
+//                    (zeros for empty slots) and counts the unit in gath[group][rank] (release);
+//                    the gather warp then acquires all four counters and arrives on a local
+//                    mbarrier that the CTA's producer waits on before a unit's first A load.  The
+//                    slot of unit i is overwritten for unit i + 2 only after prod[] shows that all
+//                    four ranks finished every GEMM-1 of unit i.  The [E, G*C, M] dispatch buffer
+//                    is then neither written nor read.
 // All CTAs are co-resident (grid <= SM count, one CTA per SM) and every wait is bounded in wall
 // time, reporting GSHARD_ERR_TIMEOUT through the status word instead of hanging.
 #include <cuda.h>
@@ -39,7 +48,9 @@ constexpr int KC = 256;                       // hidden columns per chunk
 constexpr int kGroup = 4;                     // CTAs per unit
 constexpr int kRing = 4;                      // scratch ring depth in rounds
 constexpr int kEpiWarps = 4;
-constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kThreads = 64 + 32 * kEpiWarps + 32;   // + the row-gather warp
+constexpr int kGatherWarp = 2 + kEpiWarps;
+constexpr int kASlots = 2;                    // gathered units in flight per group
 constexpr int kABytes = BM * BK * 2;          // 16 KB
 constexpr int kBoxBytes = 64 * 64 * 2;        // 8 KB
 constexpr int kStageBytes = kABytes + 4 * kBoxBytes;   // 48 KB: A + up to 256 B-columns
@@ -59,6 +70,13 @@ struct GroupParams {
   int units, groups;
   int* prod;                // [groups][kGroup] finished epilogue warps per rank
   int* status;
+  // row-gather mode (x != nullptr): A rows of unit (e, mt) come from x[G*S, M] through
+  // slot_token[E][G*C] into a_slots[groups][kASlots][128][M]
+  const uint4* x;
+  const int32_t* slot_token;
+  uint4* a_slots;
+  int* gath;                // [groups][kGroup] units gathered by each rank
+  int S, C;
 };
 
 __device__ __forceinline__ int ld_acquire(const int* p) {
@@ -128,7 +146,8 @@ ffn_group4_kernel(const __grid_constant__ CUtensorMap map_buf, const __grid_cons
   uint64_t* g1_empty = g1_full + 1;         // [1]
   uint64_t* out_full = g1_empty + 1;        // [1]
   uint64_t* out_empty = out_full + 1;       // [1]
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(out_empty + 1);
+  uint64_t* a_ready = out_empty + 1;        // [kASlots] gathered rows of a unit complete on all ranks
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(a_ready + kASlots);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -143,6 +162,7 @@ ffn_group4_kernel(const __grid_constant__ CUtensorMap map_buf, const __grid_cons
     ptx::mbar_init(g1_empty, kEpiWarps);
     ptx::mbar_init(out_full, 1);
     ptx::mbar_init(out_empty, kEpiWarps);
+    for (int a = 0; a < kASlots; ++a) ptx::mbar_init(a_ready + a, 1);
     *abort_flag = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&map_buf); ptx::prefetch_tensormap(&map_wi);
@@ -170,12 +190,19 @@ ffn_group4_kernel(const __grid_constant__ CUtensorMap map_buf, const __grid_cons
           const int u = group + (T / p.rounds) * p.groups, t = T % p.rounds;
           const int e = u / p.m_tiles, mt = u % p.m_tiles;
           const int hcol = (t * kGroup + rank) * KC;
+          const int ui = T / p.rounds;
+          if (p.x && t == 0) {                             // this unit's gathered rows are complete
+            if (!ptx::mbar_wait(a_ready + (ui % kASlots), (uint32_t)(ui / kASlots) & 1u, abort_flag)) { ok = false; break; }
+            asm volatile("fence.proxy.async;" ::: "memory");
+          }
+          const int a_row = p.x ? 0 : mt * BM;
+          const int a_idx = p.x ? group * kASlots + (ui % kASlots) : e;
           for (int kb = 0; kb < p.k1_blocks; ++kb) {
             if (!ptx::mbar_wait(empty + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
             unsigned char* sa = smem + stage * kStageBytes;
             unsigned char* sb = sa + kABytes;
             ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)(kABytes + (KC / 64) * kBoxBytes));
-            ptx::tma_load_3d(sa, &map_buf, full + stage, kb * BK, mt * BM, e, pol_a);
+            ptx::tma_load_3d(sa, &map_buf, full + stage, kb * BK, a_row, a_idx, pol_a);
 #pragma unroll
             for (int j = 0; j < KC / 64; ++j)
               ptx::tma_load_3d(sb + j * kBoxBytes, &map_wi, full + stage, hcol + j * 64, kb * BK, e, pol_w);
@@ -259,6 +286,70 @@ ffn_group4_kernel(const __grid_constant__ CUtensorMap map_buf, const __grid_cons
           if (!ok) break;
           if (t == p.rounds - 1) ptx::umma_commit(out_full);
         }
+      }
+    }
+  } else if (warp == kGatherWarp) {
+    // ------------------------------ row gather --------------------------------------------
+    if (p.x) {
+      const int row_vec = p.M / 8;                           // 16-byte pieces per row
+      const uint64_t pol_keep = ptx::policy_evict_last();    // the slots are re-read 32 times from L2
+      constexpr int kRowsPerRank = BM / kGroup;
+      for (int ui = 0; ui < my_units && ok; ++ui) {
+        const int u = group + ui * p.groups;
+        const int e = u / p.m_tiles, mt = u % p.m_tiles;
+        if (ui >= kASlots) {
+          // the slot's previous unit: every rank has finished all of its GEMM-1 rounds
+          const int target = (ui - kASlots + 1) * p.rounds * kEpiWarps;
+          int w = 1;
+          if (lane < kGroup) w = wait_counter(p.prod + group * kGroup + lane, target, abort_flag) ? 1 : 0;
+          if (__any_sync(0xffffffffu, w == 0)) { ok = false; break; }
+        }
+        uint4* dst = p.a_slots + ((size_t)(group * kASlots + (ui % kASlots)) * BM + rank * kRowsPerRank) * row_vec;
+#pragma unroll 1
+        for (int r0 = 0; r0 < kRowsPerRank; r0 += 4) {
+          const uint4* src[4];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const int row = mt * BM + rank * kRowsPerRank + r0 + i;
+            src[i] = nullptr;
+            if (row < p.rows) {
+              const int s_tok = __ldg(p.slot_token + (long long)e * p.rows + row);
+              if (s_tok >= 0) src[i] = p.x + ((long long)(row / p.C) * p.S + s_tok) * row_vec;
+            }
+          }
+          for (int v0 = 0; v0 < row_vec; v0 += 32 * 4) {
+            uint4 val[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int v = v0 + j * 32 + lane;
+                val[i][j] = (src[i] && v < row_vec) ? __ldg(src[i] + v) : make_uint4(0u, 0u, 0u, 0u);
+              }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int v = v0 + j * 32 + lane;
+                if (v < row_vec)
+                  asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(
+                                   dst + (size_t)(r0 + i) * row_vec + v),
+                               "r"(val[i][j].x), "r"(val[i][j].y), "r"(val[i][j].z), "r"(val[i][j].w), "l"(pol_keep)
+                               : "memory");
+              }
+          }
+        }
+        __threadfence();                                     // rows visible GPU-wide ...
+        asm volatile("fence.proxy.async;" ::: "memory");     // ... and to the async proxy (TMA)
+        __syncwarp();
+        if (lane == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(p.gath + group * kGroup + rank) : "memory");
+        // all four quarters of the unit are in place: tell this CTA's producer through shared
+        // memory, so that its only wait at the start of a unit is a local one
+        int w = 1;
+        if (lane < kGroup) w = wait_counter(p.gath + group * kGroup + lane, ui + 1, abort_flag) ? 1 : 0;
+        if (__any_sync(0xffffffffu, w == 0)) { ok = false; break; }
+        asm volatile("fence.proxy.async;" ::: "memory");
+        if (lane == 0) ptx::mbar_arrive(a_ready + (ui % kASlots));
       }
     }
   } else {
@@ -355,13 +446,13 @@ bool ffn_fused_supported(const Dims& d) {
 
 // Scratch bytes: the per-group chunk ring plus the hand-over counters.
 size_t ffn_fused_scratch_bytes(const Dims& d) {
-  (void)d;
   const size_t groups = 256 / kGroup;            // enough for any SM count up to 256
-  return groups * kRing * kGroup * BM * KC * 2 + 256 + groups * kGroup * sizeof(int);
+  return groups * kRing * kGroup * BM * KC * 2 + 256 + groups * 2 * kGroup * sizeof(int) + 256 +
+         groups * kASlots * BM * (size_t)d.M * 2;
 }
 
 int launch_ffn_fused(const Dims& d, const void* buf, const void* wi, const void* wo, void* scratch, void* out,
-                     int* status, cudaStream_t st) {
+                     int* status, cudaStream_t st, const void* x_gather, const int32_t* slot_token) {
   GroupParams p;
   const int sms = device_sms();
   p.groups = sms / kGroup;
@@ -377,11 +468,17 @@ int launch_ffn_fused(const Dims& d, const void* buf, const void* wi, const void*
   p.scratch = static_cast<__nv_bfloat16*>(scratch);
   p.prod = reinterpret_cast<int*>(static_cast<unsigned char*>(scratch) + ring_bytes + 256);
   p.out = static_cast<__nv_bfloat16*>(out);
+  p.gath = p.prod + (256 / kGroup) * kGroup;
+  p.a_slots = reinterpret_cast<uint4*>(static_cast<unsigned char*>(scratch) + ring_bytes + 256 +
+                                       (size_t)(256 / kGroup) * 2 * kGroup * sizeof(int) + 256);
+  p.x = static_cast<const uint4*>(x_gather);
+  p.slot_token = slot_token; p.S = d.S; p.C = d.C;
   p.status = status;
-  if (cudaMemsetAsync(p.prod, 0, sizeof(int) * (256 / kGroup) * kGroup, st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  if (cudaMemsetAsync(p.prod, 0, sizeof(int) * (256 / kGroup) * 2 * kGroup, st) != cudaSuccess) return GSHARD_ERR_CUDA;
   CUtensorMap m_buf, m_wi, m_hs, m_wo;
   const long long rows = d.rows;
-  bool okm = make_map(&m_buf, buf, d.M, rows, d.E, d.M, rows * d.M, BK, BM);
+  bool okm = x_gather ? make_map(&m_buf, p.a_slots, d.M, BM, (long long)p.groups * kASlots, d.M, (long long)BM * d.M, BK, BM)
+                      : make_map(&m_buf, buf, d.M, rows, d.E, d.M, rows * d.M, BK, BM);
   okm = okm && make_map(&m_wi, wi, d.H, d.M, d.E, d.H, (long long)d.M * d.H, 64, BK);
   okm = okm && make_map(&m_hs, scratch, KC, BM, (long long)p.groups * kRing * kGroup, KC, (long long)BM * KC, BK, BM);
   okm = okm && make_map(&m_wo, wo, d.M, d.H, d.E, d.M, (long long)d.H * d.M, 64, BK);

@@ -48,7 +48,10 @@ int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st);
 // chunks of the hidden activations through a small L2-resident scratch ring.
 bool ffn_fused_supported(const Dims& d);
 size_t ffn_fused_scratch_bytes(const Dims& d);
+// With x_gather / slot_token the rows of GEMM-1's A operand are gathered from x[G*S, M] by index
+// (TMA tile::gather4) and `buf` is not read.
 int launch_ffn_fused(const Dims& d, const void* buf, const void* wi, const void* wo, void* scratch, void* out,
-                     int* status, cudaStream_t st);
+                     int* status, cudaStream_t st, const void* x_gather = nullptr,
+                     const int32_t* slot_token = nullptr);
 
 }  // namespace gshard

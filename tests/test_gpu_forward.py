@@ -118,6 +118,11 @@ SMALL = [
     # <= 128 rows per expert and H a multiple of 1024: the single-launch FFN is chosen by default
     ("bf16_fused_ffn_auto", 2, 256, 256, 1024, 32, 16, "bf16", 0),
     ("bf16_unfused_forced", 2, 256, 256, 1024, 32, 16, "bf16", B.GSHARD_FLAG_UNFUSED_FFN),
+    # the FFN gathers its rows from x by index (no dispatch buffer): one ragged tile per expert, and
+    # two row tiles per expert (160 rows) with the single-launch form forced
+    ("bf16_gather_dispatch", 2, 256, 256, 1024, 32, 16, "bf16", B.GSHARD_FLAG_GATHER_DISPATCH),
+    ("bf16_gather_dispatch_two_tiles", 2, 1024, 256, 1024, 16, 80, "bf16",
+     B.GSHARD_FLAG_GATHER_DISPATCH | B.GSHARD_FLAG_FUSED_FFN),
 ]
 
 
@@ -145,6 +150,25 @@ def test_umma_matches_simt_contractions():
     assert rel_fro(to_np(y_t), to_np(y_s)) < 5e-3
     same = (rt_t["expert_idx"] == rt_s["expert_idx"]).all(dim=-1).float().mean().item()
     assert same > 0.999
+
+
+def test_gather_dispatch_matches_dispatch_buffer_bitwise():
+    # the same rows reach the same MMAs either way, so y must not differ in a single bit
+    cfg = MoEConfig("gd", G=4, S=512, M=512, H=2048, E=64, C=16, dtype="bf16", seed=79)
+    inp = make_inputs(cfg, "cuda")
+    y_b, l_b, rt_b = run_forward(cfg, inp, 0)
+    y_g, l_g, rt_g = run_forward(cfg, inp, B.GSHARD_FLAG_GATHER_DISPATCH)
+    assert torch.equal(y_b.view(torch.int16), y_g.view(torch.int16)) and torch.equal(l_b, l_g)
+    assert torch.equal(rt_b["slot_token"], rt_g["slot_token"])
+
+
+def test_gather_dispatch_full_size_bitwise():
+    # MoE(2048E) shape, 55 units per CTA group: the two-deep slot rotation and its reuse waits
+    cfg = CONFIGS["c4_2048e"]
+    inp = make_inputs(cfg, "cuda")
+    y_b, l_b, _ = run_forward(cfg, inp, 0)
+    y_g, l_g, _ = run_forward(cfg, inp, B.GSHARD_FLAG_GATHER_DISPATCH)
+    assert torch.equal(y_b.view(torch.int16), y_g.view(torch.int16)) and torch.equal(l_b, l_g)
 
 
 def test_expert_ffn_timing_hook():
