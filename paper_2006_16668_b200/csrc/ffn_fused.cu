@@ -85,15 +85,19 @@ __device__ __forceinline__ int ld_acquire(const int* p) {
   return v;
 }
 
+// `poll_ns`: pause between polls.  The hand-over waits on the critical path poll fast; the row-gather
+// warp, which waits for a whole unit to finish, polls slowly so that it does not load the counters'
+// L2 lines.
 __device__ __forceinline__ bool wait_counter(const int* ctr, int target, volatile int* abort_flag,
-                                             uint64_t limit_ns = 2000000000ull) {
+                                             uint32_t poll_ns = 32, uint64_t limit_ns = 2000000000ull) {
   if (ld_acquire(ctr) >= target) return true;
   const uint64_t t0 = ptx::globaltimer_ns();
   uint32_t it = 0;
+  const uint32_t check_mask = poll_ns >= 1000 ? 0u : 63u;
   while (true) {
     if (ld_acquire(ctr) >= target) return true;
-    __nanosleep(32);
-    if ((++it & 63u) == 0) {
+    __nanosleep(poll_ns);
+    if ((++it & check_mask) == 0) {
       if (*abort_flag) return false;
       if (ptx::globaltimer_ns() - t0 > limit_ns) return false;
     }
@@ -301,7 +305,7 @@ ffn_group4_kernel(const __grid_constant__ CUtensorMap map_buf, const __grid_cons
           // the slot's previous unit: every rank has finished all of its GEMM-1 rounds
           const int target = (ui - kASlots + 1) * p.rounds * kEpiWarps;
           int w = 1;
-          if (lane < kGroup) w = wait_counter(p.prod + group * kGroup + lane, target, abort_flag) ? 1 : 0;
+          if (lane < kGroup) w = wait_counter(p.prod + group * kGroup + lane, target, abort_flag, 2000) ? 1 : 0;
           if (__any_sync(0xffffffffu, w == 0)) { ok = false; break; }
         }
         uint4* dst = p.a_slots + ((size_t)(group * kASlots + (ui % kASlots)) * BM + rank * kRowsPerRank) * row_vec;
@@ -346,7 +350,7 @@ ffn_group4_kernel(const __grid_constant__ CUtensorMap map_buf, const __grid_cons
         // all four quarters of the unit are in place: tell this CTA's producer through shared
         // memory, so that its only wait at the start of a unit is a local one
         int w = 1;
-        if (lane < kGroup) w = wait_counter(p.gath + group * kGroup + lane, ui + 1, abort_flag) ? 1 : 0;
+        if (lane < kGroup) w = wait_counter(p.gath + group * kGroup + lane, ui + 1, abort_flag, 500) ? 1 : 0;
         if (__any_sync(0xffffffffu, w == 0)) { ok = false; break; }
         asm volatile("fence.proxy.async;" ::: "memory");
         if (lane == 0) ptx::mbar_arrive(a_ready + (ui % kASlots));
