@@ -83,6 +83,13 @@ class ClockSampler(threading.Thread):
         except Exception:
             pass
 
+    def wait_first_sample(self, timeout_s=5.0):
+        """nvidia-smi needs up to a second to print its first line: wait for it, so that short timed
+        regions are sampled too."""
+        t0 = time.time()
+        while not self.samples and time.time() - t0 < timeout_s and self.is_alive():
+            time.sleep(0.02)
+
     def stop(self):
         if self.proc is not None:
             self.proc.terminate()          # the exact process started above
@@ -190,6 +197,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--gate-cluster", action="store_true",
+                    help="ablation: cluster gating kernel with the mean-gate partial sums fused in")
     ap.add_argument("--gather-dispatch", action="store_true",
                     help="single-launch FFN gathers its rows from x (no dispatch buffer)")
     ap.add_argument("--fused-ffn", action="store_true", help="ablation: force the single-launch expert FFN")
@@ -224,7 +233,8 @@ def main():
     shape = B.make_shape(cfg, flags=(B.GSHARD_FLAG_FUSED_FFN if args.fused_ffn else 0) |
                          (B.GSHARD_FLAG_UNFUSED_FFN if args.unfused_ffn else 0) |
                          (B.GSHARD_FLAG_TWO_SM_MMA if args.two_sm_mma else 0) |
-                         (B.GSHARD_FLAG_GATHER_DISPATCH if args.gather_dispatch else 0))
+                         (B.GSHARD_FLAG_GATHER_DISPATCH if args.gather_dispatch else 0) |
+                         (B.GSHARD_FLAG_GATE_CLUSTER if args.gate_cluster else 0))
     ws = B.alloc_workspace(shape, host_staging=True, device=dev)
     y = torch.empty_like(inp["x"])
     l_aux = torch.zeros(1, dtype=torch.float32, device=dev)
@@ -268,6 +278,7 @@ def main():
 
     sampler = ClockSampler(local_rank)
     sampler.start()
+    sampler.wait_first_sample()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     # event pairs recorded by the library around the expert FFN of each timed step (the dominant
     # kernel); recorded once here so that their handles exist before they are handed over

@@ -71,6 +71,13 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                               index list (TMA row gather) while GEMM-1 runs, and the
                                               [E, G*C, M] dispatch buffer of Algorithm 2 is not
                                               written; ignored where that FFN form is not in use */
+#define GSHARD_FLAG_GATE_CLUSTER 128u      /* bf16 tensor-core gating with the mean gates' partial sums
+                                              fused in: a thread-block cluster holds all E logits of a
+                                              token tile in tensor memory and exchanges the softmax
+                                              statistics through distributed shared memory, so no
+                                              logits are stored (needs E <= 2048, S % 32 == 0; elsewhere
+                                              ignored).  Default: logits stored once, column sums in a
+                                              second pass - measured faster on B200 */
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

@@ -32,6 +32,7 @@ GSHARD_FLAG_FUSED_FFN = 8
 GSHARD_FLAG_UNFUSED_FFN = 16
 GSHARD_FLAG_TWO_SM_MMA = 32
 GSHARD_FLAG_GATHER_DISPATCH = 64
+GSHARD_FLAG_GATE_CLUSTER = 128
 
 
 class gshard_moe_shape(Structure):

@@ -64,6 +64,17 @@ int gate_stage(const Dims& d, const FwdPlan& pl, unsigned char* ws, const void* 
     GS_TRY(gate_logits(d, x, wg, logits, status, st));
     launch_gate_rows(d, logits, expert_idx, gate12, rowmax, rowinv, st);
   } else {
+    // on request: mean gates fused into the gating kernel (no stored logits) where a cluster covers
+    // all experts
+    if (d.gate_cluster && gate_cluster_supported(d)) {
+      float* partial32 = reinterpret_cast<float*>(ws + pl.partial);
+      const int rc = launch_gate_cluster(d, x, wg, expert_idx, gate12, rowmax, rowinv, partial32, status, st);
+      if (rc == GSHARD_OK) {
+        launch_gate_mean_blocks(d, partial32, d.S / 32, m, st);
+        return GSHARD_OK;
+      }
+      if (rc != GSHARD_ERR_UNSUPPORTED_SHAPE) return rc;
+    }
     GS_TRY(launch_gate_fused(d, x, wg, logits, expert_idx, gate12, rowmax, rowinv, status, st));
   }
   launch_gate_means(d, logits, rowmax, rowinv, reinterpret_cast<float*>(ws + pl.partial), m, st);
@@ -110,7 +121,7 @@ int validate_shape(const gshard_moe_shape* s) {
   if (!s) return GSHARD_ERR_INVALID_ARG;
   if (s->G <= 0 || s->S <= 0 || s->M <= 0 || s->H <= 0 || s->E <= 0 || s->C <= 0) return GSHARD_ERR_INVALID_ARG;
   if (s->dtype != GSHARD_F32 && s->dtype != GSHARD_BF16) return GSHARD_ERR_INVALID_ARG;
-  if (s->flags & ~127u) return GSHARD_ERR_INVALID_ARG;
+  if (s->flags & ~255u) return GSHARD_ERR_INVALID_ARG;
   if ((s->flags & GSHARD_FLAG_FUSED_FFN) && (s->flags & GSHARD_FLAG_UNFUSED_FFN)) return GSHARD_ERR_INVALID_ARG;
   if (s->E < 2) return GSHARD_ERR_INVALID_ARG;
   if (s->M % 8 || s->H % 8) return GSHARD_ERR_UNSUPPORTED_SHAPE;

@@ -44,6 +44,7 @@ struct Dims {
   bool fused_ffn;       // force the single-launch FFN (h handed over through L2)
   bool unfused_ffn;     // force the two grouped-GEMM launches (h through HBM)
   bool two_sm_mma;      // grouped GEMMs on CTA pairs (tcgen05 cta_group::2) where rows > 128
+  bool gate_cluster;    // gating on clusters with the mean-gate partial sums fused in (no stored logits)
   bool gather_dispatch; // single-launch FFN gathers its rows from x instead of reading a dispatch buffer
 };
 
@@ -62,6 +63,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.unfused_ffn = (s.flags & GSHARD_FLAG_UNFUSED_FFN) != 0;
   d.two_sm_mma = (s.flags & GSHARD_FLAG_TWO_SM_MMA) != 0;
   d.gather_dispatch = (s.flags & GSHARD_FLAG_GATHER_DISPATCH) != 0;
+  d.gate_cluster = (s.flags & GSHARD_FLAG_GATE_CLUSTER) != 0;
   return d;
 }
 

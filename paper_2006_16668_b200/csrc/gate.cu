@@ -174,4 +174,9 @@ void launch_gate_means(const Dims& d, const float* logits, const float* rowmax, 
   count_launch(2);
 }
 
+void launch_gate_mean_blocks(const Dims& d, const float* partial, int blocks_per_group, float* m, cudaStream_t st) {
+  gate_mean_kernel<<<dim3(ceil_div(d.E, 128), d.G), 128, 0, st>>>(partial, d.S, d.E, blocks_per_group, m);
+  count_launch();
+}
+
 }  // namespace gshard

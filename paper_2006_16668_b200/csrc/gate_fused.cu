@@ -63,6 +63,14 @@ __device__ __forceinline__ void top2_merge(float& v1, int& i1, float& v2, int& i
   i2 = second ? l_i : w_i;
 }
 
+// 2^x with the hardware approximation (relative error about 2^-22, far inside the tolerance of the
+// softmax sums; one instruction instead of the range-checked library sequence).
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __device__ __forceinline__ int tile_cols(const GateParams& p, int nt) {   // multiple of 16, <= BN
   const int left = p.E - nt * BN;
   const int c = left < BN ? left : BN;
@@ -206,10 +214,15 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
             if (nv <= 0) break;                          // uniform over the warp
             float v[32];
             float cm[4] = {ninf, ninf, ninf, ninf};
+            if (nv == 32) {                              // uniform over the warp
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              v[i] = i < nv ? __uint_as_float(r[hh][i]) : ninf;
-              cm[i & 3] = fmaxf(cm[i & 3], v[i]);
+              for (int i = 0; i < 32; ++i) { v[i] = __uint_as_float(r[hh][i]); cm[i & 3] = fmaxf(cm[i & 3], v[i]); }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) {
+                v[i] = i < nv ? __uint_as_float(r[hh][i]) : ninf;
+                cm[i & 3] = fmaxf(cm[i & 3], v[i]);
+              }
             }
             const float cmax = fmaxf(fmaxf(cm[0], cm[1]), fmaxf(cm[2], cm[3]));
             if (cmax > m) {
@@ -222,7 +235,7 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
               const int k = i & 3;
-              s4[k] += exp2f(fmaf(v[i], kLog2e, -ml));  // exp(v - m); 0 for the padded columns
+              s4[k] += ex2_approx(fmaf(v[i], kLog2e, -ml));  // exp(v - m); 0 for the padded columns
               const bool gt1 = v[i] > a1[k];
               const bool gt2 = v[i] > a2[k];
               a2[k] = gt1 ? a1[k] : (gt2 ? v[i] : a2[k]);

@@ -11,6 +11,13 @@ void launch_gate_means(const Dims& d, const float* logits, const float* rowmax, 
                        float* partial, float* m, cudaStream_t st);
 
 // gate_fused.cu: bf16 logits GEMM on tcgen05 with row statistics and top-2 in the epilogue.
+// gate_cluster.cu: gating with the mean gates' partial sums fused in (clusters, distributed shared
+// memory); partial32 holds one row of column sums per 32-token block.
+bool gate_cluster_supported(const Dims& d);
+int launch_gate_cluster(const Dims& d, const void* x, const void* wg, int32_t* expert_idx, float* gate12,
+                        float* rowmax, float* rowinv, float* partial32, int* status, cudaStream_t st);
+// gate.cu: m[g,e] = (1/S) * sum of the group's `blocks_per_group` partial rows, in order.
+void launch_gate_mean_blocks(const Dims& d, const float* partial, int blocks_per_group, float* m, cudaStream_t st);
 int launch_gate_fused(const Dims& d, const void* x, const void* wg, float* logits, int32_t* expert_idx,
                       float* gate12, float* rowmax, float* rowinv, int* status, cudaStream_t st);
 

@@ -1,6 +1,7 @@
 // Byte offsets of every region of the caller's workspace / context buffers.  All regions are
 // 256-byte aligned; the status word is the first word of the workspace.
 #pragma once
+#include <algorithm>
 #include "common.cuh"
 #include "kernels.cuh"
 
@@ -23,7 +24,9 @@ inline FwdPlan plan_forward(const Dims& d) {
   p.logits = c.take(N * d.E * 4);
   p.rowmax = c.take(N * 4);
   p.rowinv = c.take(N * 4);
-  p.partial = c.take((size_t)d.G * d.tiles_per_group * d.E * 4);
+  // column-sum partials: one row per 128-token tile (two-pass gating) or per 32-token block
+  // (cluster gating)
+  p.partial = c.take(std::max((size_t)d.G * d.tiles_per_group, (size_t)((d.N + 31) / 32)) * d.E * 4);
   p.gate12 = c.take(N * 2 * 4);
   p.m = c.take((size_t)d.G * d.E * 4);
   p.expert_idx = c.take(N * 2 * 4);

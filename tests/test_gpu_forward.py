@@ -120,6 +120,9 @@ SMALL = [
     ("bf16_unfused_forced", 2, 256, 256, 1024, 32, 16, "bf16", B.GSHARD_FLAG_UNFUSED_FFN),
     # the FFN gathers its rows from x by index (no dispatch buffer): one ragged tile per expert, and
     # two row tiles per expert (160 rows) with the single-launch form forced
+    # gating on clusters with the mean-gate partial sums fused in (no stored logits)
+    ("bf16_gate_cluster", 2, 256, 256, 1024, 32, 16, "bf16", B.GSHARD_FLAG_GATE_CLUSTER),
+    ("bf16_gate_cluster_3ctas", 2, 320, 128, 256, 640, 1, "bf16", B.GSHARD_FLAG_GATE_CLUSTER),
     ("bf16_gather_dispatch", 2, 256, 256, 1024, 32, 16, "bf16", B.GSHARD_FLAG_GATHER_DISPATCH),
     ("bf16_gather_dispatch_two_tiles", 2, 1024, 256, 1024, 16, 80, "bf16",
      B.GSHARD_FLAG_GATHER_DISPATCH | B.GSHARD_FLAG_FUSED_FFN),
@@ -169,6 +172,20 @@ def test_gather_dispatch_full_size_bitwise():
     y_b, l_b, _ = run_forward(cfg, inp, 0)
     y_g, l_g, _ = run_forward(cfg, inp, B.GSHARD_FLAG_GATHER_DISPATCH)
     assert torch.equal(y_b.view(torch.int16), y_g.view(torch.int16)) and torch.equal(l_b, l_g)
+
+
+def test_gate_cluster_full_size_against_default():
+    # MoE(2048E) shape: eight-CTA clusters, 69 token tiles per cluster; both gating forms must
+    # agree on the picks (up to near-ties) and on the mean gates
+    cfg = CONFIGS["c4_2048e"]
+    inp = make_inputs(cfg, "cuda")
+    y_a, l_a, rt_a = run_forward(cfg, inp, 0)
+    y_b, l_b, rt_b = run_forward(cfg, inp, B.GSHARD_FLAG_GATE_CLUSTER)
+    same = (rt_a["expert_idx"] == rt_b["expert_idx"]).all(dim=-1).float().mean().item()
+    assert same > 0.9995, same
+    torch.testing.assert_close(rt_a["m"], rt_b["m"], rtol=1e-5, atol=1e-9)
+    assert float(l_b) == pytest.approx(float(l_a), rel=1e-5)
+    assert rel_fro(to_np(y_b[:2]), to_np(y_a[:2])) < 1e-2
 
 
 def test_expert_ffn_timing_hook():

@@ -158,3 +158,52 @@ def test_expert_ffn_against_oracle(E, G, C, M, H, dtype, flags):
         assert np.all(np.isfinite(got))
         err = rel_fro(got, ref)
         assert err < (1e-5 if dtype == "f32" else 1e-2), (e, err)
+
+
+CL = B.GSHARD_FLAG_GATE_CLUSTER
+GATE_CASES = [
+    # G, S, M, E, flags    (cluster size of the fused gating kernel = ceil(E / 256))
+    (2, 64, 128, 16, CL),                             # one CTA, a single 16-expert column tile
+    (2, 96, 64, 128, CL),                             # one CTA; 96 tokens: ragged 128-token tile
+    (3, 160, 128, 272, CL),                           # two CTAs, the second with 16 experts
+    (2, 256, 1024, 512, CL),                          # two CTAs, full contraction depth
+    (1, 288, 128, 768, CL),                           # three CTAs: two row quarters finalised by CTA 0
+    (2, 128, 192, 1280, CL),                          # five CTAs
+    (5, 544, 128, 2048, CL),                          # eight CTAs, more row tiles than clusters can hold at once
+    (2, 100, 128, 512, CL),                           # S not a multiple of 32: the stored-logits form is chosen
+    (2, 256, 128, 2048, 0),                           # default: stored logits + column-sum pass
+    (3, 96, 1024, 272, 0),
+]
+
+
+@pytest.mark.parametrize("G,S,M,E,flags", GATE_CASES)
+def test_gate_stage_against_oracle(G, S, M, E, flags):
+    """Gating stage (softmax gates' top-2, raw gate values, mean gates m) against the fp64 oracle."""
+    rng = np.random.default_rng(G * 7 + S + E)
+    shape = _shape(G, S, M, 64, E, 2, "bf16", flags)
+    x = torch.from_numpy(rng.standard_normal((G, S, M)).astype(np.float32)).to(torch.bfloat16).cuda()
+    wg = torch.from_numpy((rng.standard_normal((M, E)) / np.sqrt(M)).astype(np.float32)).to(torch.bfloat16).cuda()
+    ei = torch.full((G, S, 2), -1, dtype=torch.int32, device="cuda")
+    g12 = torch.zeros(G, S, 2, device="cuda")
+    m = torch.zeros(G, E, device="cuda")
+    ws = B.alloc_workspace(shape)
+    B.gshard_moe_gate(shape, x, wg, ei, g12, m, ws)
+    assert B.gshard_moe_last_device_status(ws) == B.GSHARD_OK
+    wg_np = to_np(wg)
+    for g in range(G):
+        _, p = orc.gates(to_np(x[g]), wg_np)
+        e1, e2, g1, g2, g3 = orc.top2(p)
+        margin = np.where(g3 >= 0, np.minimum(g1 - g2, g2 - g3), g1 - g2)
+        ok = margin >= 1e-6
+        got = to_np(ei[g])
+        assert np.array_equal(got[ok, 0], e1[ok]) and np.array_equal(got[ok, 1], e2[ok])
+        idx = np.arange(S)
+        # raw gate values of the picks the GPU made (identical to the oracle's outside near-ties)
+        np.testing.assert_allclose(to_np(g12[g])[:, 0], p[idx, got[:, 0]], rtol=2e-5, atol=1e-9)
+        np.testing.assert_allclose(to_np(g12[g])[:, 1], p[idx, got[:, 1]], rtol=2e-5, atol=1e-9)
+        np.testing.assert_allclose(to_np(m[g]), orc.mean_gates(p), rtol=1e-5, atol=1e-9)
+    # bit-reproducible
+    ei2, g122, m2 = torch.empty_like(ei), torch.empty_like(g12), torch.empty_like(m)
+    B.gshard_moe_gate(shape, x, wg, ei2, g122, m2, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(ei, ei2) and torch.equal(g12, g122) and torch.equal(m, m2)
