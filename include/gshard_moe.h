@@ -63,9 +63,9 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                               it is used when an expert has at most 128 rows */
 #define GSHARD_FLAG_UNFUSED_FFN 16u        /* force the two grouped-GEMM launches instead (hidden
                                               activations make a round trip through HBM) */
-#define GSHARD_FLAG_TWO_SM_MMA 32u         /* grouped GEMMs with more than 128 rows per problem run on
-                                              CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles) instead
-                                              of single CTAs (128 x 256 tiles) */
+#define GSHARD_FLAG_TWO_SM_MMA 32u         /* every grouped GEMM with more than 128 rows per problem runs
+                                              on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles); by
+                                              default only the two forward expert GEMMs do */
 #define GSHARD_FLAG_GATHER_DISPATCH 64u    /* forward with the single-launch expert FFN: the token rows
                                               of an expert are gathered straight from x by the slot
                                               index list (TMA row gather) while GEMM-1 runs, and the
@@ -78,6 +78,11 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                               logits are stored (needs E <= 2048, S % 32 == 0; elsewhere
                                               ignored).  Default: logits stored once, column sums in a
                                               second pass - measured faster on B200 */
+#define GSHARD_FLAG_ONE_SM_MMA 512u        /* no grouped GEMM runs on CTA pairs (128 x 256 tiles on
+                                              single CTAs everywhere) */
+#define GSHARD_FLAG_GATE_TWO_SM 256u       /* the default gating kernel on CTA pairs (tcgen05
+                                              cta_group::2: each CTA loads half of the wg tile); needs
+                                              E % 128 == 0, elsewhere ignored */
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

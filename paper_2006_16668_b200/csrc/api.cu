@@ -75,7 +75,10 @@ int gate_stage(const Dims& d, const FwdPlan& pl, unsigned char* ws, const void* 
       }
       if (rc != GSHARD_ERR_UNSUPPORTED_SHAPE) return rc;
     }
-    GS_TRY(launch_gate_fused(d, x, wg, logits, expert_idx, gate12, rowmax, rowinv, status, st));
+    if (d.gate_two_sm && gate_fused2_supported(d))
+      GS_TRY(launch_gate_fused2(d, x, wg, logits, expert_idx, gate12, rowmax, rowinv, status, st));
+    else
+      GS_TRY(launch_gate_fused(d, x, wg, logits, expert_idx, gate12, rowmax, rowinv, status, st));
   }
   launch_gate_means(d, logits, rowmax, rowinv, reinterpret_cast<float*>(ws + pl.partial), m, st);
   return GSHARD_OK;
@@ -101,13 +104,13 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   g.A = buf; g.B = wi; g.C = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;
   g.a_kmajor = true; g.b_kmajor = false;
   g.a_ld = d.M; g.a_bs = rows * d.M; g.b_ld = d.H; g.b_bs = (long long)d.M * d.H; g.c_ld = d.H; g.c_bs = rows * d.H;
-  g.relu = 1; g.b_stream = 1;
+  g.relu = 1; g.b_stream = 1; g.prefer_two_sm = 1;
   GS_TRY(run_gemm(d, g, status, st));
   UmmaGemm g2{};
   g2.A = h; g2.B = wo; g2.C = out; g2.rows = d.rows; g2.cols = d.M; g2.K = d.H; g2.batch = d.E;
   g2.a_kmajor = true; g2.b_kmajor = false;
   g2.a_ld = d.H; g2.a_bs = rows * d.H; g2.b_ld = d.M; g2.b_bs = (long long)d.H * d.M; g2.c_ld = d.M; g2.c_bs = rows * d.M;
-  g2.b_stream = 1;
+  g2.b_stream = 1; g2.prefer_two_sm = 1;
   return run_gemm(d, g2, status, st);
 }
 
@@ -121,7 +124,7 @@ int validate_shape(const gshard_moe_shape* s) {
   if (!s) return GSHARD_ERR_INVALID_ARG;
   if (s->G <= 0 || s->S <= 0 || s->M <= 0 || s->H <= 0 || s->E <= 0 || s->C <= 0) return GSHARD_ERR_INVALID_ARG;
   if (s->dtype != GSHARD_F32 && s->dtype != GSHARD_BF16) return GSHARD_ERR_INVALID_ARG;
-  if (s->flags & ~255u) return GSHARD_ERR_INVALID_ARG;
+  if (s->flags & ~1023u) return GSHARD_ERR_INVALID_ARG;
   if ((s->flags & GSHARD_FLAG_FUSED_FFN) && (s->flags & GSHARD_FLAG_UNFUSED_FFN)) return GSHARD_ERR_INVALID_ARG;
   if (s->E < 2) return GSHARD_ERR_INVALID_ARG;
   if (s->M % 8 || s->H % 8) return GSHARD_ERR_UNSUPPORTED_SHAPE;

@@ -8,11 +8,13 @@ namespace gshard {
 // A and B hold the configuration dtype; C holds float when g.out_f32, else the dtype.
 inline int run_gemm(const Dims& d, const UmmaGemm& g, int* status, cudaStream_t st) {
   if (!d.simt) {
-    // CTA pairs with the two-SM MMA load a third fewer operand bytes per SM and run the tensor pipe
-    // about 10 % busier in isolation, but under the board's sustained power cap they measured no
-    // faster than single CTAs (slower on the 1024-rows-per-expert shape), so they are opt-in.  A
-    // single row tile would leave the second CTA of a pair without rows.
-    if (g.rows > 128 && d.two_sm_mma) return launch_umma2_gemm(g, status, st);
+    // CTA pairs with the two-SM MMA read only half of the B tile from their own shared memory per
+    // MMA and load a third fewer operand bytes per SM; the one-SM kernel's 128 x 256 tiles keep the
+    // shared memory busy with 96 B/clk of operand reads plus 96 B/clk of TMA writes, which is what
+    // holds its tensor pipe near 65 %.  Callers mark the GEMMs that measured faster on pairs (the two
+    // forward expert GEMMs); the flags force either form everywhere.  A single row tile would leave
+    // the second CTA of a pair without rows.
+    if (g.rows > 128 && !d.one_sm_mma && (d.two_sm_mma || g.prefer_two_sm)) return launch_umma2_gemm(g, status, st);
     return launch_umma_gemm(g, status, st);
   }
   SimtGemm s{};

@@ -18,6 +18,10 @@ int launch_gate_cluster(const Dims& d, const void* x, const void* wg, int32_t* e
                         float* rowmax, float* rowinv, float* partial32, int* status, cudaStream_t st);
 // gate.cu: m[g,e] = (1/S) * sum of the group's `blocks_per_group` partial rows, in order.
 void launch_gate_mean_blocks(const Dims& d, const float* partial, int blocks_per_group, float* m, cudaStream_t st);
+// gate_fused2.cu: the same gating kernel on CTA pairs (tcgen05 cta_group::2, half of the wg tile per CTA).
+bool gate_fused2_supported(const Dims& d);
+int launch_gate_fused2(const Dims& d, const void* x, const void* wg, float* logits, int32_t* expert_idx,
+                       float* gate12, float* rowmax, float* rowinv, int* status, cudaStream_t st);
 int launch_gate_fused(const Dims& d, const void* x, const void* wg, float* logits, int32_t* expert_idx,
                       float* gate12, float* rowmax, float* rowinv, int* status, cudaStream_t st);
 
@@ -46,6 +50,7 @@ struct UmmaGemm {
   int out_f32;               // C is float instead of bf16
   int relu;
   int a_stream, b_stream;    // operand is read once: load with an evict-first L2 hint
+  int prefer_two_sm;         // run on CTA pairs (cta_group::2) when a problem has more than 128 rows
 };
 int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st);
 // umma2_gemm.cu: the same contraction with the two-SM MMA (CTA pairs, 256 x 256 tiles).

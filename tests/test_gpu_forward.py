@@ -120,6 +120,9 @@ SMALL = [
     ("bf16_unfused_forced", 2, 256, 256, 1024, 32, 16, "bf16", B.GSHARD_FLAG_UNFUSED_FFN),
     # the FFN gathers its rows from x by index (no dispatch buffer): one ragged tile per expert, and
     # two row tiles per expert (160 rows) with the single-launch form forced
+    # 160 rows per expert: expert GEMMs on CTA pairs (default) and on single CTAs
+    ("bf16_two_sm_default", 2, 512, 256, 512, 16, 80, "bf16", 0),
+    ("bf16_one_sm_forced", 2, 512, 256, 512, 16, 80, "bf16", B.GSHARD_FLAG_ONE_SM_MMA),
     # gating on clusters with the mean-gate partial sums fused in (no stored logits)
     ("bf16_gate_cluster", 2, 256, 256, 1024, 32, 16, "bf16", B.GSHARD_FLAG_GATE_CLUSTER),
     ("bf16_gate_cluster_3ctas", 2, 320, 128, 256, 640, 1, "bf16", B.GSHARD_FLAG_GATE_CLUSTER),

@@ -122,6 +122,9 @@ FFN_CASES = [
     (2, 2, 100, 1024, 2048, "bf16", 0),          # 200 rows: ragged second row tile
     (3, 1, 24, 192, 448, "bf16", 0),             # fewer rows than a tile, ragged column tile
     (1, 4, 96, 512, 1024, "bf16", 0),            # 384 rows
+    # more than 128 rows run on CTA pairs by default: the same shapes on single CTAs
+    (2, 2, 100, 1024, 2048, "bf16", B.GSHARD_FLAG_ONE_SM_MMA),
+    (1, 4, 96, 512, 1024, "bf16", B.GSHARD_FLAG_ONE_SM_MMA),
     # the single-launch FFN (groups of four CTAs, h chunks handed over through an L2-resident ring)
     (40, 1, 128, 512, 2048, "bf16", B.GSHARD_FLAG_FUSED_FFN),
     (6, 2, 100, 256, 1024, "bf16", B.GSHARD_FLAG_FUSED_FFN),     # 200 rows: two row tiles per expert
@@ -161,6 +164,7 @@ def test_expert_ffn_against_oracle(E, G, C, M, H, dtype, flags):
 
 
 CL = B.GSHARD_FLAG_GATE_CLUSTER
+TS = B.GSHARD_FLAG_GATE_TWO_SM
 GATE_CASES = [
     # G, S, M, E, flags    (cluster size of the fused gating kernel = ceil(E / 256))
     (2, 64, 128, 16, CL),                             # one CTA, a single 16-expert column tile
@@ -173,6 +177,10 @@ GATE_CASES = [
     (2, 100, 128, 512, CL),                           # S not a multiple of 32: the stored-logits form is chosen
     (2, 256, 128, 2048, 0),                           # default: stored logits + column-sum pass
     (3, 96, 1024, 272, 0),
+    (2, 256, 128, 2048, TS),                          # CTA pairs, eight column tiles
+    (3, 160, 1024, 128, TS),                          # CTA pairs, one 128-expert tile; 480 tokens: odd number of row tiles... (4 tiles) 
+    (1, 352, 192, 384, TS),                           # three row tiles: the last pair has an idle CTA; ragged second column tile
+    (2, 100, 128, 272, TS),                           # E not a multiple of 128: the one-SM kernel is chosen
 ]
 
 
