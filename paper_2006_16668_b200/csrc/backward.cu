@@ -257,7 +257,7 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   g.A = dout; g.B = wo; g.C = dh; g.mask = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;
   g.a_kmajor = true; g.b_kmajor = true;
   g.a_ld = d.M; g.a_bs = rows * d.M; g.b_ld = d.M; g.b_bs = (long long)d.H * d.M; g.c_ld = d.H; g.c_bs = rows * d.H;
-  g.b_stream = 1;
+  g.b_stream = 1; g.prefer_two_sm = 1;
   int rc = run_gemm(d, g, status, st);
   if (rc) return rc;
   // dwo[e] = h[e]^T . dout[e]   [H x M]
@@ -279,7 +279,7 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   g.A = dh; g.B = wi; g.C = dbuf; g.rows = d.rows; g.cols = d.M; g.K = d.H; g.batch = d.E;
   g.a_kmajor = true; g.b_kmajor = true;
   g.a_ld = d.H; g.a_bs = rows * d.H; g.b_ld = d.H; g.b_bs = (long long)d.M * d.H; g.c_ld = d.M; g.c_bs = rows * d.M;
-  g.b_stream = 1;
+  g.b_stream = 1; g.prefer_two_sm = 1;
   rc = run_gemm(d, g, status, st);
   if (rc) return rc;
 

@@ -22,10 +22,13 @@
 #include "kernels.cuh"
 #include "sm100_ptx.cuh"
 #include "tensor_map.cuh"
+#include "umma_epilogue.cuh"
 
 namespace gshard {
 
 namespace {
+
+using namespace umma_epi;
 
 constexpr int BM = 128, BK = 64, BN = 256, BNH = BN / 2;
 constexpr int kEpiWarps = 8;
@@ -38,8 +41,6 @@ constexpr int kStages = 6;
 constexpr int kTmemCols = 2 * BN;
 constexpr int kBarOff = kStages * kStageBytes;
 constexpr int kStgOff = kBarOff + 256;
-constexpr int kStgRowBytes = 128;
-constexpr int kStgWarpBytes = 32 * kStgRowBytes;
 constexpr int kSmemBytes = kStgOff + kEpiWarps * kStgWarpBytes + 1024;
 
 struct Params2 {
@@ -53,8 +54,6 @@ struct Params2 {
   int n_fastest;
   int* status;
 };
-
-struct TileCoord { int mt, nt, b; };
 
 __device__ __forceinline__ TileCoord decode(const Params2& p, int tile) {
   TileCoord t;
@@ -125,73 +124,7 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
       : "memory");
 }
 
-__device__ __forceinline__ void flush_rows2(const unsigned char* stg, const Params2& p, int b, int row0, int col0,
-                                            int lane) {
-  __syncwarp();
-  const int esz = p.out_f32 ? 4 : 2;
-  const int piece = lane & 7;
-  const int col = col0 + piece * (16 / esz);
-  unsigned char* cbase = reinterpret_cast<unsigned char*>(p.C) + ((long long)b * p.c_bs + col) * esz;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int r = 4 * i + (lane >> 3);
-    const int row = row0 + r;
-    if (row < p.rows && col < p.cols) {
-      const uint4 val = *reinterpret_cast<const uint4*>(stg + r * kStgRowBytes + ((piece ^ (r & 7)) * 16));
-      *reinterpret_cast<uint4*>(cbase + (long long)row * p.c_ld * esz) = val;
-    }
-  }
-  __syncwarp();
-}
-
-__device__ __forceinline__ void process_chunk2(const uint32_t* r, const Params2& p, unsigned char* srow, int lane,
-                                               int piece0, bool row_ok, long long row_off, int col0) {
-  float v[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    v[i] = __uint_as_float(r[i]);
-    if (p.relu) v[i] = fmaxf(v[i], 0.f);
-  }
-  if (p.mask && row_ok) {
-    const __nv_bfloat16* mk = reinterpret_cast<const __nv_bfloat16*>(p.mask) + row_off + col0;
-    if (col0 + 32 <= p.cols) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint4 mv = __ldg(reinterpret_cast<const uint4*>(mk) + i);
-        const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const uint32_t lo = w[j] & 0xffffu, hi = w[j] >> 16;      // bf16 > 0: sign clear, magnitude non-zero
-          if (!(lo != 0u && lo < 0x8000u)) v[8 * i + 2 * j] = 0.f;
-          if (!(hi != 0u && hi < 0x8000u)) v[8 * i + 2 * j + 1] = 0.f;
-        }
-      }
-    } else {
-#pragma unroll
-      for (int i = 0; i < 32; ++i)
-        if (col0 + i < p.cols && !(__bfloat162float(mk[i]) > 0.f)) v[i] = 0.f;
-    }
-  }
-  if (p.out_f32) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      *reinterpret_cast<float4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16)) =
-          make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-  } else {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      uint32_t w[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const __nv_bfloat162 pr = __floats2bfloat162_rn(v[8 * i + 2 * j], v[8 * i + 2 * j + 1]);
-        w[j] = *reinterpret_cast<const uint32_t*>(&pr);
-      }
-      *reinterpret_cast<uint4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-  }
-}
-
-template <bool A_K, bool B_K>
+template <bool A_K, bool B_K, bool MASK>
 __global__ void __launch_bounds__(kThreads, 1)
 umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const Params2 p) {
@@ -298,37 +231,16 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const int ew = warp - 2;
     const int q = warp & 3;
     const int half = ew >> 2;
-    constexpr int kHalfCols = BN / 2;
     unsigned char* stg = smem + kStgOff + ew * kStgWarpBytes;
-    unsigned char* srow = stg + lane * kStgRowBytes;
     int acc = 0; uint32_t acc_phase = 0;
     for (int tile = pair; tile < p.total_tiles && ok; tile += n_pairs) {
       const TileCoord t = decode(p, tile);
+      const int tile_row0 = t.mt * 2 * BM + (int)rank * BM;     // this CTA's 128 rows of the 256-row tile
+      uint4 mreg[MASK ? 8 : 1];
+      if (MASK) load_mask_block(p, t.b, tile_row0 + q * 32, round_col0<BN>(t, half, 0), lane, mreg);
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      const int row0 = t.mt * 2 * BM + (int)rank * BM + q * 32;
-      const bool row_ok = row0 + lane < p.rows;
-      const long long row_off = (long long)t.b * p.c_bs + (long long)(row0 + lane) * p.c_ld;
-      const uint32_t t_acc = tmem_base + (uint32_t)(acc * BN + half * kHalfCols) + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
-      for (int c = 0; c < kHalfCols / 64; ++c) {
-        const int col0 = t.nt * BN + half * kHalfCols + c * 64;
-        if (col0 >= p.cols) break;
-        uint32_t r0[32], r1[32];
-        ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r0);
-        ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r1);
-        ptx::tmem_ld_wait();
-        if (p.out_f32) {
-          process_chunk2(r0, p, srow, lane, 0, row_ok, row_off, col0);
-          flush_rows2(stg, p, t.b, row0, col0, lane);
-          process_chunk2(r1, p, srow, lane, 0, row_ok, row_off, col0 + 32);
-          flush_rows2(stg, p, t.b, row0, col0 + 32, lane);
-        } else {
-          process_chunk2(r0, p, srow, lane, 0, row_ok, row_off, col0);
-          process_chunk2(r1, p, srow, lane, 4, row_ok, row_off, col0 + 32);
-          flush_rows2(stg, p, t.b, row0, col0, lane);
-        }
-      }
+      epilogue_tile<BN, MASK>(p, t, tile_row0, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, mreg);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(map_to_cta(ptx::smem_u32(acc_empty + acc), 0));   // the leader's barrier
@@ -353,9 +265,9 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   }
 }
 
-template <bool A_K, bool B_K>
+template <bool A_K, bool B_K, bool MASK>
 int launch2_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params2& p, int pairs, cudaStream_t st) {
-  auto kern = umma2_gemm_kernel<A_K, B_K>;
+  auto kern = umma2_gemm_kernel<A_K, B_K, MASK>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
     return GSHARD_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
@@ -381,6 +293,7 @@ int launch2_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params2& p, in
 // launch_umma_gemm.  Worth it when a problem has more than one 128-row tile.
 int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (g.rows <= 0 || g.cols <= 0 || g.K <= 0 || g.batch <= 0) return GSHARD_OK;
+  if (g.mask && g.out_f32) return GSHARD_ERR_INTERNAL;   // the mask is staged as bf16 rows
   CUtensorMap ma, mb;
   bool okm;
   if (g.a_kmajor) okm = make_map(&ma, g.A, g.K, g.rows, g.batch, g.a_ld, g.a_bs, BK, BM);
@@ -401,10 +314,13 @@ int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   int pairs = sms / 2;
   if (pairs > p.total_tiles) pairs = p.total_tiles;
-  if (g.a_kmajor && g.b_kmajor) return launch2_t<true, true>(ma, mb, p, pairs, st);
-  if (g.a_kmajor && !g.b_kmajor) return launch2_t<true, false>(ma, mb, p, pairs, st);
-  if (!g.a_kmajor && g.b_kmajor) return launch2_t<false, true>(ma, mb, p, pairs, st);
-  return launch2_t<false, false>(ma, mb, p, pairs, st);
+#define GSHARD_DISPATCH2(AK, BKM) \
+  (p.mask ? launch2_t<AK, BKM, true>(ma, mb, p, pairs, st) : launch2_t<AK, BKM, false>(ma, mb, p, pairs, st))
+  if (g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH2(true, true);
+  if (g.a_kmajor && !g.b_kmajor) return GSHARD_DISPATCH2(true, false);
+  if (!g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH2(false, true);
+  return GSHARD_DISPATCH2(false, false);
+#undef GSHARD_DISPATCH2
 }
 
 }  // namespace gshard

@@ -21,18 +21,19 @@
 #include "kernels.cuh"
 #include "sm100_ptx.cuh"
 #include "tensor_map.cuh"
+#include "umma_epilogue.cuh"
 
 namespace gshard {
 
 namespace {
+
+using namespace umma_epi;
 
 constexpr int BM = 128, BK = 64;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kABytes = BM * BK * 2;        // 16 KB
 constexpr int kBoxBytes = 64 * 64 * 2;      // one 64x64 box of an MN-major operand
-constexpr int kStgRowBytes = 128;           // epilogue staging: 32 rows x 128 bytes per warp
-constexpr int kStgWarpBytes = 32 * kStgRowBytes;
 
 template <int BN> struct Cfg {
   static constexpr int b_bytes = BN * BK * 2;
@@ -56,146 +57,12 @@ struct Params {
   int* status;
 };
 
-struct TileCoord { int mt, nt, b; };
-
 __device__ __forceinline__ TileCoord decode(const Params& p, int tile) {
   TileCoord t;
   t.mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
   t.nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
   t.b = tile / (p.m_tiles * p.n_tiles);
   return t;
-}
-
-// Writes a warp's staged 32 rows x 128 bytes to C: lane l handles 16-byte piece (l & 7) of rows
-// 4*i + (l >> 3); pieces beyond the matrix edge are skipped (cols is a multiple of the piece width).
-__device__ __forceinline__ void flush_rows(const unsigned char* stg, const Params& p, int b, int row0, int col0,
-                                           int lane) {
-  __syncwarp();
-  const int esz = p.out_f32 ? 4 : 2;
-  const int piece = lane & 7;
-  const int col = col0 + piece * (16 / esz);
-  unsigned char* cbase = reinterpret_cast<unsigned char*>(p.C) + ((long long)b * p.c_bs + col) * esz;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int r = 4 * i + (lane >> 3);
-    const int row = row0 + r;
-    if (row < p.rows && col < p.cols) {
-      const uint4 val = *reinterpret_cast<const uint4*>(stg + r * kStgRowBytes + ((piece ^ (r & 7)) * 16));
-      *reinterpret_cast<uint4*>(cbase + (long long)row * p.c_ld * esz) = val;
-    }
-  }
-  __syncwarp();
-}
-
-// Coalesced load of a warp's 32 x 64 block of the bf16 mask (128 bytes per row): lane l takes piece
-// (l & 7) of rows 4*i + (l >> 3), the pattern of flush_rows.  Pieces outside the matrix read as zero.
-__device__ __forceinline__ void load_mask_block(const Params& p, int b, int row0, int col0, int lane, uint4* m) {
-  const int piece = lane & 7;
-  const int col = col0 + piece * 8;
-  const unsigned char* base = reinterpret_cast<const unsigned char*>(p.mask) + ((long long)b * p.c_bs + col) * 2;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int row = row0 + 4 * i + (lane >> 3);
-    m[i] = (row < p.rows && col < p.cols) ? __ldg(reinterpret_cast<const uint4*>(base + (long long)row * p.c_ld * 2))
-                                          : make_uint4(0u, 0u, 0u, 0u);
-  }
-}
-
-__device__ __forceinline__ void stage_mask_block(unsigned char* stg, int lane, const uint4* m) {
-  const int piece = lane & 7;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int r = 4 * i + (lane >> 3);
-    *reinterpret_cast<uint4*>(stg + r * kStgRowBytes + ((piece ^ (r & 7)) * 16)) = m[i];
-  }
-  __syncwarp();
-}
-
-// ReLU / mask on one 32-column chunk of this thread's row, then into the staging row (XOR-swizzled
-// 16-byte pieces: conflict-free for the row-wise writes here and the piece-wise reads of the flush).
-template <bool MASK>
-__device__ __forceinline__ void process_chunk(const uint32_t* r, const Params& p, unsigned char* srow, int lane,
-                                              int piece0) {
-  float v[32];
-#pragma unroll
-  for (int i = 0; i < 32; ++i) {
-    v[i] = __uint_as_float(r[i]);
-    if (p.relu) v[i] = fmaxf(v[i], 0.f);
-  }
-  if (MASK) {
-    // the mask block was staged into this row's pieces (same swizzle as the output written below)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint4 mv = *reinterpret_cast<const uint4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16));
-      const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        // bf16 > 0  <=>  sign bit clear and magnitude bits non-zero
-        const uint32_t lo = w[j] & 0xffffu, hi = w[j] >> 16;
-        if (!(lo != 0u && lo < 0x8000u)) v[8 * i + 2 * j] = 0.f;
-        if (!(hi != 0u && hi < 0x8000u)) v[8 * i + 2 * j + 1] = 0.f;
-      }
-    }
-  }
-  if (p.out_f32) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      *reinterpret_cast<float4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16)) =
-          make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-  } else {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      uint32_t w[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const __nv_bfloat162 pr = __floats2bfloat162_rn(v[8 * i + 2 * j], v[8 * i + 2 * j + 1]);
-        w[j] = *reinterpret_cast<const uint32_t*>(&pr);
-      }
-      *reinterpret_cast<uint4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16)) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-  }
-}
-
-// First column of round c of this warp's half of the tile.
-template <int BN>
-__device__ __forceinline__ int round_col0(const TileCoord& t, int half, int c) {
-  return t.nt * BN + half * (BN / 2) + c * 64;
-}
-
-// One epilogue warp's share of a finished 128 x BN accumulator: lane quarter q, column half `half`.
-// With a mask (bf16 output only) `mreg` holds the mask block of round 0, loaded by the caller
-// before it waited for the accumulator; the block of round c + 1 is fetched while round c is
-// processed, so the mask's global-memory latency stays off the accumulator's critical path.
-template <int BN, bool MASK>
-__device__ __forceinline__ void epilogue_tile(const Params& p, const TileCoord& t, uint32_t tmem_acc, int q, int half,
-                                              unsigned char* stg, int lane, uint4* mreg) {
-  constexpr int kHalfCols = BN / 2;
-  unsigned char* srow = stg + lane * kStgRowBytes;
-  const int row0 = t.mt * BM + q * 32;
-  const uint32_t t_acc = tmem_acc + (uint32_t)(half * kHalfCols) + ((uint32_t)(q * 32) << 16);
-#pragma unroll 1
-  for (int c = 0; c < kHalfCols / 64; ++c) {     // 64 columns per round: two TMEM loads in flight
-    const int col0 = round_col0<BN>(t, half, c);
-    if (col0 >= p.cols) break;                   // uniform over the warp
-    uint32_t r0[32], r1[32];
-    ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r0);
-    ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r1);
-    if (MASK) {
-      stage_mask_block(stg, lane, mreg);
-      if (c + 1 < kHalfCols / 64) load_mask_block(p, t.b, row0, col0 + 64, lane, mreg);
-    }
-    ptx::tmem_ld_wait();
-    if (p.out_f32) {                             // 32 fp32 columns = one 128-byte staging row
-      process_chunk<MASK>(r0, p, srow, lane, 0);
-      flush_rows(stg, p, t.b, row0, col0, lane);
-      process_chunk<MASK>(r1, p, srow, lane, 0);
-      flush_rows(stg, p, t.b, row0, col0 + 32, lane);
-    } else {                                     // 64 bf16 columns = one 128-byte staging row
-      process_chunk<MASK>(r0, p, srow, lane, 0);
-      process_chunk<MASK>(r1, p, srow, lane, 4);
-      flush_rows(stg, p, t.b, row0, col0, lane);
-    }
-  }
 }
 
 template <bool A_K, bool B_K, int BN, bool MASK>
@@ -308,7 +175,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       if (MASK) load_mask_block(p, t.b, t.mt * BM + q * 32, round_col0<BN>(t, half, 0), lane, mreg);
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      epilogue_tile<BN, MASK>(p, t, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, mreg);
+      epilogue_tile<BN, MASK>(p, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, mreg);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
@@ -470,7 +337,7 @@ umma_gemm_resident_b_kernel(const __grid_constant__ CUtensorMap map_a, const __g
       for (t.mt = 0; t.mt < p.m_tiles; ++t.mt) {
         if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
         ptx::tc_fence_after_sync();
-        epilogue_tile<BN, false>(p, t, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, nullptr);
+        epilogue_tile<BN, false>(p, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, nullptr);
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
