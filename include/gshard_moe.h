@@ -131,7 +131,10 @@ size_t gshard_moe_top2_host_staging_bytes(const gshard_moe_shape* shape);
  *   Algorithm 1's group loss.  routing_out: NULL or a struct of optional outputs.
  *   context: NULL, or gshard_moe_top2_context_bytes() bytes when SAVE_FOR_BACKWARD is set.
  *   workspace: at least gshard_moe_top2_workspace_bytes(shape, 0) bytes, 256-byte aligned;
- *   its contents are scratch. */
+ *   its contents are scratch.
+ * The call only enqueues kernels and memsets on cuda_stream (no allocation, no synchronisation, no
+ * work on other streams), so it may be recorded into a CUDA graph by stream capture and replayed
+ * on new contents of the same buffers. */
 int gshard_moe_top2_forward(const gshard_moe_shape* shape, const void* x, const void* wg,
                             const void* wi, const void* wo, const float* u, void* y,
                             float* l_aux, const gshard_moe_routing* routing_out, void* context,

@@ -61,3 +61,36 @@ def test_host_calls_match_device_call(dtype, H):
     for i in range(steps):
         assert torch.equal(yhs[i].view(torch.uint8), ref[i][0].view(torch.uint8)), f"step {i}"
         assert float(lhs[i]) == ref[i][1]
+
+
+def test_forward_replays_from_a_cuda_graph():
+    """The device-buffer forward only enqueues work on the caller's stream (no allocation, no
+    synchronisation), so it can be captured once and replayed on new inputs in the same buffers."""
+    cfg = MoEConfig("graph", G=2, S=256, M=256, H=1024, E=32, C=16, dtype="bf16", seed=93)
+    inp = make_inputs(cfg, "cuda")
+    shape = B.make_shape(cfg)
+    ws = B.alloc_workspace(shape)
+    x, u = inp["x"].clone(), inp["u"].clone()
+    y = torch.empty_like(x)
+    l_aux = torch.zeros(1, device="cuda")
+    # eager reference on two different inputs
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    x2 = torch.randn(cfg.G, cfg.S, cfg.M, generator=gen, device="cuda").to(torch.bfloat16)
+    u2 = torch.rand(cfg.G, cfg.S, generator=gen, device="cuda")
+    refs = []
+    for xi, ui in ((inp["x"], inp["u"]), (x2, u2)):
+        yi = torch.empty_like(xi)
+        li = torch.zeros(1, device="cuda")
+        B.gshard_moe_top2_forward(shape, xi, inp["wg"], inp["wi"], inp["wo"], ui, yi, li, None, None, ws)
+        torch.cuda.synchronize()
+        refs.append((yi.clone(), float(li)))
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        B.gshard_moe_top2_forward(shape, x, inp["wg"], inp["wi"], inp["wo"], u, y, l_aux, None, None, ws,
+                                  torch.cuda.current_stream())
+    for (xi, ui), (y_ref, l_ref) in zip(((inp["x"], inp["u"]), (x2, u2)), refs):
+        x.copy_(xi); u.copy_(ui)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert B.gshard_moe_last_device_status(ws) == B.GSHARD_OK
+        assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16)) and float(l_aux) == l_ref
