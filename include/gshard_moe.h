@@ -80,6 +80,10 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                               second pass - measured faster on B200 */
 #define GSHARD_FLAG_ONE_SM_MMA 512u        /* no grouped GEMM runs on CTA pairs (128 x 256 tiles on
                                               single CTAs everywhere) */
+#define GSHARD_FLAG_ADD_RESIDUAL 1024u      /* forward: y = x + layer(x), the residual connection around the
+                                              layer (section 2.2, expert capacity: overflowed tokens pass through it) folded
+                                              into the combine; backward: dx also receives dy.  Not
+                                              applied by the stage call gshard_moe_combine */
 #define GSHARD_FLAG_GATE_TWO_SM 256u       /* the default gating kernel on CTA pairs (tcgen05
                                               cta_group::2: each CTA loads half of the wg tile); needs
                                               E % 128 == 0, elsewhere ignored */

@@ -35,6 +35,7 @@ GSHARD_FLAG_GATHER_DISPATCH = 64
 GSHARD_FLAG_GATE_CLUSTER = 128
 GSHARD_FLAG_GATE_TWO_SM = 256
 GSHARD_FLAG_ONE_SM_MMA = 512
+GSHARD_FLAG_ADD_RESIDUAL = 1024
 
 
 class gshard_moe_shape(Structure):

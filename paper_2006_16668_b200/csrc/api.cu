@@ -124,7 +124,7 @@ int validate_shape(const gshard_moe_shape* s) {
   if (!s) return GSHARD_ERR_INVALID_ARG;
   if (s->G <= 0 || s->S <= 0 || s->M <= 0 || s->H <= 0 || s->E <= 0 || s->C <= 0) return GSHARD_ERR_INVALID_ARG;
   if (s->dtype != GSHARD_F32 && s->dtype != GSHARD_BF16) return GSHARD_ERR_INVALID_ARG;
-  if (s->flags & ~1023u) return GSHARD_ERR_INVALID_ARG;
+  if (s->flags & ~2047u) return GSHARD_ERR_INVALID_ARG;
   if ((s->flags & GSHARD_FLAG_FUSED_FFN) && (s->flags & GSHARD_FLAG_UNFUSED_FFN)) return GSHARD_ERR_INVALID_ARG;
   if (s->E < 2) return GSHARD_ERR_INVALID_ARG;
   if (s->M % 8 || s->H % 8) return GSHARD_ERR_UNSUPPORTED_SHAPE;
@@ -183,7 +183,7 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
   GS_TRY(ffn_stage(d, buf, wi, wo, h, save, out, ws + pl.ffn_scratch, status, st, gather ? x : nullptr, slot_token));
   if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.stop), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   ft.start = ft.stop = nullptr;
-  launch_combine(d, out, expert_idx, slot, weight, y, st);
+  launch_combine(d, out, expert_idx, slot, weight, y, st, d.add_residual ? x : nullptr);
 
   if (save) {   // hand the caller the routing tensors it asked for
     struct { void* dst; const void* src; size_t n; } cps[] = {

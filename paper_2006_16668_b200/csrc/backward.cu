@@ -160,7 +160,8 @@ __global__ void __launch_bounds__(256) gate_bwd_kernel(const float* __restrict__
 template <typename T>
 __global__ void __launch_bounds__(256) dx_kernel(const float4* __restrict__ dxg, const uint4* __restrict__ dbuf,
                                                  const int32_t* __restrict__ expert_idx, const int32_t* __restrict__ slot,
-                                                 uint4* __restrict__ dx, long long N, int G, int S, int C, int row_vec) {
+                                                 const uint4* __restrict__ dy_res, uint4* __restrict__ dx, long long N,
+                                                 int G, int S, int C, int row_vec) {
   constexpr int n = Row16<T>::n;
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -186,6 +187,12 @@ __global__ void __launch_bounds__(256) dx_kernel(const float4* __restrict__ dxg,
         if (!r[k]) continue;
         float f[n];
         Row16<T>::load(__ldg(r[k] + i), f);
+#pragma unroll
+        for (int j = 0; j < n; ++j) acc[j] += f[j];
+      }
+      if (dy_res) {                                  // residual connection: dx also receives dy
+        float f[n];
+        Row16<T>::load(__ldg(dy_res + t * row_vec + i), f);
 #pragma unroll
         for (int j = 0; j < n; ++j) acc[j] += f[j];
       }
@@ -326,8 +333,9 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   rc = run_gemm(d, g, status, st);
   if (rc) return rc;
   dx_kernel<T><<<grid_rows(d.N), 256, 0, st>>>(reinterpret_cast<const float4*>(dxg), reinterpret_cast<const uint4*>(dbuf),
-                                               expert_idx, slot, reinterpret_cast<uint4*>(dx), d.N, d.G, d.S, d.C,
-                                               row_vec);
+                                               expert_idx, slot,
+                                               d.add_residual ? reinterpret_cast<const uint4*>(dy) : nullptr,
+                                               reinterpret_cast<uint4*>(dx), d.N, d.G, d.S, d.C, row_vec);
   count_launch();
   return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }

@@ -59,12 +59,14 @@ template <> struct Vec16<__nv_bfloat16> {
   }
 };
 
-// y[t,:] = w0*out[e0, g*C+slot0, :] + w1*out[e1, g*C+slot1, :] over the kept choices, fp32 FMA.
+// y[t,:] = w0*out[e0, g*C+slot0, :] + w1*out[e1, g*C+slot1, :] over the kept choices, fp32 FMA;
+// with `residual` the token's input row is added (the residual connection around the layer).
 template <typename T>
 __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ out,
                                                       const int32_t* __restrict__ expert_idx,
                                                       const int32_t* __restrict__ slot,
                                                       const float* __restrict__ weight,
+                                                      const uint4* __restrict__ residual,
                                                       uint4* __restrict__ y, long long N, int G, int S,
                                                       int C, int row_vec) {
   constexpr int n = Vec16<T>::n;
@@ -82,11 +84,12 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
       float acc[n];
 #pragma unroll
       for (int j = 0; j < n; ++j) acc[j] = 0.f;
+      if (residual) Vec16<T>::load(__ldg(residual + t * row_vec + i), acc);
       if (r0) {
         float f[n];
         Vec16<T>::load(__ldg(r0 + i), f);
 #pragma unroll
-        for (int j = 0; j < n; ++j) acc[j] = w0 * f[j];
+        for (int j = 0; j < n; ++j) acc[j] = fmaf(w0, f[j], acc[j]);
       }
       if (r1) {
         float f[n];
@@ -113,16 +116,16 @@ void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, vo
 }
 
 void launch_combine(const Dims& d, const void* out, const int32_t* expert_idx, const int32_t* slot,
-                    const float* weight, void* y, cudaStream_t st) {
+                    const float* weight, void* y, cudaStream_t st, const void* residual) {
   const int row_vec = (int)((size_t)d.M * d.esize / 16);
   if (d.bf16)
     combine_kernel<__nv_bfloat16><<<grid_for_rows(d.N), 256, 0, st>>>(
-        reinterpret_cast<const uint4*>(out), expert_idx, slot, weight, reinterpret_cast<uint4*>(y), d.N, d.G, d.S,
-        d.C, row_vec);
+        reinterpret_cast<const uint4*>(out), expert_idx, slot, weight, reinterpret_cast<const uint4*>(residual),
+        reinterpret_cast<uint4*>(y), d.N, d.G, d.S, d.C, row_vec);
   else
     combine_kernel<float><<<grid_for_rows(d.N), 256, 0, st>>>(
-        reinterpret_cast<const uint4*>(out), expert_idx, slot, weight, reinterpret_cast<uint4*>(y), d.N, d.G, d.S,
-        d.C, row_vec);
+        reinterpret_cast<const uint4*>(out), expert_idx, slot, weight, reinterpret_cast<const uint4*>(residual),
+        reinterpret_cast<uint4*>(y), d.N, d.G, d.S, d.C, row_vec);
   count_launch();
 }
 

@@ -35,7 +35,7 @@ int capacity_warps_for(int E);
 // dispatch_combine.cu
 void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st);
 void launch_combine(const Dims& d, const void* out, const int32_t* expert_idx, const int32_t* slot,
-                    const float* weight, void* y, cudaStream_t st);
+                    const float* weight, void* y, cudaStream_t st, const void* residual = nullptr);
 
 // umma_gemm.cu: batched bf16 GEMM on tcgen05, C[b] = act(A[b] . B[b]).
 struct UmmaGemm {

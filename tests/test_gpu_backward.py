@@ -168,3 +168,35 @@ def test_backward_training_config_sampled():
         _, dlogit, xs = _token_grads(cfg, inp, ei, slot, fc, wg, g, s, 0.0, to_np(inp["dy"][g, s]))
         ref_dwg += np.outer(xs.astype(np.float64), dlogit)          # dwg = sum x^T dlogit
     assert rel_fro(to_np(dwg2), ref_dwg) <= GRAD_TOL
+
+
+@pytest.mark.parametrize("dtype,tol", [("f32", 1e-5), ("bf16", 1e-2)])
+def test_residual_connection_folded_into_combine_and_dx(dtype, tol):
+    """GSHARD_FLAG_ADD_RESIDUAL: y = x + layer(x) and dx = dx_layer + dy, against the same layer without the
+    flag (whose parity with the oracle the other tests establish)."""
+    M, H = (64, 128)
+    cfg = MoEConfig("res", G=2, S=128, M=M, H=H, E=16, C=12, dtype=dtype, seed=5, backward=True, k_aux=0.01)
+    inp = make_inputs(cfg, "cuda")
+    outs = {}
+    for flag in (0, B.GSHARD_FLAG_ADD_RESIDUAL):
+        shape = B.make_shape(cfg, flags=B.GSHARD_FLAG_SAVE_FOR_BACKWARD | flag)
+        ws = B.alloc_workspace(shape, for_backward=True)
+        wsf = B.alloc_workspace(shape)
+        ctx = torch.empty(B.gshard_moe_top2_context_bytes(shape), dtype=torch.uint8, device="cuda")
+        y = torch.empty_like(inp["x"])
+        l_aux = torch.zeros(1, device="cuda")
+        B.gshard_moe_top2_forward(shape, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l_aux, None, ctx, wsf)
+        dx = torch.empty_like(inp["x"])
+        dwg = torch.empty(cfg.M, cfg.E, device="cuda")
+        dwi, dwo = torch.empty_like(inp["wi"]), torch.empty_like(inp["wo"])
+        B.gshard_moe_top2_backward(shape, inp["x"], inp["wg"], inp["wi"], inp["wo"], ctx, inp["dy"], cfg.k_aux, dx, dwg,
+                                   dwi, dwo, ws)
+        assert B.gshard_moe_last_device_status(ws) == B.GSHARD_OK
+        outs[flag] = (y.float().cpu(), dx.float().cpu(), dwg.cpu(), dwi.float().cpu(), dwo.float().cpu())
+    y0, dx0, dwg0, dwi0, dwo0 = outs[0]
+    y1, dx1, dwg1, dwi1, dwo1 = outs[B.GSHARD_FLAG_ADD_RESIDUAL]
+    x, dy = inp["x"].float().cpu(), inp["dy"].float().cpu()
+    assert rel_fro(y1.numpy(), (y0 + x).numpy()) <= tol
+    assert rel_fro(dx1.numpy(), (dx0 + dy).numpy()) <= tol
+    # the weight gradients do not see the residual path
+    assert torch.equal(dwg0, dwg1) and torch.equal(dwi0, dwi1) and torch.equal(dwo0, dwo1)
