@@ -198,7 +198,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--one-sm-mma", action="store_true", help="ablation: no grouped GEMM on CTA pairs")
-    ap.add_argument("--gate-two-sm", action="store_true", help="ablation: gating GEMM on CTA pairs (cta_group::2)")
+    ap.add_argument("--gate-one-sm", action="store_true", help="ablation: gating GEMM on single CTAs, row-major logits")
     ap.add_argument("--gate-cluster", action="store_true",
                     help="ablation: cluster gating kernel with the mean-gate partial sums fused in")
     ap.add_argument("--gather-dispatch", action="store_true",
@@ -237,7 +237,7 @@ def main():
                          (B.GSHARD_FLAG_TWO_SM_MMA if args.two_sm_mma else 0) |
                          (B.GSHARD_FLAG_GATHER_DISPATCH if args.gather_dispatch else 0) |
                          (B.GSHARD_FLAG_GATE_CLUSTER if args.gate_cluster else 0) |
-                         (B.GSHARD_FLAG_GATE_TWO_SM if args.gate_two_sm else 0) |
+                         (B.GSHARD_FLAG_GATE_ONE_SM if args.gate_one_sm else 0) |
                          (B.GSHARD_FLAG_ONE_SM_MMA if args.one_sm_mma else 0))
     ws = B.alloc_workspace(shape, host_staging=True, device=dev)
     y = torch.empty_like(inp["x"])

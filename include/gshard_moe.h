@@ -84,9 +84,10 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                               layer (section 2.2, expert capacity: overflowed tokens pass through it) folded
                                               into the combine; backward: dx also receives dy.  Not
                                               applied by the stage call gshard_moe_combine */
-#define GSHARD_FLAG_GATE_TWO_SM 256u       /* the default gating kernel on CTA pairs (tcgen05
-                                              cta_group::2: each CTA loads half of the wg tile); needs
-                                              E % 128 == 0, elsewhere ignored */
+#define GSHARD_FLAG_GATE_ONE_SM 256u       /* gating GEMM on single CTAs with row-major stored logits.  By
+                                              default, where E % 128 == 0, it runs on CTA pairs (tcgen05
+                                              cta_group::2: each CTA loads half of the wg tile) and stores
+                                              the logits in 16-byte granules laid out [E/4][N] */
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

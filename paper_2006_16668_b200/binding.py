@@ -33,7 +33,7 @@ GSHARD_FLAG_UNFUSED_FFN = 16
 GSHARD_FLAG_TWO_SM_MMA = 32
 GSHARD_FLAG_GATHER_DISPATCH = 64
 GSHARD_FLAG_GATE_CLUSTER = 128
-GSHARD_FLAG_GATE_TWO_SM = 256
+GSHARD_FLAG_GATE_ONE_SM = 256
 GSHARD_FLAG_ONE_SM_MMA = 512
 GSHARD_FLAG_ADD_RESIDUAL = 1024
 

@@ -46,7 +46,7 @@ struct Dims {
   bool two_sm_mma;      // grouped GEMMs on CTA pairs (tcgen05 cta_group::2) where rows > 128
   bool add_residual;    // y = x + layer(x); dx gains dy
   bool one_sm_mma;      // never use CTA pairs for the grouped GEMMs
-  bool gate_two_sm;     // stored-logits gating kernel on CTA pairs (cta_group::2)
+  bool gate_one_sm;     // stored-logits gating kernel on single CTAs instead of CTA pairs
   bool gate_cluster;    // gating on clusters with the mean-gate partial sums fused in (no stored logits)
   bool gather_dispatch; // single-launch FFN gathers its rows from x instead of reading a dispatch buffer
 };
@@ -67,7 +67,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.two_sm_mma = (s.flags & GSHARD_FLAG_TWO_SM_MMA) != 0;
   d.gather_dispatch = (s.flags & GSHARD_FLAG_GATHER_DISPATCH) != 0;
   d.gate_cluster = (s.flags & GSHARD_FLAG_GATE_CLUSTER) != 0;
-  d.gate_two_sm = (s.flags & GSHARD_FLAG_GATE_TWO_SM) != 0;
+  d.gate_one_sm = (s.flags & GSHARD_FLAG_GATE_ONE_SM) != 0;
   d.one_sm_mma = (s.flags & GSHARD_FLAG_ONE_SM_MMA) != 0;
   d.add_residual = (s.flags & GSHARD_FLAG_ADD_RESIDUAL) != 0;
   return d;

@@ -150,6 +150,70 @@ __global__ void __launch_bounds__(128) gate_colsum4_kernel(const float4* __restr
   partial[(long long)tile * E4 + e4] = acc;
 }
 
+
+// Column sums from logits stored in 16-byte granules of four experts, float4 [E/4][N] (the layout the
+// CTA-pair gating kernel writes): a warp takes one granule column and a 128-token tile, its lanes
+// read 32 consecutive tokens (512 contiguous bytes) per load, four granule columns in flight, and
+// the 32 partial sums meet in a shuffle tree (fixed order).
+__global__ void __launch_bounds__(128) gate_colsum_t_kernel(const float4* __restrict__ logits_t,
+                                                            const float* __restrict__ rowmax,
+                                                            const float* __restrict__ rowinv, long long N,
+                                                            int S, int E4, int tiles_per_group,
+                                                            float4* __restrict__ partial) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int tile = blockIdx.y;
+  const int g = tile / tiles_per_group;
+  const int s0 = (tile % tiles_per_group) * kGateTile;
+  const int n = min(S, s0 + kGateTile) - s0;
+  const long long row0 = (long long)g * S + s0;
+  constexpr float kLog2e = 1.4426950408889634f;
+  float mxl[4], iv[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    const int i = r * 32 + lane;
+    mxl[r] = i < n ? rowmax[row0 + i] * kLog2e : 0.f;
+    iv[r] = i < n ? rowinv[row0 + i] : 0.f;          // rows past the group's end contribute nothing
+  }
+  // this block's granule columns: 64 per block, 16 per warp, four at a time
+  const int c_first = blockIdx.x * 64 + warp * 16;
+  for (int cb = 0; cb < 16; cb += 4) {
+    float4 acc[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 v[4][4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int c4 = c_first + cb + j;
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int i = r * 32 + lane;
+        v[j][r] = (c4 < E4 && i < n) ? __ldcs(logits_t + (long long)c4 * N + row0 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        acc[j].x += exp2f(fmaf(v[j][r].x, kLog2e, -mxl[r])) * iv[r];
+        acc[j].y += exp2f(fmaf(v[j][r].y, kLog2e, -mxl[r])) * iv[r];
+        acc[j].z += exp2f(fmaf(v[j][r].z, kLog2e, -mxl[r])) * iv[r];
+        acc[j].w += exp2f(fmaf(v[j][r].w, kLog2e, -mxl[r])) * iv[r];
+      }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+#pragma unroll
+      for (int off = 16; off >= 1; off >>= 1) {
+        acc[j].x += __shfl_xor_sync(0xffffffffu, acc[j].x, off);
+        acc[j].y += __shfl_xor_sync(0xffffffffu, acc[j].y, off);
+        acc[j].z += __shfl_xor_sync(0xffffffffu, acc[j].z, off);
+        acc[j].w += __shfl_xor_sync(0xffffffffu, acc[j].w, off);
+      }
+      const int c4 = c_first + cb + j;
+      if (lane == 0 && c4 < E4) partial[(long long)tile * E4 + c4] = acc[j];
+    }
+  }
+}
+
 void launch_gate_rows(const Dims& d, const float* logits, int32_t* expert_idx, float* gate12,
                       float* rowmax, float* rowinv, cudaStream_t st) {
   const long long warps_needed = d.N;
@@ -170,6 +234,17 @@ void launch_gate_means(const Dims& d, const float* logits, const float* rowmax, 
     dim3 grid(ceil_div(d.E, 128), d.G * d.tiles_per_group);
     gate_colsum_kernel<<<grid, 128, 0, st>>>(logits, rowmax, rowinv, d.S, d.E, d.tiles_per_group, partial);
   }
+  gate_mean_kernel<<<dim3(ceil_div(d.E, 128), d.G), 128, 0, st>>>(partial, d.S, d.E, d.tiles_per_group, m);
+  count_launch(2);
+}
+
+// m[g,e] from logits stored as float4 [E/4][N] and row statistics (two launches).
+void launch_gate_means_t(const Dims& d, const float* logits_t, const float* rowmax, const float* rowinv,
+                         float* partial, float* m, cudaStream_t st) {
+  const int E4 = d.E / 4;
+  dim3 grid(ceil_div(E4, 64), d.G * d.tiles_per_group);
+  gate_colsum_t_kernel<<<grid, 128, 0, st>>>(reinterpret_cast<const float4*>(logits_t), rowmax, rowinv, d.N, d.S, E4,
+                                             d.tiles_per_group, reinterpret_cast<float4*>(partial));
   gate_mean_kernel<<<dim3(ceil_div(d.E, 128), d.G), 128, 0, st>>>(partial, d.S, d.E, d.tiles_per_group, m);
   count_launch(2);
 }

@@ -441,7 +441,7 @@ gate_cluster_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
       }
       ptx::tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(acc_empty + acc2);
+      if (lane == 0) ptx::mbar_arrive_relaxed(acc_empty + acc2);
       acc2 ^= 1;
     }
   }

@@ -267,7 +267,7 @@ gate_fused_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_consta
         }
         ptx::tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
+        if (lane == 0) ptx::mbar_arrive_relaxed(acc_empty + acc);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
       if (!ok) break;

@@ -1,7 +1,7 @@
 // Gating for the bf16 dtype on CTA pairs (tcgen05.mma.cta_group::2): the same computation as
 // gate_fused.cu - logits = x . wg with fp32 accumulation and, while the accumulator is read out of
 // tensor memory, the online softmax statistics and the top-2 pick of Algorithm 1, plus the stored
-// fp32 logits for the mean-gate pass - but a pair of CTAs (a cluster of two) works on 256 tokens:
+// fp32 logits for the mean-gate pass (here in the granule-transposed layout [E/4][N][4]) - but a pair of CTAs (a cluster of two) works on 256 tokens:
 // each CTA loads its own 128 token rows of x and only HALF of the 256-expert slice of wg per
 // k-block (32 KB per stage instead of 48 KB), and the leader's MMA thread multiplies both halves
 // into the accumulators of both CTAs.  The one-SM kernel is bound by the operand feed from L2
@@ -29,13 +29,11 @@ constexpr int BNH = BN / 2;
 constexpr int kBBytes = BNH * BK * 2;          // this CTA's half of the wg tile
 constexpr int kBoxBytes = 64 * 64 * 2;
 constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kStages = 4;
+constexpr int kStages = 6;
 constexpr int kTmemCols = 2 * BN;
 constexpr int kBarOff = kStages * kStageBytes;
 constexpr int kStgOff = kBarOff + 256;
-constexpr int kStgRowBytes = 128;
-constexpr int kStgWarpBytes = 32 * kStgRowBytes;
-constexpr int kXchgOff = kStgOff + kEpiWarps * kStgWarpBytes;   // 24 B [4 quarters][3 parts][32 rows]
+constexpr int kXchgOff = kStgOff;                                // 24 B [4 quarters][3 parts][32 rows]
 constexpr int kSmemBytes = kXchgOff + 4 * 3 * 32 * 24 + 1024;
 static_assert(kSmemBytes <= 232448, "shared memory budget");
 
@@ -43,7 +41,7 @@ struct GateParams {
   long long N;          // tokens
   int E, M;
   int row_tiles, n_tiles, k_blocks;   // row tiles of 128 tokens; a pair takes two
-  float* logits;        // [N,E] fp32
+  float* logits;        // fp32, granules of four experts: float4 [E/4][N]
   int32_t* expert_idx;  // [N,2]
   float* gate12;        // [N,2] raw softmax values of the two picks
   float* rowmax;        // [N]
@@ -65,8 +63,11 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// Arrive on a barrier of the peer CTA.  What the barrier hands over is a TMEM accumulator, ordered
+// by the tcgen05 fences around it, so the arrive carries no release: that would first
+// wait for every global store this warp has in flight (the output rows it has just written).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // tiled load into this CTA's shared memory, completion counted on a barrier given by its
 // shared::cluster address (the leader's)
@@ -246,8 +247,6 @@ gate_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
     const int ew = warp - 2;
     const int q = warp & 3;
     const int part = ew >> 2;
-    unsigned char* stg = smem + kStgOff + ew * kStgWarpBytes;       // 32 rows x 128 B staging
-    unsigned char* srow = stg + lane * kStgRowBytes;
     float* xslot = reinterpret_cast<float*>(smem + kXchgOff) + ((q * 3 + (part > 0 ? part - 1 : 0)) * 32 + lane) * 6;
     int acc = 0; uint32_t acc_phase = 0, x_phase = 0;
     const float ninf = __int_as_float(0xff800000);
@@ -306,26 +305,17 @@ gate_fused2_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_const
               a1[k] = gt1 ? v[i] : a1[k];
               j1[k] = gt1 ? hh * 32 + i : j1[k];
             }
-            // logits: stage the 32 fp32 of this row (one 128-byte staging row, XOR-swizzled pieces),
-            // then write 128-byte row segments: 8 lanes per row, 4 rows per instruction
+            // logits, in 16-byte granules of four experts laid out [E/4][N]: the 32 lanes (32
+            // consecutive tokens) of one store instruction write 512 contiguous bytes, so the rows
+            // need no staging in shared memory (whose bandwidth the MMA operand reads and the TMA
+            // writes already use up); the column-sum pass reads the same layout
+            if (row_ok) {
+              float4* dst = reinterpret_cast<float4*>(p.logits) + (long long)(col0 >> 2) * p.N + row;
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-              *reinterpret_cast<float4*>(srow + ((i ^ (lane & 7)) * 16)) =
-                  make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-            __syncwarp();
-            {
-              const int piece = lane & 7;
-              const int col = col0 + piece * 4;
-#pragma unroll
-              for (int i = 0; i < 8; ++i) {
-                const int rr = 4 * i + (lane >> 3);
-                if (row0 + rr < p.N && col < p.E) {
-                  const float4 val = *reinterpret_cast<const float4*>(stg + rr * kStgRowBytes + ((piece ^ (rr & 7)) * 16));
-                  __stcs(reinterpret_cast<float4*>(p.logits + (row0 + rr) * p.E + col), val);
-                }
-              }
+              for (int i = 0; i < 8; ++i)
+                if (col0 + 4 * i < p.E)
+                  __stcs(dst + (long long)i * p.N, make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
             }
-            __syncwarp();
           }
         }
         ptx::tc_fence_before_sync();

@@ -18,6 +18,9 @@ int launch_gate_cluster(const Dims& d, const void* x, const void* wg, int32_t* e
                         float* rowmax, float* rowinv, float* partial32, int* status, cudaStream_t st);
 // gate.cu: m[g,e] = (1/S) * sum of the group's `blocks_per_group` partial rows, in order.
 void launch_gate_mean_blocks(const Dims& d, const float* partial, int blocks_per_group, float* m, cudaStream_t st);
+// gate.cu: the mean-gate pass over logits stored as float4 [E/4][N] (what gate_fused2 writes).
+void launch_gate_means_t(const Dims& d, const float* logits_t, const float* rowmax, const float* rowinv,
+                         float* partial, float* m, cudaStream_t st);
 // gate_fused2.cu: the same gating kernel on CTA pairs (tcgen05 cta_group::2, half of the wg tile per CTA).
 bool gate_fused2_supported(const Dims& d);
 int launch_gate_fused2(const Dims& d, const void* x, const void* wg, float* logits, int32_t* expert_idx,

@@ -77,8 +77,11 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// Arrive on a barrier of the peer CTA.  What the barrier hands over is a TMEM accumulator, ordered
+// by the tcgen05 fences around it, so the arrive carries no release: that would first
+// wait for every global store this warp has in flight (the output rows it has just written).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // tiled load into this CTA's shared memory, completion counted on a barrier given by its
 // shared::cluster address (the leader's); not multicast

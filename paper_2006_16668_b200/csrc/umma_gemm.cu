@@ -178,7 +178,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       epilogue_tile<BN, MASK>(p, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, mreg);
       ptx::tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
+      if (lane == 0) ptx::mbar_arrive_relaxed(acc_empty + acc);
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }
@@ -340,7 +340,7 @@ umma_gemm_resident_b_kernel(const __grid_constant__ CUtensorMap map_a, const __g
         epilogue_tile<BN, false>(p, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, nullptr);
         ptx::tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(acc_empty + acc);
+        if (lane == 0) ptx::mbar_arrive_relaxed(acc_empty + acc);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }

@@ -164,7 +164,7 @@ def test_expert_ffn_against_oracle(E, G, C, M, H, dtype, flags):
 
 
 CL = B.GSHARD_FLAG_GATE_CLUSTER
-TS = B.GSHARD_FLAG_GATE_TWO_SM
+OS = B.GSHARD_FLAG_GATE_ONE_SM
 GATE_CASES = [
     # G, S, M, E, flags    (cluster size of the fused gating kernel = ceil(E / 256))
     (2, 64, 128, 16, CL),                             # one CTA, a single 16-expert column tile
@@ -175,12 +175,14 @@ GATE_CASES = [
     (2, 128, 192, 1280, CL),                          # five CTAs
     (5, 544, 128, 2048, CL),                          # eight CTAs, more row tiles than clusters can hold at once
     (2, 100, 128, 512, CL),                           # S not a multiple of 32: the stored-logits form is chosen
-    (2, 256, 128, 2048, 0),                           # default: stored logits + column-sum pass
+    # default: stored logits + column-sum pass; on CTA pairs where E % 128 == 0
+    (2, 256, 128, 2048, 0),                           # eight column tiles
+    (3, 160, 1024, 128, 0),                           # one 128-expert tile, full contraction depth
+    (1, 352, 192, 384, 0),                            # three row tiles: the last pair has an idle CTA; ragged second column tile
+    (2, 100, 128, 272, 0),                            # E not a multiple of 128: the one-SM kernel is chosen
     (3, 96, 1024, 272, 0),
-    (2, 256, 128, 2048, TS),                          # CTA pairs, eight column tiles
-    (3, 160, 1024, 128, TS),                          # CTA pairs, one 128-expert tile; 480 tokens: odd number of row tiles... (4 tiles) 
-    (1, 352, 192, 384, TS),                           # three row tiles: the last pair has an idle CTA; ragged second column tile
-    (2, 100, 128, 272, TS),                           # E not a multiple of 128: the one-SM kernel is chosen
+    (2, 256, 128, 2048, OS),                          # single CTAs forced
+    (2, 200, 128, 384, OS),
 ]
 
 
