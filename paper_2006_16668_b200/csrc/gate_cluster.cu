@@ -60,22 +60,6 @@ struct ClusterGateParams {
   int* status;
 };
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
 __device__ __forceinline__ void st_remote_f2(uint32_t cluster_addr, float a, float b) {
   asm volatile("st.shared::cluster.v2.f32 [%0], {%1, %2};" ::"r"(cluster_addr), "f"(a), "f"(b) : "memory");
 }
@@ -179,7 +163,7 @@ gate_cluster_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
   float* pairbuf = reinterpret_cast<float*>(smem + kPairOff);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int rank = (int)cluster_ctarank();
+  const int rank = (int)ptx::cluster_ctarank();
   const int cid = blockIdx.x / p.cl;
   const int cols = cta_cols(p, rank);
 
@@ -199,7 +183,7 @@ gate_cluster_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
-  cluster_sync_all();                          // every CTA's barriers exist before any remote arrive
+  ptx::cluster_sync_all();                          // every CTA's barriers exist before any remote arrive
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -365,12 +349,12 @@ gate_cluster_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     auto publish = [&](uint32_t it1) {
       const uint32_t par = it1 & 1u;
       const uint32_t mz_addr = ptx::smem_u32(mz + ((par * kMaxCl + rank) * BM + q * 32 + lane));
-      for (int r = 0; r < p.cl; ++r) st_remote_f2(map_to_cta(mz_addr, (uint32_t)r), c_m, c_s);
+      for (int r = 0; r < p.cl; ++r) st_remote_f2(ptx::map_to_cta(mz_addr, (uint32_t)r), c_m, c_s);
       const int slot = rank * qpc + q / p.cl;
-      st_remote_u4(map_to_cta(ptx::smem_u32(t2 + ((par * 8 + slot) * 32 + lane)), (uint32_t)fin), __float_as_uint(c_v1),
+      st_remote_u4(ptx::map_to_cta(ptx::smem_u32(t2 + ((par * 8 + slot) * 32 + lane)), (uint32_t)fin), __float_as_uint(c_v1),
                    __float_as_uint(c_v2), (uint32_t)c_i1, (uint32_t)c_i2);
       __syncwarp();
-      if (lane < p.cl) mbar_arrive_remote(map_to_cta(ptx::smem_u32(stats_full + par), (uint32_t)lane));
+      if (lane < p.cl) ptx::mbar_arrive_remote_release(ptx::map_to_cta(ptx::smem_u32(stats_full + par), (uint32_t)lane));
     };
 
     // Tile loop.  Pass 1 and pass 2 of a tile run back to back (the second accumulator lets the
@@ -456,7 +440,7 @@ gate_cluster_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
   __syncwarp();
   ptx::tc_fence_before_sync();
   __syncthreads();
-  cluster_sync_all();                  // no CTA leaves while a peer may still store into its shared memory
+  ptx::cluster_sync_all();                  // no CTA leaves while a peer may still store into its shared memory
   if (warp == 1) {
     ptx::tc_fence_after_sync();
     ptx::tmem_dealloc(tmem_base, kTmemCols);

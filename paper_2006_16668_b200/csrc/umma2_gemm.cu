@@ -63,69 +63,6 @@ __device__ __forceinline__ TileCoord decode(const Params2& p, int tile) {
   return t;
 }
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-// shared::cluster address of the same shared-memory location in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t smem_addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Arrive on a barrier of the peer CTA.  What the barrier hands over is a TMEM accumulator, ordered
-// by the tcgen05 fences around it, so the arrive carries no release: that would first
-// wait for every global store this warp has in flight (the output rows it has just written).
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-// tiled load into this CTA's shared memory, completion counted on a barrier given by its
-// shared::cluster address (the leader's); not multicast
-__device__ __forceinline__ void tma_load_3d_pair(void* smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr,
-                                                 int c0, int c1, int c2, uint64_t policy) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-      " [%0], [%1, {%3, %4, %5}], [%2], %6;"
-      :
-      : "r"(ptx::smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1),
-        "r"(c2), "l"(policy)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_dst, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(ptx::smem_u32(smem_dst)),
-               "r"(ncols)
-               : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish_pair() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                               uint32_t accumulate) {
-  asm volatile(
-      "{\n\t"
-      ".reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t"
-      "}"
-      :
-      : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// arrive on the barrier at this shared-memory offset in BOTH CTAs of the pair once the MMAs issued
-// so far have completed (a tcgen05.commit, not a load)
-__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
-  asm volatile(
-      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-      ::"r"(ptx::smem_u32(bar)), "h"((uint16_t)3)
-      : "memory");
-}
 
 template <bool A_K, bool B_K, bool MASK>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -142,7 +79,7 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t rank = cluster_ctarank();          // 0 = leader
+  const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
   const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
 
   if (threadIdx.x == 0) {
@@ -154,12 +91,12 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     ptx::prefetch_tensormap(&map_b);
   }
   if (warp == 1) {
-    tmem_alloc_pair(tmem_slot, kTmemCols);
-    tmem_relinquish_pair();
+    ptx::tmem_alloc_pair(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish_pair();
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
-  cluster_sync_all();                               // barriers of both CTAs initialised before any remote use
+  ptx::cluster_sync_all();                               // barriers of both CTAs initialised before any remote use
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -178,21 +115,21 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           if (!ptx::mbar_wait(empty + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
           unsigned char* sa = smem + stage * kStageBytes;
           unsigned char* sb = sa + kABytes;
-          const uint32_t bar = map_to_cta(ptx::smem_u32(full + stage), 0);
+          const uint32_t bar = ptx::map_to_cta(ptx::smem_u32(full + stage), 0);
           if (rank == 0) ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)(2 * kStageBytes));
           if (A_K) {
-            tma_load_3d_pair(sa, &map_a, bar, kb * BK, row0, t.b, pol_a);
+            ptx::tma_load_3d_pair(sa, &map_a, bar, kb * BK, row0, t.b, pol_a);
           } else {
 #pragma unroll
             for (int j = 0; j < BM / 64; ++j)
-              tma_load_3d_pair(sa + j * kBoxBytes, &map_a, bar, row0 + j * 64, kb * BK, t.b, pol_a);
+              ptx::tma_load_3d_pair(sa + j * kBoxBytes, &map_a, bar, row0 + j * 64, kb * BK, t.b, pol_a);
           }
           if (B_K) {
-            tma_load_3d_pair(sb, &map_b, bar, kb * BK, col0, t.b, pol_b);
+            ptx::tma_load_3d_pair(sb, &map_b, bar, kb * BK, col0, t.b, pol_b);
           } else {
 #pragma unroll
             for (int j = 0; j < BNH / 64; ++j)
-              tma_load_3d_pair(sb + j * kBoxBytes, &map_b, bar, col0 + j * 64, kb * BK, t.b, pol_b);
+              ptx::tma_load_3d_pair(sb + j * kBoxBytes, &map_b, bar, col0 + j * 64, kb * BK, t.b, pol_b);
           }
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
@@ -219,13 +156,13 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                                     : ptx::make_smem_desc(sa + k * 2048, kBoxBytes, 1024);
             const uint64_t db = B_K ? ptx::make_smem_desc(sb + k * 32, 16, 1024)
                                     : ptx::make_smem_desc(sb + k * 2048, kBoxBytes, 1024);
-            umma_bf16_pair(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+            ptx::umma_bf16_pair(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          umma_commit_pair(empty + stage);             // stage free in both CTAs
+          ptx::umma_commit_pair(empty + stage);             // stage free in both CTAs
           if (++stage == kStages) { stage = 0; phase ^= 1u; }
         }
         if (!ok) break;
-        umma_commit_pair(acc_full + acc);              // accumulator complete in both CTAs
+        ptx::umma_commit_pair(acc_full + acc);              // accumulator complete in both CTAs
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
@@ -246,7 +183,7 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       epilogue_tile<BN, MASK>(p, t, tile_row0, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, mreg);
       ptx::tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(map_to_cta(ptx::smem_u32(acc_empty + acc), 0));   // the leader's barrier
+      if (lane == 0) ptx::mbar_arrive_remote_relaxed(ptx::map_to_cta(ptx::smem_u32(acc_empty + acc), 0));   // the leader's barrier
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }
@@ -261,10 +198,10 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   __syncwarp();
   ptx::tc_fence_before_sync();
   __syncthreads();
-  cluster_sync_all();                  // no CTA frees TMEM or exits while its peer may still use it
+  ptx::cluster_sync_all();                  // no CTA frees TMEM or exits while its peer may still use it
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    tmem_dealloc_pair(tmem_base, kTmemCols);
+    ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
   }
 }
 
