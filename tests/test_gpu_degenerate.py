@@ -16,11 +16,20 @@ pytestmark = pytest.mark.gpu
 PATHS = [("f32", 0), ("bf16", B.GSHARD_FLAG_SIMT_CONTRACTIONS), ("bf16", 0)]
 
 
-@pytest.mark.parametrize("dtype,flags", PATHS)
-def test_exact_ties_lowest_index_wins(dtype, flags):
+# (dtype, flags, E): the gating kernels differ in where the twin of an expert lives - the same
+# 32-column chunk (E = 32, one-SM kernel), another column part of a CTA (E = 256, CTA pairs),
+# another column tile (E = 512), another CTA of the cluster (cluster kernel)
+TIE_PATHS = [(d, f, 32) for d, f in PATHS] + [
+    ("bf16", 0, 256), ("bf16", 0, 512), ("bf16", B.GSHARD_FLAG_GATE_ONE_SM, 512),
+    ("bf16", B.GSHARD_FLAG_GATE_CLUSTER, 256), ("bf16", B.GSHARD_FLAG_GATE_CLUSTER, 1024),
+]
+
+
+@pytest.mark.parametrize("dtype,flags,E", TIE_PATHS)
+def test_exact_ties_lowest_index_wins(dtype, flags, E):
     # every expert j < E/2 has a twin j + E/2 with identical gating weights: the two largest gates
     # of every token tie exactly, so Algorithm 1's top_2 must return (j, j + E/2), w1 = w2 = 1/2.
-    cfg = MoEConfig("ties", G=2, S=192, M=64, H=64, E=32, C=12, dtype=dtype, seed=31)
+    cfg = MoEConfig("ties", G=2, S=192, M=64, H=64, E=E, C=12, dtype=dtype, seed=31)
     inp = make_inputs(cfg, "cuda")
     half = cfg.E // 2
     inp["wg"][:, half:] = inp["wg"][:, :half]
