@@ -197,6 +197,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--chained-ffn", action="store_true", help="both expert GEMMs in one launch (rows > 128)")
     ap.add_argument("--one-sm-mma", action="store_true", help="ablation: no grouped GEMM on CTA pairs")
     ap.add_argument("--gate-one-sm", action="store_true", help="ablation: gating GEMM on single CTAs, row-major logits")
     ap.add_argument("--gate-cluster", action="store_true",
@@ -238,7 +239,8 @@ def main():
                          (B.GSHARD_FLAG_GATHER_DISPATCH if args.gather_dispatch else 0) |
                          (B.GSHARD_FLAG_GATE_CLUSTER if args.gate_cluster else 0) |
                          (B.GSHARD_FLAG_GATE_ONE_SM if args.gate_one_sm else 0) |
-                         (B.GSHARD_FLAG_ONE_SM_MMA if args.one_sm_mma else 0))
+                         (B.GSHARD_FLAG_ONE_SM_MMA if args.one_sm_mma else 0) |
+                         (B.GSHARD_FLAG_CHAINED_FFN if args.chained_ffn else 0))
     ws = B.alloc_workspace(shape, host_staging=True, device=dev)
     y = torch.empty_like(inp["x"])
     l_aux = torch.zeros(1, dtype=torch.float32, device=dev)

@@ -80,6 +80,9 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                               second pass - measured faster on B200 */
 #define GSHARD_FLAG_ONE_SM_MMA 512u        /* no grouped GEMM runs on CTA pairs (128 x 256 tiles on
                                               single CTAs everywhere) */
+#define GSHARD_FLAG_CHAINED_FFN 2048u       /* experts with more than 128 rows: both expert GEMMs in one
+                                              persistent launch of CTA pairs, GEMM-2 reading the hidden
+                                              activations from L2 (they are still written once) */
 #define GSHARD_FLAG_ADD_RESIDUAL 1024u      /* forward: y = x + layer(x), the residual connection around the
                                               layer (section 2.2, expert capacity: overflowed tokens pass through it) folded
                                               into the combine; backward: dx also receives dy.  Not

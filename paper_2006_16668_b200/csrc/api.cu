@@ -103,6 +103,7 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   // more rows per expert the two grouped-GEMM launches keep the tensor pipe busier.  Not available
   // when the caller keeps h for the backward pass.
   if (ffn_runs_fused(d, keep_h)) return launch_ffn_fused(d, buf, wi, wo, fused_scratch, out, status, st, x, slot_token);
+  if (d.chained_ffn && ffn_chained_supported(d)) return launch_ffn_chained(d, buf, wi, wo, h, out, fused_scratch, status, st);
   UmmaGemm g{};
   g.A = buf; g.B = wi; g.C = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;
   g.a_kmajor = true; g.b_kmajor = false;
@@ -127,7 +128,7 @@ int validate_shape(const gshard_moe_shape* s) {
   if (!s) return GSHARD_ERR_INVALID_ARG;
   if (s->G <= 0 || s->S <= 0 || s->M <= 0 || s->H <= 0 || s->E <= 0 || s->C <= 0) return GSHARD_ERR_INVALID_ARG;
   if (s->dtype != GSHARD_F32 && s->dtype != GSHARD_BF16) return GSHARD_ERR_INVALID_ARG;
-  if (s->flags & ~2047u) return GSHARD_ERR_INVALID_ARG;
+  if (s->flags & ~4095u) return GSHARD_ERR_INVALID_ARG;
   if ((s->flags & GSHARD_FLAG_FUSED_FFN) && (s->flags & GSHARD_FLAG_UNFUSED_FFN)) return GSHARD_ERR_INVALID_ARG;
   if (s->E < 2) return GSHARD_ERR_INVALID_ARG;
   if (s->M % 8 || s->H % 8) return GSHARD_ERR_UNSUPPORTED_SHAPE;

@@ -44,6 +44,7 @@ struct Dims {
   bool fused_ffn;       // force the single-launch FFN (h handed over through L2)
   bool unfused_ffn;     // force the two grouped-GEMM launches (h through HBM)
   bool two_sm_mma;      // grouped GEMMs on CTA pairs (tcgen05 cta_group::2) where rows > 128
+  bool chained_ffn;     // more than 128 rows per expert: both GEMMs in one launch, h consumed from L2
   bool add_residual;    // y = x + layer(x); dx gains dy
   bool one_sm_mma;      // never use CTA pairs for the grouped GEMMs
   bool gate_one_sm;     // stored-logits gating kernel on single CTAs instead of CTA pairs
@@ -70,6 +71,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.gate_one_sm = (s.flags & GSHARD_FLAG_GATE_ONE_SM) != 0;
   d.one_sm_mma = (s.flags & GSHARD_FLAG_ONE_SM_MMA) != 0;
   d.add_residual = (s.flags & GSHARD_FLAG_ADD_RESIDUAL) != 0;
+  d.chained_ffn = (s.flags & GSHARD_FLAG_CHAINED_FFN) != 0;
   return d;
 }
 

@@ -16,10 +16,17 @@ struct TileCoord { int mt, nt, b; };
 
 // Writes a warp's staged 32 rows x 128 bytes to C: lane l handles 16-byte piece (l & 7) of rows
 // 4*i + (l >> 3); pieces beyond the matrix edge are skipped (cols is a multiple of the piece width).
+// Whether the output rows should be kept in L2 (they are re-read soon by the same launch).  A kernel
+// whose parameter struct wants that overloads this for its struct.
+template <typename P>
+__device__ __forceinline__ bool epi_keep_in_l2(const P&) { return false; }
+
 template <typename P>
 __device__ __forceinline__ void flush_rows(const unsigned char* stg, const P& p, int b, int row0, int col0,
                                            int lane) {
   __syncwarp();
+  const bool keep = epi_keep_in_l2(p);
+  const uint64_t pol = keep ? ptx::policy_evict_last() : 0ull;
   const int esz = p.out_f32 ? 4 : 2;
   const int piece = lane & 7;
   const int col = col0 + piece * (16 / esz);
@@ -30,7 +37,13 @@ __device__ __forceinline__ void flush_rows(const unsigned char* stg, const P& p,
     const int row = row0 + r;
     if (row < p.rows && col < p.cols) {
       const uint4 val = *reinterpret_cast<const uint4*>(stg + r * kStgRowBytes + ((piece ^ (r & 7)) * 16));
-      *reinterpret_cast<uint4*>(cbase + (long long)row * p.c_ld * esz) = val;
+      uint4* dst = reinterpret_cast<uint4*>(cbase + (long long)row * p.c_ld * esz);
+      if (keep)
+        asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(dst), "r"(val.x), "r"(val.y),
+                     "r"(val.z), "r"(val.w), "l"(pol)
+                     : "memory");
+      else
+        *dst = val;
     }
   }
   __syncwarp();

@@ -68,7 +68,7 @@ def test_workspace_sizes_for_the_paper_configs():
     (dict(C=0), B.GSHARD_ERR_INVALID_ARG), (dict(M=20), B.GSHARD_ERR_UNSUPPORTED_SHAPE),
     (dict(S=40000), B.GSHARD_ERR_UNSUPPORTED_SHAPE), (dict(E=20000), B.GSHARD_ERR_UNSUPPORTED_SHAPE),
     (dict(dtype="bf16", M=72), B.GSHARD_ERR_UNSUPPORTED_SHAPE),
-    (dict(flags=2048), B.GSHARD_ERR_INVALID_ARG),
+    (dict(flags=4096), B.GSHARD_ERR_INVALID_ARG),
     (dict(flags=B.GSHARD_FLAG_FUSED_FFN | B.GSHARD_FLAG_UNFUSED_FFN), B.GSHARD_ERR_INVALID_ARG),
 ])
 def test_bad_shapes_are_rejected(kw, code):
