@@ -80,24 +80,31 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
     const uint4* r0 = s0 >= 0 ? out + (((long long)expert_idx[2 * t] * G + g) * C + s0) * row_vec : nullptr;
     const uint4* r1 = s1 >= 0 ? out + (((long long)expert_idx[2 * t + 1] * G + g) * C + s1) * row_vec : nullptr;
     uint4* dst = y + t * row_vec;
-    for (int i = lane; i < row_vec; i += 32) {
-      float acc[n];
+    // four 16-byte pieces per lane and row at a time, every load issued before the first use (the
+    // rows are scattered in HBM)
+    for (int i0 = lane; i0 < row_vec; i0 += 128) {
+      const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+      uint4 v0[4], v1[4], vr[4];
 #pragma unroll
-      for (int j = 0; j < n; ++j) acc[j] = 0.f;
-      if (residual) Vec16<T>::load(__ldg(residual + t * row_vec + i), acc);
-      if (r0) {
-        float f[n];
-        Vec16<T>::load(__ldg(r0 + i), f);
-#pragma unroll
-        for (int j = 0; j < n; ++j) acc[j] = fmaf(w0, f[j], acc[j]);
+      for (int k = 0; k < 4; ++k) {
+        const int i = i0 + 32 * k;
+        const bool in = i < row_vec;
+        v0[k] = (r0 && in) ? __ldg(r0 + i) : z;
+        v1[k] = (r1 && in) ? __ldg(r1 + i) : z;
+        vr[k] = (residual && in) ? __ldg(residual + t * row_vec + i) : z;
       }
-      if (r1) {
-        float f[n];
-        Vec16<T>::load(__ldg(r1 + i), f);
 #pragma unroll
-        for (int j = 0; j < n; ++j) acc[j] = fmaf(w1, f[j], acc[j]);
+      for (int k = 0; k < 4; ++k) {
+        const int i = i0 + 32 * k;
+        if (i >= row_vec) break;
+        float acc[n], f0[n], f1[n];
+        Vec16<T>::load(vr[k], acc);
+        Vec16<T>::load(v0[k], f0);
+        Vec16<T>::load(v1[k], f1);
+#pragma unroll
+        for (int j = 0; j < n; ++j) acc[j] = fmaf(w1, f1[j], fmaf(w0, f0[j], acc[j]));
+        dst[i] = Vec16<T>::store(acc);
       }
-      dst[i] = Vec16<T>::store(acc);
     }
   }
 }
