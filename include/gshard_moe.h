@@ -50,47 +50,53 @@ typedef enum {
 
 typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
 
-/* flags of gshard_moe_shape */
-#define GSHARD_FLAG_SAVE_FOR_BACKWARD 1u   /* forward fills `context` for the backward call */
-#define GSHARD_FLAG_SECOND_SKIP_FREES_SLOT 2u /* other reading of Algorithm 1's second loop: a
-                                                 token that fails 2*g2 > rnd does not advance
-                                                 the counter of its second expert */
-#define GSHARD_FLAG_SIMT_CONTRACTIONS 4u   /* bf16 only: run every contraction on CUDA cores
-                                              (fp32 FMA) instead of tcgen05; for debugging */
-#define GSHARD_FLAG_FUSED_FFN 8u           /* bf16 tensor-core path: force the single-launch expert FFN
-                                              (hidden activations handed over through L2, never
-                                              written to HBM) where the shape allows it; by default
-                                              it is used when an expert has at most 128 rows */
-#define GSHARD_FLAG_UNFUSED_FFN 16u        /* force the two grouped-GEMM launches instead (hidden
-                                              activations make a round trip through HBM) */
-#define GSHARD_FLAG_TWO_SM_MMA 32u         /* every grouped GEMM with more than 128 rows per problem runs
-                                              on CTA pairs (tcgen05 cta_group::2, 256 x 256 tiles); by
-                                              default only the two forward expert GEMMs do */
-#define GSHARD_FLAG_GATHER_DISPATCH 64u    /* forward with the single-launch expert FFN: the token rows
-                                              of an expert are gathered straight from x by the slot
-                                              index list (TMA row gather) while GEMM-1 runs, and the
-                                              [E, G*C, M] dispatch buffer of Algorithm 2 is not
-                                              written; ignored where that FFN form is not in use */
-#define GSHARD_FLAG_GATE_CLUSTER 128u      /* bf16 tensor-core gating with the mean gates' partial sums
-                                              fused in: a thread-block cluster holds all E logits of a
-                                              token tile in tensor memory and exchanges the softmax
-                                              statistics through distributed shared memory, so no
-                                              logits are stored (needs E <= 2048, S % 32 == 0; elsewhere
-                                              ignored).  Default: logits stored once, column sums in a
-                                              second pass - measured faster on B200 */
-#define GSHARD_FLAG_ONE_SM_MMA 512u        /* no grouped GEMM runs on CTA pairs (128 x 256 tiles on
-                                              single CTAs everywhere) */
-#define GSHARD_FLAG_CHAINED_FFN 2048u       /* experts with more than 128 rows: both expert GEMMs in one
-                                              persistent launch of CTA pairs, GEMM-2 reading the hidden
-                                              activations from L2 (they are still written once) */
-#define GSHARD_FLAG_ADD_RESIDUAL 1024u      /* forward: y = x + layer(x), the residual connection around the
-                                              layer (section 2.2, expert capacity: overflowed tokens pass through it) folded
-                                              into the combine; backward: dx also receives dy.  Not
-                                              applied by the stage call gshard_moe_combine */
-#define GSHARD_FLAG_GATE_ONE_SM 256u       /* gating GEMM on single CTAs with row-major stored logits.  By
-                                              default, where E % 128 == 0, it runs on CTA pairs (tcgen05
-                                              cta_group::2: each CTA loads half of the wg tile) and stores
-                                              the logits in 16-byte granules laid out [E/4][N] */
+/* flags of gshard_moe_shape.  Bits 4..2048 choose between kernel forms of the bf16 tensor-core
+ * path; the defaults are the forms that measured fastest on B200, results agree within the stated
+ * tolerances whichever form runs. */
+#define GSHARD_FLAG_SAVE_FOR_BACKWARD 1u      /* forward fills `context` for the backward call */
+#define GSHARD_FLAG_SECOND_SKIP_FREES_SLOT 2u /* other reading of Algorithm 1's second loop: a token
+                                                 that fails 2*g2 > rnd does not advance the counter
+                                                 of its second expert */
+#define GSHARD_FLAG_SIMT_CONTRACTIONS 4u      /* bf16 only: run every contraction on CUDA cores (fp32
+                                                 FMA) instead of tcgen05; for debugging */
+#define GSHARD_FLAG_FUSED_FFN 8u              /* force the single-launch expert FFN (hidden activations
+                                                 handed over through L2, never written to HBM) where
+                                                 the shape allows it; by default it is used when an
+                                                 expert has at most 128 rows */
+#define GSHARD_FLAG_UNFUSED_FFN 16u           /* force the two grouped-GEMM launches instead (hidden
+                                                 activations make a round trip through HBM) */
+#define GSHARD_FLAG_TWO_SM_MMA 32u            /* every grouped GEMM with more than 128 rows per problem
+                                                 runs on CTA pairs (tcgen05 cta_group::2, 256 x 256
+                                                 tiles); by default the forward expert GEMMs and two
+                                                 of the backward ones (dh, dbuf) do */
+#define GSHARD_FLAG_GATHER_DISPATCH 64u       /* forward with the single-launch expert FFN: a warp of
+                                                 every CTA gathers the next experts' token rows from x
+                                                 by the slot index list into an L2-resident buffer while
+                                                 the GEMMs run, and the [E, G*C, M] dispatch buffer of
+                                                 Algorithm 2 is not written; ignored where that FFN
+                                                 form is not in use */
+#define GSHARD_FLAG_GATE_CLUSTER 128u         /* gating with the mean gates' partial sums fused in: a
+                                                 thread-block cluster holds all E logits of a token
+                                                 tile in tensor memory and exchanges the softmax
+                                                 statistics through distributed shared memory, so no
+                                                 logits are stored (needs E <= 2048, S % 32 == 0;
+                                                 elsewhere ignored).  Default: logits stored once,
+                                                 column sums in a second pass */
+#define GSHARD_FLAG_GATE_ONE_SM 256u          /* gating GEMM on single CTAs with row-major stored
+                                                 logits.  By default, where E % 128 == 0, it runs on CTA
+                                                 pairs (each CTA loads half of the wg tile) and stores
+                                                 the logits in 16-byte granules laid out [E/4][N] */
+#define GSHARD_FLAG_ONE_SM_MMA 512u           /* no grouped GEMM runs on CTA pairs (128 x 256 tiles on
+                                                 single CTAs everywhere) */
+#define GSHARD_FLAG_ADD_RESIDUAL 1024u        /* forward: y = x + layer(x), the residual connection
+                                                 around the layer (section 2.2, expert capacity:
+                                                 overflowed tokens pass through it) folded into the
+                                                 combine; backward: dx also receives dy.  Not applied
+                                                 by the stage call gshard_moe_combine */
+#define GSHARD_FLAG_CHAINED_FFN 2048u         /* experts with more than 128 rows: both expert GEMMs in
+                                                 one persistent launch of CTA pairs, GEMM-2 reading
+                                                 the hidden activations from L2 (they are still written
+                                                 once) */
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,
