@@ -75,9 +75,10 @@ int gate_stage(const Dims& d, const FwdPlan& pl, unsigned char* ws, const void* 
       }
       if (rc != GSHARD_ERR_UNSUPPORTED_SHAPE) return rc;
     }
-    if (!d.gate_one_sm && gate_fused2_supported(d)) {
-      // the pair kernel stores the logits as float4 [E/4][N]; its own column-sum pass follows
-      GS_TRY(launch_gate_fused2(d, x, wg, logits, expert_idx, gate12, rowmax, rowinv, status, st));
+    if (!d.gate_one_sm && gate_fused2_supported(d) &&
+        launch_gate_fused2(d, x, wg, logits, expert_idx, gate12, rowmax, rowinv, status, st) == GSHARD_OK) {
+      // the pair kernel stores the logits as float4 [E/4][N]; its own column-sum pass follows.  (If
+      // the cluster launch is refused, nothing ran and the one-SM kernel below takes over.)
       launch_gate_means_t(d, logits, rowmax, rowinv, reinterpret_cast<float*>(ws + pl.partial), m, st);
       return GSHARD_OK;
     } else

@@ -14,7 +14,10 @@ inline int run_gemm(const Dims& d, const UmmaGemm& g, int* status, cudaStream_t 
     // holds its tensor pipe near 65 %.  Callers mark the GEMMs that measured faster on pairs (the two
     // forward expert GEMMs); the flags force either form everywhere.  A single row tile would leave
     // the second CTA of a pair without rows.
-    if (g.rows > 128 && !d.one_sm_mma && (d.two_sm_mma || g.prefer_two_sm)) return launch_umma2_gemm(g, status, st);
+    if (g.rows > 128 && !d.one_sm_mma && (d.two_sm_mma || g.prefer_two_sm)) {
+      const int rc = launch_umma2_gemm(g, status, st);
+      if (rc == GSHARD_OK) return rc;       // a refused cluster launch ran nothing: single CTAs take over
+    }
     return launch_umma_gemm(g, status, st);
   }
   SimtGemm s{};
