@@ -123,6 +123,8 @@ SMALL = [
     # 160 rows per expert: expert GEMMs on CTA pairs (default) and on single CTAs
     ("bf16_two_sm_default", 2, 512, 256, 512, 16, 80, "bf16", 0),
     ("bf16_one_sm_forced", 2, 512, 256, 512, 16, 80, "bf16", B.GSHARD_FLAG_ONE_SM_MMA),
+    # far more experts than tokens per group (16 column tiles in the gating kernel, almost all experts empty)
+    ("bf16_many_experts", 2, 96, 64, 64, 4096, 1, "bf16", 0),
     # gating on clusters with the mean-gate partial sums fused in (no stored logits)
     ("bf16_gate_cluster", 2, 256, 256, 1024, 32, 16, "bf16", B.GSHARD_FLAG_GATE_CLUSTER),
     ("bf16_gate_cluster_3ctas", 2, 320, 128, 256, 640, 1, "bf16", B.GSHARD_FLAG_GATE_CLUSTER),
