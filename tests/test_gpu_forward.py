@@ -218,18 +218,19 @@ def test_expert_ffn_timing_hook():
         B._check(B.load().gshard_moe_time_expert_ffn(a.cuda_event, None), "one-sided event pair")
 
 
-FULL = [("c2_128e", [0, 9], 10), ("c3_512e_skew", [3, 15], 10), ("c4_2048e", [0, 17, 31], 10)]
+FULL = [("c2_128e", None, 3), ("c3_512e_skew", None, 3), ("c4_2048e", None, 2)]
 
 
 @pytest.mark.parametrize("name,groups,tokens", FULL, ids=[c[0] for c in FULL])
 def test_full_size_sampled(name, groups, tokens):
     """The paper-shaped configurations in the launch configuration the benchmark times:
-    routing of whole sampled groups (groups are independent), y on sampled tokens."""
+    routing of EVERY group and token (the oracle's gating and Algorithm 1 take seconds even at
+    131072 tokens), y on a few sampled tokens of every group plus tokens with dropped choices."""
     cfg = CONFIGS[name]
     inp = make_inputs(cfg, "cuda")
     y, l_aux, rt = run_forward(cfg, inp)
     rep = {}
-    check_forward(cfg, inp, y, l_aux, rt, groups, tokens, report=rep)
+    check_forward(cfg, inp, y, l_aux, rt, groups if groups is not None else range(cfg.G), tokens, report=rep)
     print(f"\n[{name}] near-tie tokens excluded: {rep['excluded']}, of which flipped: {rep['flips']}, "
           f"y rel. Frobenius error on {rep['tokens']} tokens: {rep['y_err']:.3e}")
     # properties that hold at any size
