@@ -127,13 +127,13 @@ def test_backward_training_config_sampled():
     cfg = CONFIGS["c5_512e_train"]
     inp = make_inputs(cfg, "cuda")
     rng = np.random.default_rng(11)
-    toks = sorted({(int(rng.integers(cfg.G)), int(rng.integers(cfg.S))) for _ in range(10)})
+    toks = sorted({(int(rng.integers(cfg.G)), int(rng.integers(cfg.S))) for _ in range(16)})
     y, l_aux, rt, dx, dwg, dwi, dwo = run_fwd_bwd(cfg, inp)
     ei, slot, wt = to_np(rt["expert_idx"]), to_np(rt["slot"]), to_np(rt["weight"]).astype(np.float64)
     st = to_np(rt["slot_token"])
     fc = to_np(rt["first_count"])
     wg = to_np(inp["wg"])
-    for e in (0, 300):                         # expert 0 is one of the overflowing experts
+    for e in (0, 7, 300, 511):                 # experts 0..7 overflow (all their slots filled)
         wi_e, wo_e = to_np(inp["wi"][e]), to_np(inp["wo"][e])
         rows_x, rows_dout = [], []
         for g in range(cfg.G):
