@@ -63,17 +63,6 @@ CONFIGS = {
     "c3_512e_skew": MoEConfig("c3_512e_skew", G=16, S=4096, M=1024, H=8192, E=512, C=16,
                               seed=20200633, skew=True),
     "c4_2048e": MoEConfig("c4_2048e", G=32, S=4096, M=1024, H=8192, E=2048, C=4, seed=20200634),
-    # a 64-expert slice of the MoE(2048E) layer (same per-expert shapes: 128 rows, M=1024, H=8192,
-    # C=4; 2.1 GB of expert weights) - the small case profiler captures run on
-    "p4_slice": MoEConfig("p4_slice", G=32, S=128, M=1024, H=8192, E=64, C=4, seed=20200636),
-    # the MoE(2048E) layer with a thin expert hidden dimension: gating, capacity, dispatch and combine
-    # see exactly the c4 sizes (131072 tokens, 2048 experts) while the expert weights shrink to
-    # 0.5 GB - the small case for profiler captures of those kernels
-    "p4_routing": MoEConfig("p4_routing", G=32, S=4096, M=1024, H=64, E=2048, C=4, seed=20200637),
-    # a 16-expert slice of the MoE(128E) layer (1024 rows per expert, tensor-bound expert GEMMs)
-    "p2_slice": MoEConfig("p2_slice", G=16, S=512, M=1024, H=8192, E=16, C=64, seed=20200638),
-    # a 32-expert slice of the MoE(512E) training step (256 rows per expert; 1.1 GB of expert weights)
-    "p5_slice": MoEConfig("p5_slice", G=16, S=256, M=1024, H=8192, E=32, C=16, seed=20200639, backward=True),
     # configs[4]: training step
     "c5_512e_train": MoEConfig("c5_512e_train", G=16, S=4096, M=1024, H=8192, E=512, C=16,
                                seed=20200635, backward=True),
