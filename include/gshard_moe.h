@@ -63,6 +63,11 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  handed over through L2, never written to HBM) where
                                                  the shape allows it; by default it is used when an
                                                  expert has at most 128 rows */
+/* The single-launch forms (FUSED_FFN, its GATHER_DISPATCH mode, CHAINED_FFN) are persistent grids
+ * whose CTAs wait on one another, one CTA per multiprocessor.  They are launched cooperatively: the
+ * runtime starts them only when the whole grid can be resident, so work of other streams that holds
+ * multiprocessors delays them instead of breaking them; if the runtime refuses the launch, the two
+ * grouped-GEMM launches run instead. */
 #define GSHARD_FLAG_UNFUSED_FFN 16u           /* force the two grouped-GEMM launches instead (hidden
                                                  activations make a round trip through HBM) */
 #define GSHARD_FLAG_TWO_SM_MMA 32u            /* every grouped GEMM with more than 128 rows per problem
@@ -231,8 +236,9 @@ int gshard_moe_capacity(const gshard_moe_shape* shape, const int32_t* expert_idx
  * Arguments as gshard_moe_capacity, except that there is no workspace, so routing_out and its
  * slot, weight, flags, first_count, total_count, slot_token and l_aux_group must all be given
  * (stats and l_aux stay optional).  The call allocates nothing and calls no allocating routine.
- * The first call on each device looks up the array's device address (the device must be
- * current); make that first call before any stream capture begins.  All calls on a device share
+ * Every call looks up the array's device address for the current device (the device the stream
+ * belongs to must be current); the first call on a device also loads the library's module there,
+ * so make that first call before any stream capture begins.  All calls on a device share
  * the one array: the kernel rewrites every entry it later reads, so nothing needs clearing
  * between calls, but two calls whose kernels overlap on the GPU (different streams) race on it;
  * keep them on one stream or order them yourself.  Results equal gshard_moe_capacity's. */
@@ -256,6 +262,28 @@ int gshard_moe_expert_ffn(const gshard_moe_shape* shape, const void* buf, const 
  * y[g,s,:] = sum over k in {0,1} with slot[g,s,k] >= 0 of weight[g,s,k] * out[e_k, g*C+slot, :]. */
 int gshard_moe_combine(const gshard_moe_shape* shape, const void* out, const int32_t* expert_idx,
                        const int32_t* slot, const float* weight, void* y, void* cuda_stream);
+
+/* The position-wise feed-forward sub-layer of the ordinary Transformer layers that alternate with
+ * the MoE layers (section 2.1: every other feed-forward layer is replaced by a MoE layer; the
+ * performance section times "MoE layer + adjacent Transformer layer"): y = relu(x . wi) . wo over
+ * all tokens, no bias - eq. (2) with a single expert that sees every token, run by the same two
+ * grouped tensor-core GEMMs as the expert FFN.
+ *   x, y [n_tokens, M], wi [M, H], wo [H, M]: dtype (gshard_dtype); bf16 needs M % 64 == 0 and
+ *   H % 64 == 0.  workspace: gshard_dense_ffn_workspace_bytes() bytes, 256-byte aligned; it holds a
+ *   status word (read with gshard_moe_last_device_status) and the hidden activations [n_tokens, H]. */
+size_t gshard_dense_ffn_workspace_bytes(int64_t n_tokens, int32_t M, int32_t H, int32_t dtype);
+int gshard_dense_ffn_forward(int64_t n_tokens, int32_t M, int32_t H, int32_t dtype, const void* x,
+                             const void* wi, const void* wo, void* y, void* workspace,
+                             size_t workspace_bytes, void* cuda_stream);
+
+/* Self-test of the give-up path shared by every bounded device-side wait (the paper has no
+ * counterpart; this is robustness plumbing).  Launches one small CTA that allocates tensor
+ * memory, waits on an mbarrier nothing arrives at with a limit of limit_us microseconds
+ * (1..1000), and leaves through the same teardown as the GEMM kernels: abort flag,
+ * GSHARD_ERR_TIMEOUT into the status word of `workspace` (its first word; 256-byte aligned, at
+ * least 256 bytes), tensor memory released, normal return.  gshard_moe_last_device_status then
+ * reports GSHARD_ERR_TIMEOUT and the workspace and the context remain usable. */
+int gshard_moe_debug_wait_timeout(void* workspace, uint32_t limit_us, void* cuda_stream);
 
 /* Synchronises `cuda_stream` and returns the device status word of `workspace`
  * (GSHARD_OK, GSHARD_ERR_TIMEOUT, ...) or GSHARD_ERR_CUDA if the stream reported an error. */

@@ -73,6 +73,10 @@ EXPORTS = {
     "gshard_moe_dispatch": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 4),
     "gshard_moe_expert_ffn": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 5 + [c_size_t, c_void_p]),
     "gshard_moe_combine": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6),
+    "gshard_dense_ffn_workspace_bytes": (c_size_t, [ctypes.c_int64, c_int32, c_int32, c_int32]),
+    "gshard_dense_ffn_forward": (c_int, [ctypes.c_int64, c_int32, c_int32, c_int32] + [c_void_p] * 5 +
+                                 [c_size_t, c_void_p]),
+    "gshard_moe_debug_wait_timeout": (c_int, [c_void_p, c_uint32, c_void_p]),
     "gshard_moe_last_device_status": (c_int, [c_void_p, c_void_p]),
     "gshard_moe_last_launch_count": (c_int, []),
     "gshard_moe_time_expert_ffn": (c_int, [c_void_p, c_void_p]),
@@ -254,6 +258,27 @@ def gshard_moe_expert_ffn(shape, buf, wi, wo, out, workspace, stream=None):
 def gshard_moe_combine(shape, out, expert_idx, slot, weight, y, stream=None):
     _check(load().gshard_moe_combine(ctypes.byref(shape), _p(out), _p(expert_idx), _p(slot), _p(weight), _p(y),
                                      _stream(stream)), "gshard_moe_combine")
+
+
+def _dtype_code(t) -> int:
+    return GSHARD_BF16 if t.dtype == torch.bfloat16 else GSHARD_F32
+
+
+def gshard_dense_ffn_workspace_bytes(n_tokens, M, H, dtype_code) -> int:
+    return int(load().gshard_dense_ffn_workspace_bytes(int(n_tokens), int(M), int(H), int(dtype_code)))
+
+
+def gshard_dense_ffn_forward(x, wi, wo, y, workspace, stream=None):
+    """y = relu(x . wi) . wo for x [n, M], wi [M, H], wo [H, M] (the dense Transformer FFN)."""
+    n, M = x.shape
+    H = wi.shape[1]
+    _check(load().gshard_dense_ffn_forward(n, M, H, _dtype_code(x), _p(x), _p(wi), _p(wo), _p(y), _p(workspace),
+                                           workspace.numel(), _stream(stream)), "gshard_dense_ffn_forward")
+
+
+def gshard_moe_debug_wait_timeout(workspace, limit_us=200, stream=None):
+    _check(load().gshard_moe_debug_wait_timeout(_p(workspace), int(limit_us), _stream(stream)),
+           "gshard_moe_debug_wait_timeout")
 
 
 def gshard_moe_last_device_status(workspace, stream=None) -> int:

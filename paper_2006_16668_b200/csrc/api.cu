@@ -103,8 +103,17 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   // the FFN is bound by streaming the expert weights (at most one 128-row tile per expert); with
   // more rows per expert the two grouped-GEMM launches keep the tensor pipe busier.  Not available
   // when the caller keeps h for the backward pass.
-  if (ffn_runs_fused(d, keep_h)) return launch_ffn_fused(d, buf, wi, wo, fused_scratch, out, status, st, x, slot_token);
-  if (d.chained_ffn && ffn_chained_supported(d)) return launch_ffn_chained(d, buf, wi, wo, h, out, fused_scratch, status, st);
+  // Both single-launch forms need their whole grid resident at once and are launched cooperatively;
+  // when the runtime refuses that (GSHARD_ERR_UNSUPPORTED_SHAPE, nothing launched) the two
+  // grouped-GEMM launches below take over.
+  if (ffn_runs_fused(d, keep_h)) {
+    const int rc = launch_ffn_fused(d, buf, wi, wo, fused_scratch, out, status, st, x, slot_token);
+    if (rc != GSHARD_ERR_UNSUPPORTED_SHAPE) return rc;
+    if (x) launch_dispatch(d, x, slot_token, const_cast<void*>(buf), st);   // rows were to be gathered in the launch
+  } else if (d.chained_ffn && ffn_chained_supported(d)) {
+    const int rc = launch_ffn_chained(d, buf, wi, wo, h, out, fused_scratch, status, st);
+    if (rc != GSHARD_ERR_UNSUPPORTED_SHAPE) return rc;
+  }
   UmmaGemm g{};
   g.A = buf; g.B = wi; g.C = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;
   g.a_kmajor = true; g.b_kmajor = false;
@@ -136,6 +145,14 @@ int validate_shape(const gshard_moe_shape* s) {
   if (s->S > 32767 || s->E > 16384 || s->C > 32767) return GSHARD_ERR_UNSUPPORTED_SHAPE;
   if ((long long)s->G * s->S > (1ll << 30) || (long long)s->E * s->G * s->C > (1ll << 30)) return GSHARD_ERR_UNSUPPORTED_SHAPE;
   if (capacity_warps_for(s->E) == 0) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  // grid limits of the launches: the column-sum kernels index (group, 128-token tile) and the
+  // group-level kernels the group through gridDim.y; the CUDA-core GEMM its 64-row tiles
+  if ((long long)s->G * ((s->S + kGateTile - 1) / kGateTile) > 65535) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  if (((long long)s->G * s->S + 63) / 64 > 65535 && (s->dtype == GSHARD_F32 || (s->flags & GSHARD_FLAG_SIMT_CONTRACTIONS)))
+    return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  // a tensor map's strides stay below 2^40 bytes
+  if ((long long)s->G * s->S * std::max(s->M, s->E) >= (1ll << 37)) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  if ((long long)s->G * s->C * s->H >= (1ll << 37)) return GSHARD_ERR_UNSUPPORTED_SHAPE;
   const bool umma = s->dtype == GSHARD_BF16 && !(s->flags & GSHARD_FLAG_SIMT_CONTRACTIONS);
   if (umma && (s->M % 64 || s->H % 64 || s->E % 16)) return GSHARD_ERR_UNSUPPORTED_SHAPE;
   return GSHARD_OK;
@@ -150,7 +167,7 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
   if (workspace_bytes < pl.total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   const bool save = (shape->flags & GSHARD_FLAG_SAVE_FOR_BACKWARD) != 0;
-  if (save && !context) return GSHARD_ERR_INVALID_ARG;
+  if (save && (!context || reinterpret_cast<uintptr_t>(context) % kAlign)) return GSHARD_ERR_INVALID_ARG;
   unsigned char* ctx = static_cast<unsigned char*>(context);
   const CtxPlan cp = plan_context(d);
   gshard_moe_routing r{};
@@ -198,7 +215,7 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
     for (auto& c : cps)
       if (c.dst && cudaMemcpyAsync(c.dst, c.src, c.n, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return GSHARD_ERR_CUDA;
   }
-  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
 int backward_device(const gshard_moe_shape* shape, const void* x, const void* wg, const void* wi, const void* wo,
@@ -345,7 +362,8 @@ int gshard_moe_top2_backward(const gshard_moe_shape* shape, const void* x, const
   GS_REQUIRE_PTR(x); GS_REQUIRE_PTR(wg); GS_REQUIRE_PTR(wi); GS_REQUIRE_PTR(wo); GS_REQUIRE_PTR(context);
   GS_REQUIRE_PTR(dy); GS_REQUIRE_PTR(dx); GS_REQUIRE_PTR(dwg); GS_REQUIRE_PTR(dwi); GS_REQUIRE_PTR(dwo);
   GS_REQUIRE_PTR(workspace);
-  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign || reinterpret_cast<uintptr_t>(context) % kAlign)
+    return GSHARD_ERR_INVALID_ARG;
   if (workspace_bytes < gshard_moe_top2_workspace_bytes(shape, 1)) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
   GS_TRY(check_device());
   return backward_device(shape, x, wg, wi, wo, context, dy, l_aux_weight, dx, dwg, dwi, dwo, workspace,
@@ -368,7 +386,7 @@ int gshard_moe_gate(const gshard_moe_shape* shape, const void* x, const void* wg
   if (cudaMemsetAsync(ws + pl.status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   GS_TRY(gate_stage(d, pl, ws, x, wg, expert_idx, gate12, m, reinterpret_cast<float*>(ws + pl.rowmax),
                     reinterpret_cast<float*>(ws + pl.rowinv), st));
-  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
 int gshard_moe_capacity(const gshard_moe_shape* shape, const int32_t* expert_idx, const float* gate12,
@@ -400,7 +418,7 @@ int gshard_moe_dispatch(const gshard_moe_shape* shape, const void* x, const int3
   GS_REQUIRE_PTR(x); GS_REQUIRE_PTR(slot_token); GS_REQUIRE_PTR(buf);
   GS_TRY(check_device());
   launch_dispatch(make_dims(*shape), x, slot_token, buf, static_cast<cudaStream_t>(cuda_stream));
-  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
 int gshard_moe_expert_ffn(const gshard_moe_shape* shape, const void* buf, const void* wi, const void* wo,
@@ -418,7 +436,7 @@ int gshard_moe_expert_ffn(const gshard_moe_shape* shape, const void* buf, const 
   if (cudaMemsetAsync(ws + pl.status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   GS_TRY(ffn_stage(d, buf, wi, wo, ws + pl.h, false, out, ws + pl.ffn_scratch,
                    reinterpret_cast<int*>(ws + pl.status), st));
-  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
 int gshard_moe_combine(const gshard_moe_shape* shape, const void* out, const int32_t* expert_idx,
@@ -428,7 +446,47 @@ int gshard_moe_combine(const gshard_moe_shape* shape, const void* out, const int
   GS_REQUIRE_PTR(out); GS_REQUIRE_PTR(expert_idx); GS_REQUIRE_PTR(slot); GS_REQUIRE_PTR(weight); GS_REQUIRE_PTR(y);
   GS_TRY(check_device());
   launch_combine(make_dims(*shape), out, expert_idx, slot, weight, y, static_cast<cudaStream_t>(cuda_stream));
-  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+size_t gshard_dense_ffn_workspace_bytes(int64_t n_tokens, int32_t M, int32_t H, int32_t dtype) {
+  if (n_tokens <= 0 || n_tokens > (1ll << 30) || M <= 0 || H <= 0 || M % 8 || H % 8) return 0;
+  if (dtype != GSHARD_F32 && dtype != GSHARD_BF16) return 0;
+  if (dtype == GSHARD_BF16 && (M % 64 || H % 64)) return 0;
+  if (dtype == GSHARD_F32 && (n_tokens + 63) / 64 > 65535) return 0;
+  return kAlign + align_up((size_t)n_tokens * H * (dtype == GSHARD_BF16 ? 2 : 4));
+}
+
+int gshard_dense_ffn_forward(int64_t n_tokens, int32_t M, int32_t H, int32_t dtype, const void* x, const void* wi,
+                             const void* wo, void* y, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  launch_counter().n = 0;
+  const size_t need = gshard_dense_ffn_workspace_bytes(n_tokens, M, H, dtype);
+  if (need == 0) return (n_tokens <= 0 || M <= 0 || H <= 0) ? GSHARD_ERR_INVALID_ARG : GSHARD_ERR_UNSUPPORTED_SHAPE;
+  GS_REQUIRE_PTR(x); GS_REQUIRE_PTR(wi); GS_REQUIRE_PTR(wo); GS_REQUIRE_PTR(y); GS_REQUIRE_PTR(workspace);
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  if (workspace_bytes < need) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  GS_TRY(check_device());
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  int* status = reinterpret_cast<int*>(ws);
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  // the expert FFN's two grouped GEMMs with a single problem of n_tokens rows
+  gshard_moe_shape one{};
+  one.G = 1; one.S = 1; one.C = 1; one.E = 2; one.M = M; one.H = H; one.dtype = dtype;
+  Dims d = make_dims(one);
+  d.rows = (int)n_tokens;
+  void* h = ws + kAlign;
+  UmmaGemm g{};
+  g.A = x; g.B = wi; g.C = h; g.rows = d.rows; g.cols = H; g.K = M; g.batch = 1;
+  g.a_kmajor = true; g.b_kmajor = false; g.a_ld = M; g.b_ld = H; g.c_ld = H;
+  g.relu = 1; g.a_stream = 1; g.prefer_two_sm = 1;
+  GS_TRY(run_gemm(d, g, status, st));
+  UmmaGemm g2{};
+  g2.A = h; g2.B = wo; g2.C = y; g2.rows = d.rows; g2.cols = M; g2.K = H; g2.batch = 1;
+  g2.a_kmajor = true; g2.b_kmajor = false; g2.a_ld = H; g2.b_ld = M; g2.c_ld = M;
+  g2.a_stream = 1; g2.prefer_two_sm = 1;
+  GS_TRY(run_gemm(d, g2, status, st));
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
 int gshard_moe_last_device_status(void* workspace, void* cuda_stream) {

@@ -17,41 +17,13 @@ int gate_logits(const Dims& d, const void* x, const void* wg, float* logits, int
 
 namespace {
 
-template <typename T> struct Row16;
-template <> struct Row16<float> {
-  static constexpr int n = 4;
-  __device__ static void load(const uint4& v, float* f) {
-    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
-  }
-  __device__ static uint4 store(const float* f) {
-    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
-  }
-};
-template <> struct Row16<__nv_bfloat16> {
-  static constexpr int n = 8;
-  __device__ static void load(const uint4& v, float* f) {
-    const unsigned w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) { f[2 * i] = __uint_as_float(w[i] << 16); f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
-  }
-  __device__ static uint4 store(const float* f) {
-    unsigned w[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-      w[i] = *reinterpret_cast<const unsigned*>(&p);
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
-  }
-};
-
 // dw[t,k] = <dy[t,:], out[e_k, g*C+slot_k, :]> for kept choices, else 0.  One warp per token.
 template <typename T>
 __global__ void __launch_bounds__(256) combine_bwd_kernel(const uint4* __restrict__ dy, const uint4* __restrict__ out,
                                                           const int32_t* __restrict__ expert_idx,
                                                           const int32_t* __restrict__ slot, float* __restrict__ dw,
                                                           long long N, int G, int S, int C, int row_vec) {
-  constexpr int n = Row16<T>::n;
+  constexpr int n = Vec16<T>::n;
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -66,8 +38,8 @@ __global__ void __launch_bounds__(256) combine_bwd_kernel(const uint4* __restric
       const uint4* dyr = dy + t * row_vec;
       for (int i = lane; i < row_vec; i += 32) {
         float a[n], b[n];
-        Row16<T>::load(__ldg(r + i), a);
-        Row16<T>::load(__ldg(dyr + i), b);
+        Vec16<T>::load(__ldg(r + i), a);
+        Vec16<T>::load(__ldg(dyr + i), b);
 #pragma unroll
         for (int j = 0; j < n; ++j) acc[k] = fmaf(a[j], b[j], acc[k]);
       }
@@ -88,7 +60,7 @@ __global__ void __launch_bounds__(256) dout_kernel(const uint4* __restrict__ dy,
                                                    const int32_t* __restrict__ slot, const float* __restrict__ weight,
                                                    uint4* __restrict__ dout, long long R, int G, int S, int C,
                                                    int row_vec) {
-  constexpr int n = Row16<T>::n;
+  constexpr int n = Vec16<T>::n;
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -108,10 +80,10 @@ __global__ void __launch_bounds__(256) dout_kernel(const uint4* __restrict__ dy,
     const uint4* src = dy + t * row_vec;
     for (int i = lane; i < row_vec; i += 32) {
       float f[n];
-      Row16<T>::load(__ldg(src + i), f);
+      Vec16<T>::load(__ldg(src + i), f);
 #pragma unroll
       for (int j = 0; j < n; ++j) f[j] *= w;
-      dst[i] = Row16<T>::store(f);
+      dst[i] = Vec16<T>::store(f);
     }
   }
 }
@@ -162,7 +134,7 @@ __global__ void __launch_bounds__(256) dx_kernel(const float4* __restrict__ dxg,
                                                  const int32_t* __restrict__ expert_idx, const int32_t* __restrict__ slot,
                                                  const uint4* __restrict__ dy_res, uint4* __restrict__ dx, long long N,
                                                  int G, int S, int C, int row_vec) {
-  constexpr int n = Row16<T>::n;
+  constexpr int n = Vec16<T>::n;
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
@@ -186,17 +158,17 @@ __global__ void __launch_bounds__(256) dx_kernel(const float4* __restrict__ dxg,
       for (int k = 0; k < 2; ++k) {
         if (!r[k]) continue;
         float f[n];
-        Row16<T>::load(__ldg(r[k] + i), f);
+        Vec16<T>::load(__ldg(r[k] + i), f);
 #pragma unroll
         for (int j = 0; j < n; ++j) acc[j] += f[j];
       }
       if (dy_res) {                                  // residual connection: dx also receives dy
         float f[n];
-        Row16<T>::load(__ldg(dy_res + t * row_vec + i), f);
+        Vec16<T>::load(__ldg(dy_res + t * row_vec + i), f);
 #pragma unroll
         for (int j = 0; j < n; ++j) acc[j] += f[j];
       }
-      dx[t * row_vec + i] = Row16<T>::store(acc);
+      dx[t * row_vec + i] = Vec16<T>::store(acc);
     }
   }
 }
@@ -212,12 +184,6 @@ __global__ void __launch_bounds__(256) sum_partials_kernel(const float4* __restr
     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
   }
   out[i] = acc;
-}
-
-int grid_rows(long long rows) {
-  long long blocks = (rows + 7) / 8;
-  const long long cap = 148LL * 32;
-  return (int)(blocks < cap ? (blocks > 0 ? blocks : 1) : cap);
 }
 
 template <typename T>
@@ -250,10 +216,10 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   const long long rows = d.rows;
 
   // combine backward
-  combine_bwd_kernel<T><<<grid_rows(d.N), 256, 0, st>>>(reinterpret_cast<const uint4*>(dy),
+  combine_bwd_kernel<T><<<grid_for_rows(d.N), 256, 0, st>>>(reinterpret_cast<const uint4*>(dy),
                                                         reinterpret_cast<const uint4*>(out), expert_idx, slot, dw, d.N,
                                                         d.G, d.S, d.C, row_vec);
-  dout_kernel<T><<<grid_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(dy), slot_token, expert_idx, slot,
+  dout_kernel<T><<<grid_for_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(dy), slot_token, expert_idx, slot,
                                                  weight, reinterpret_cast<uint4*>(dout), d.R, d.G, d.S, d.C, row_vec);
   count_launch(2);
   launch_dispatch(d, x, slot_token, buf, st);
@@ -294,7 +260,7 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   rc = gate_logits(d, x, wg, logits, status, st);
   if (rc) return rc;
   const float aux_coef = k_aux / ((float)d.G * (float)d.E * (float)d.S * (float)d.S);
-  gate_bwd_kernel<T><<<grid_rows(d.N), 256, 0, st>>>(logits, rowmax, rowinv, expert_idx, gate12, dw, first_count,
+  gate_bwd_kernel<T><<<grid_for_rows(d.N), 256, 0, st>>>(logits, rowmax, rowinv, expert_idx, gate12, dw, first_count,
                                                      aux_coef, dlogits, d.N, d.S, d.E);
   count_launch();
   // dwg = x^T . dlogits   [M x E] fp32
@@ -307,7 +273,7 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   int splits = 1;
   if (!d.simt) {
     const long long tiles = (long long)ceil_div(d.M, 128) * ceil_div(d.E, d.E > 128 ? 256 : 128);
-    for (int sp = (int)(148 / tiles); sp > 1; --sp)
+    for (int sp = (int)(device_sms() / tiles); sp > 1; --sp)
       if (d.N % ((long long)sp * 64) == 0 && (long long)sp * d.E <= d.N && ((long long)d.M * d.E) % 4 == 0) {
         splits = sp;
         break;
@@ -332,7 +298,7 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   g.a_kmajor = true; g.b_kmajor = true; g.a_ld = d.E; g.b_ld = d.E; g.c_ld = d.M; g.out_f32 = 1;
   rc = run_gemm(d, g, status, st);
   if (rc) return rc;
-  dx_kernel<T><<<grid_rows(d.N), 256, 0, st>>>(reinterpret_cast<const float4*>(dxg), reinterpret_cast<const uint4*>(dbuf),
+  dx_kernel<T><<<grid_for_rows(d.N), 256, 0, st>>>(reinterpret_cast<const float4*>(dxg), reinterpret_cast<const uint4*>(dbuf),
                                                expert_idx, slot,
                                                d.add_residual ? reinterpret_cast<const uint4*>(dy) : nullptr,
                                                reinterpret_cast<uint4*>(dx), d.N, d.G, d.S, d.C, row_vec);

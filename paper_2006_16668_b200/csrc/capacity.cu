@@ -242,23 +242,16 @@ static __device__ __align__(256) int32_t g_static_stats_group[kStaticMaxGroups *
 
 namespace {
 // In host code the array's name above is only a host-side stand-in, not a device address; the
-// address a kernel can use comes from cudaGetSymbolAddress, asked once per device with that
-// device current.
+// address a kernel can use comes from cudaGetSymbolAddress with the target device current.  It is
+// asked on every call: the lookup allocates nothing once the library's module is loaded on the
+// device (the first call loads it), and a cached pointer would dangle after a device reset.
 int static_scratch_for_current_device(int32_t** out) {
-  constexpr int kMaxDevices = 64;
-  static int32_t* ptrs[kMaxDevices] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return GSHARD_ERR_CUDA; }
-  if (dev < 0 || dev >= kMaxDevices) return GSHARD_ERR_INTERNAL;
-  if (ptrs[dev] == nullptr) {
-    int32_t* p = nullptr;
-    if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_stats_group) != cudaSuccess || p == nullptr) {
-      cudaGetLastError();
-      return GSHARD_ERR_CUDA;
-    }
-    ptrs[dev] = p;     // same value whichever thread stores it
+  int32_t* p = nullptr;
+  if (cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_static_stats_group) != cudaSuccess || p == nullptr) {
+    cudaGetLastError();
+    return GSHARD_ERR_CUDA;
   }
-  *out = ptrs[dev];
+  *out = p;
   return GSHARD_OK;
 }
 }  // namespace

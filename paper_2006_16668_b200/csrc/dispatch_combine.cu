@@ -6,7 +6,9 @@
 
 namespace gshard {
 
-// buf[e, g*C + c, :] = x[g, slot_token[e,g,c], :]  or zeros for an empty slot.
+// buf[e, g*C + c, :] = x[g, slot_token[e,g,c], :]  or zeros for an empty slot.  The index list may
+// come straight from a caller (stage entry point): a token index outside [0, S) is treated as an
+// empty slot instead of being used as an address.
 __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__ x,
                                                        const int32_t* __restrict__ slot_token,
                                                        uint4* __restrict__ buf, long long R, int G,
@@ -18,7 +20,7 @@ __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__
     const int tok = slot_token[r];                       // r = (e*G + g)*C + c
     const int g = (int)((r / C) % G);
     uint4* dst = buf + r * row_vec;
-    if (tok >= 0) {
+    if (tok >= 0 && tok < S) {
       const uint4* src = x + ((long long)g * S + tok) * row_vec;
       for (int i = lane; i < row_vec; i += 32) dst[i] = __ldg(src + i);
     } else {
@@ -28,39 +30,10 @@ __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__
   }
 }
 
-template <typename T> struct Vec16;
-template <> struct Vec16<float> {
-  static constexpr int n = 4;
-  __device__ static void load(const uint4& v, float* f) {
-    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
-  }
-  __device__ static uint4 store(const float* f) {
-    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
-  }
-};
-template <> struct Vec16<__nv_bfloat16> {
-  static constexpr int n = 8;
-  __device__ static void load(const uint4& v, float* f) {
-    const unsigned w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      f[2 * i] = __uint_as_float(w[i] << 16);
-      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-  }
-  __device__ static uint4 store(const float* f) {
-    unsigned w[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const __nv_bfloat162 p = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
-      w[i] = *reinterpret_cast<const unsigned*>(&p);
-    }
-    return make_uint4(w[0], w[1], w[2], w[3]);
-  }
-};
-
 // y[t,:] = w0*out[e0, g*C+slot0, :] + w1*out[e1, g*C+slot1, :] over the kept choices, fp32 FMA;
-// with `residual` the token's input row is added (the residual connection around the layer).
+// with `residual` the token's input row is added (the residual connection around the layer).  A
+// choice whose expert id is outside [0, E) or whose slot is outside [0, C) contributes nothing (the
+// stage entry point takes these tensors from the caller; they are checked, not trusted).
 template <typename T>
 __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ out,
                                                       const int32_t* __restrict__ expert_idx,
@@ -68,7 +41,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
                                                       const float* __restrict__ weight,
                                                       const uint4* __restrict__ residual,
                                                       uint4* __restrict__ y, long long N, int G, int S,
-                                                      int C, int row_vec) {
+                                                      int C, int E, int row_vec) {
   constexpr int n = Vec16<T>::n;
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -77,8 +50,10 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
     const int g = (int)(t / S);
     const int s0 = slot[2 * t], s1 = slot[2 * t + 1];
     const float w0 = weight[2 * t], w1 = weight[2 * t + 1];
-    const uint4* r0 = s0 >= 0 ? out + (((long long)expert_idx[2 * t] * G + g) * C + s0) * row_vec : nullptr;
-    const uint4* r1 = s1 >= 0 ? out + (((long long)expert_idx[2 * t + 1] * G + g) * C + s1) * row_vec : nullptr;
+    const int x0 = expert_idx[2 * t], x1 = expert_idx[2 * t + 1];
+    const bool k0 = s0 >= 0 && s0 < C && x0 >= 0 && x0 < E, k1 = s1 >= 0 && s1 < C && x1 >= 0 && x1 < E;
+    const uint4* r0 = k0 ? out + (((long long)x0 * G + g) * C + s0) * row_vec : nullptr;
+    const uint4* r1 = k1 ? out + (((long long)x1 * G + g) * C + s1) * row_vec : nullptr;
     uint4* dst = y + t * row_vec;
     // four 16-byte pieces per lane and row at a time, every load issued before the first use (the
     // rows are scattered in HBM)
@@ -109,12 +84,6 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
   }
 }
 
-static int grid_for_rows(long long rows) {
-  long long blocks = (rows + 7) / 8;
-  const long long cap = 148LL * 32;
-  return (int)(blocks < cap ? (blocks > 0 ? blocks : 1) : cap);
-}
-
 void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st) {
   const int row_vec = (int)((size_t)d.M * d.esize / 16);
   dispatch_kernel<<<grid_for_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(x), slot_token,
@@ -128,11 +97,11 @@ void launch_combine(const Dims& d, const void* out, const int32_t* expert_idx, c
   if (d.bf16)
     combine_kernel<__nv_bfloat16><<<grid_for_rows(d.N), 256, 0, st>>>(
         reinterpret_cast<const uint4*>(out), expert_idx, slot, weight, reinterpret_cast<const uint4*>(residual),
-        reinterpret_cast<uint4*>(y), d.N, d.G, d.S, d.C, row_vec);
+        reinterpret_cast<uint4*>(y), d.N, d.G, d.S, d.C, d.E, row_vec);
   else
     combine_kernel<float><<<grid_for_rows(d.N), 256, 0, st>>>(
         reinterpret_cast<const uint4*>(out), expert_idx, slot, weight, reinterpret_cast<const uint4*>(residual),
-        reinterpret_cast<uint4*>(y), d.N, d.G, d.S, d.C, row_vec);
+        reinterpret_cast<uint4*>(y), d.N, d.G, d.S, d.C, d.E, row_vec);
   count_launch();
 }
 

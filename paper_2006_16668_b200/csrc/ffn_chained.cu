@@ -315,8 +315,7 @@ int launch_ffn_chained(const Dims& d, const void* buf, const void* wi, const voi
   okm = okm && make_map(&m_h, h, d.H, rows, d.E, d.H, rows * d.H, BK, BM);
   okm = okm && make_map(&m_wo, wo, d.M, d.H, d.E, d.M, (long long)d.H * d.M, 64, BK);
   if (!okm) return GSHARD_ERR_CUDA;
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = device_sms();
   long long pairs = sms / 2;
   if (pairs > p.total_items) pairs = p.total_items;
   if (cudaFuncSetAttribute(ffn_chained_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
@@ -326,16 +325,21 @@ int launch_ffn_chained(const Dims& d, const void* buf, const void* wi, const voi
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = kSmemBytes;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  // GEMM-2 items wait for GEMM-1 items of other pairs: cooperative launch, so that the runtime
+  // guarantees the whole grid is resident at once (a refusal launches nothing; the caller then
+  // runs the two grouped-GEMM launches).
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeCooperative;
+  attr[1].val.cooperative = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   if (cudaLaunchKernelEx(&cfg, ffn_chained_kernel, m_buf, m_wi, m_h, m_wo, p) != cudaSuccess) {
     cudaGetLastError();
-    return GSHARD_ERR_CUDA;
+    return GSHARD_ERR_UNSUPPORTED_SHAPE;
   }
   count_launch();
   return GSHARD_OK;

@@ -31,8 +31,8 @@
 //                    slot of unit i is overwritten for unit i + 2 only after prod[] shows that all
 //                    four ranks finished every GEMM-1 of unit i.  The [E, G*C, M] dispatch buffer
 //                    is then neither written nor read.
-// All CTAs are co-resident (grid <= SM count, one CTA per SM) and every wait is bounded in wall
-// time, reporting GSHARD_ERR_TIMEOUT through the status word instead of hanging.
+// All CTAs are co-resident (grid <= SM count, one CTA per SM, cooperative launch) and every wait is
+// bounded in wall time, reporting GSHARD_ERR_TIMEOUT through the status word instead of hanging.
 #include <cuda.h>
 
 #include "kernels.cuh"
@@ -433,12 +433,6 @@ ffn_group4_kernel(const __grid_constant__ CUtensorMap map_buf, const __grid_cons
   }
 }
 
-int device_sms() {
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  return sms;
-}
-
 }  // namespace
 
 // Shapes the four-CTA kernel handles: the output columns split evenly over four ranks with at most
@@ -489,9 +483,27 @@ int launch_ffn_fused(const Dims& d, const void* buf, const void* wi, const void*
   if (!okm) return GSHARD_ERR_CUDA;
   if (cudaFuncSetAttribute(ffn_group4_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
     return GSHARD_ERR_CUDA;
-  ffn_group4_kernel<<<p.groups * kGroup, kThreads, kSmemBytes, st>>>(m_buf, m_wi, m_hs, m_wo, p);
+  // The four CTAs of a group wait on one another's counters, so every CTA of the grid must be
+  // resident at once.  A cooperative launch makes the runtime guarantee that: it starts the grid
+  // only when all of it fits beside whatever else the process is running, and refuses a grid that
+  // can never fit.  A refusal launches nothing and is reported as "unsupported" so that the caller
+  // falls back to the two grouped-GEMM launches.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(p.groups * kGroup), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = kSmemBytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, ffn_group4_kernel, m_buf, m_wi, m_hs, m_wo, p) != cudaSuccess) {
+    cudaGetLastError();
+    return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  }
   count_launch();
-  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+  return GSHARD_OK;
 }
 
 }  // namespace gshard

@@ -218,7 +218,8 @@ void launch_gate_rows(const Dims& d, const float* logits, int32_t* expert_idx, f
                       float* rowmax, float* rowinv, cudaStream_t st) {
   const long long warps_needed = d.N;
   int blocks = (int)((warps_needed + 7) / 8);
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  const long long cap = (long long)device_sms() * 16;
+  if (blocks > cap) blocks = (int)cap;
   gate_rows_kernel<<<blocks, 256, 0, st>>>(logits, d.N, d.E, expert_idx, gate12, rowmax, rowinv);
   count_launch();
 }

@@ -484,8 +484,7 @@ int launch_gate_cluster(const Dims& d, const void* x, const void* wg, int32_t* e
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   // every cluster of the grid must be resident at once (persistent tiles, peers wait on each other)
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = device_sms();
   cfg.gridDim = dim3((unsigned)(sms / p.cl * p.cl), 1, 1);
   int max_clusters = 0;
   if (cudaOccupancyMaxActiveClusters(&max_clusters, gate_cluster_kernel, &cfg) != cudaSuccess || max_clusters < 1) {

@@ -340,8 +340,7 @@ int launch_gate_fused(const Dims& d, const void* x, const void* wg, float* logit
   bool okm = make_map(&mx, x, d.M, d.N, 1, d.M, 0, BK, BM);
   okm = okm && make_map(&mw, wg, d.E, d.M, 1, d.E, 0, 64, BK);
   if (!okm) return GSHARD_ERR_CUDA;
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = device_sms();
   const int grid = p.row_tiles < sms ? p.row_tiles : sms;
   if (cudaFuncSetAttribute(gate_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
     return GSHARD_ERR_CUDA;

@@ -342,8 +342,7 @@ int launch_gate_fused2(const Dims& d, const void* x, const void* wg, float* logi
   bool okm = make_map(&mx, x, d.M, d.N, 1, d.M, 0, BK, BM);
   okm = okm && make_map(&mw, wg, d.E, d.M, 1, d.E, 0, 64, BK);
   if (!okm) return GSHARD_ERR_CUDA;
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = device_sms();
   const int pair_tiles = (p.row_tiles + 1) / 2;
   const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
   if (cudaFuncSetAttribute(gate_fused2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)

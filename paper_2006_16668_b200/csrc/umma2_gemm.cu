@@ -250,8 +250,7 @@ int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   p.out_f32 = g.out_f32; p.relu = g.relu; p.a_stream = g.a_stream; p.b_stream = g.b_stream;
   p.n_fastest = (g.rows > g.cols) ? 1 : 0;
   p.status = status;
-  int sms = 148, dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = device_sms();
   int pairs = sms / 2;
   if (pairs > p.total_tiles) pairs = p.total_tiles;
 #define GSHARD_DISPATCH2(AK, BKM) \

@@ -396,9 +396,7 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   // stream the larger operand once: walk the tiles that share it back to back
   p.n_fastest = (g.rows > g.cols) ? 1 : 0;
   p.status = status;
-  int sms = 148;
-  int dev = 0;
-  if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = device_sms();
   if (!g.a_kmajor && !g.b_kmajor && !g.mask && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
     // short contraction, several row tiles per column block: keep the B tile resident
     const int n_groups = p.n_tiles * g.batch;

@@ -69,6 +69,8 @@ def test_workspace_sizes_for_the_paper_configs():
     (dict(S=40000), B.GSHARD_ERR_UNSUPPORTED_SHAPE), (dict(E=20000), B.GSHARD_ERR_UNSUPPORTED_SHAPE),
     (dict(dtype="bf16", M=72), B.GSHARD_ERR_UNSUPPORTED_SHAPE),
     (dict(flags=4096), B.GSHARD_ERR_INVALID_ARG),
+    # more (group, 128-token tile) pairs, or 64-row tiles of the CUDA-core GEMM, than a grid's y extent
+    (dict(G=70000, S=1), B.GSHARD_ERR_UNSUPPORTED_SHAPE), (dict(G=600, S=16384), B.GSHARD_ERR_UNSUPPORTED_SHAPE),
     (dict(flags=B.GSHARD_FLAG_FUSED_FFN | B.GSHARD_FLAG_UNFUSED_FFN), B.GSHARD_ERR_INVALID_ARG),
 ])
 def test_bad_shapes_are_rejected(kw, code):
@@ -98,8 +100,10 @@ def test_bad_pointers_and_short_workspace():
     assert f(ctypes.byref(shape), *misaligned, None, None, fake, need, None) == B.GSHARD_ERR_INVALID_ARG
     assert f(ctypes.byref(shape), *args, None, None, fake + 16, need, None) == B.GSHARD_ERR_INVALID_ARG
     assert f(None, *args, None, None, fake, need, None) == B.GSHARD_ERR_INVALID_ARG
-    # save-for-backward without a context buffer
+    # save-for-backward without a context buffer, or with one that is not 256-byte aligned
     shape_s = B.make_shape(CONFIGS["c1_tiny"], flags=B.GSHARD_FLAG_SAVE_FOR_BACKWARD)
+    assert B.load().gshard_moe_top2_backward(ctypes.byref(shape_s), *([fake] * 4), fake + 16, fake, 0.01,
+                                             *([fake] * 5), 1 << 40, None) == B.GSHARD_ERR_INVALID_ARG
     if not torch.cuda.is_available():
         # with valid arguments the next check is the device: no GPU here, nothing is launched
         assert f(ctypes.byref(shape), *args, None, None, fake, need, None) in (B.GSHARD_ERR_CUDA, B.GSHARD_ERR_ARCH)

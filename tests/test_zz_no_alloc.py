@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import gshard_oracle as orc
 from paper_2006_16668_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
@@ -52,6 +53,30 @@ def test_static_capacity_matches_workspace_capacity_twice():
             torch.testing.assert_close(got[k], ref[k], rtol=1e-5, atol=0)
         torch.testing.assert_close(got_aux, ref_aux, rtol=1e-5, atol=0)
         assert int(got["stats"][4]) == int((got["slot"] >= 0).sum()) > 0
+
+
+def test_static_capacity_against_the_oracle_at_the_largest_group_count():
+    """G = 4096 fills the built-in scratch to its last entry; a sample of groups, the first and the
+    last among them, is compared with the oracle's two token loops (Algorithm 1) directly."""
+    G, S, E, C = 4096, 48, 12, 5
+    shape = B.make_shape(G=G, S=S, M=8, H=8, E=E, C=C, dtype="f32")
+    ei, g12, u, m = _inputs(G, S, E, 303)
+    got, got_aux = _run(shape, (ei, g12, u, m), static=True)
+    e_np, g_np, u_np, m_np = (t.cpu().numpy() for t in (ei, g12, u, m))
+    for g in (0, 1, 2047, 4094, 4095):
+        ga, gb = g_np[g, :, 0], g_np[g, :, 1]
+        w2 = gb.astype(np.float64) / (ga.astype(np.float64) + gb.astype(np.float64))
+        flags = got["flags"][g].cpu().numpy()
+        near = np.abs(2 * w2 - u_np[g]) < 1e-6       # decided in fp32 on the GPU: taken over in the replay
+        override = np.where(near, ((flags & 2) != 0).astype(np.int8), np.int8(-1)).astype(np.int8)
+        r = orc.capacity(E, C, e_np[g, :, 0], e_np[g, :, 1], ga, gb, u_np[g], m_np[g], pass_override=override)
+        assert np.array_equal(got["slot"][g].cpu().numpy(), r.slot)
+        assert np.array_equal(flags, r.flags)
+        assert np.array_equal(got["first_count"][g].cpu().numpy(), r.first_count)
+        assert np.array_equal(got["total_count"][g].cpu().numpy(), r.total_count)
+        assert float(got["l_aux_group"][g]) == pytest.approx(r.l_aux, rel=1e-5)
+    assert int(got["stats"][4]) == int((got["slot"] >= 0).sum())
+    assert float(got_aux) == pytest.approx(float(got["l_aux_group"].double().mean()), rel=1e-5)
 
 
 def test_static_capacity_rejects_what_it_cannot_hold():
