@@ -127,13 +127,22 @@ def test_backward_training_config_sampled():
     cfg = CONFIGS["c5_512e_train"]
     inp = make_inputs(cfg, "cuda")
     rng = np.random.default_rng(11)
-    toks = sorted({(int(rng.integers(cfg.G)), int(rng.integers(cfg.S))) for _ in range(16)})
+    toks = sorted({(int(rng.integers(cfg.G)), int(rng.integers(cfg.S))) for _ in range(132)})
+    assert len(toks) >= 128
     y, l_aux, rt, dx, dwg, dwi, dwo = run_fwd_bwd(cfg, inp)
+    # the forward that saves its context (two grouped-GEMM launches, h and out written into the
+    # context) must give the layer output too: routing of three groups and y on sampled tokens
+    from test_gpu_forward import check_forward
+    rep = {}
+    check_forward(cfg, inp, y, l_aux, rt, [0, 7, cfg.G - 1], 12, report=rep)
+    print(f"\n[c5 forward with saved context] y rel. Frobenius error on {rep['tokens']} tokens: {rep['y_err']:.3e}")
     ei, slot, wt = to_np(rt["expert_idx"]), to_np(rt["slot"]), to_np(rt["weight"]).astype(np.float64)
     st = to_np(rt["slot_token"])
     fc = to_np(rt["first_count"])
     wg = to_np(inp["wg"])
-    for e in (0, 7, 300, 511):                 # experts 0..7 overflow (all their slots filled)
+    # 16 experts: the first and last of the batch, both sides of a CTA pair's tile boundary, and the
+    # neighbours of the multiples of the SM count at which the persistent tile lists wrap
+    for e in (0, 1, 7, 73, 74, 147, 148, 149, 255, 256, 295, 296, 300, 443, 510, 511):
         wi_e, wo_e = to_np(inp["wi"][e]), to_np(inp["wo"][e])
         rows_x, rows_dout = [], []
         for g in range(cfg.G):
