@@ -102,6 +102,13 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  one persistent launch of CTA pairs, GEMM-2 reading
                                                  the hidden activations from L2 (they are still written
                                                  once) */
+#define GSHARD_FLAG_BWD_PAIRED_GEMMS 4096u    /* backward: the GEMM that computes dh runs beside the one
+                                                 for dwo, and dbuf beside dwi, each on half of the
+                                                 multiprocessors (second, library-owned stream), so
+                                                 that HBM sees reads and writes mixed.  Measured
+                                                 slower than the default (one after another on all
+                                                 multiprocessors); kept for measurement */
+#define GSHARD_FLAG_ALL 8191u
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

@@ -138,7 +138,7 @@ int validate_shape(const gshard_moe_shape* s) {
   if (!s) return GSHARD_ERR_INVALID_ARG;
   if (s->G <= 0 || s->S <= 0 || s->M <= 0 || s->H <= 0 || s->E <= 0 || s->C <= 0) return GSHARD_ERR_INVALID_ARG;
   if (s->dtype != GSHARD_F32 && s->dtype != GSHARD_BF16) return GSHARD_ERR_INVALID_ARG;
-  if (s->flags & ~4095u) return GSHARD_ERR_INVALID_ARG;
+  if (s->flags & ~GSHARD_FLAG_ALL) return GSHARD_ERR_INVALID_ARG;
   if ((s->flags & GSHARD_FLAG_FUSED_FFN) && (s->flags & GSHARD_FLAG_UNFUSED_FFN)) return GSHARD_ERR_INVALID_ARG;
   if (s->E < 2) return GSHARD_ERR_INVALID_ARG;
   if (s->M % 8 || s->H % 8) return GSHARD_ERR_UNSUPPORTED_SHAPE;

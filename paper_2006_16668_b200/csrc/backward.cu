@@ -8,6 +8,8 @@
 //   dlogit = g * (dg - <g, dg>),  dwg = x^T dlogit,  dx += dlogit wg^T
 //   expert path: dout[slot] = w dy,  dh = (dout wo^T) * 1[h > 0],  dwo = h^T dout,
 //                dwi = buf^T dh,  dbuf = dh wi^T,  dx += dbuf[slot]
+#include <mutex>
+
 #include "gemm_dispatch.cuh"
 #include "plan.cuh"
 
@@ -186,6 +188,55 @@ __global__ void __launch_bounds__(256) sum_partials_kernel(const float4* __restr
   out[i] = acc;
 }
 
+// A second stream and two events per device for the pairs of expert GEMMs that run side by side
+// (host-side objects, created on first use and kept for the life of the process).
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+SideStream* side_stream_for_current_device() {
+  constexpr int kMaxDevices = 64;
+  static SideStream pool[kMaxDevices];
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return nullptr; }
+  std::lock_guard<std::mutex> lock(mu);
+  SideStream& s = pool[dev];
+  if (!s.stream) {
+    cudaStream_t st = nullptr; cudaEvent_t a = nullptr, b = nullptr;
+    if (cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&a, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&b, cudaEventDisableTiming) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    s.stream = st; s.fork = a; s.join = b;
+  }
+  return &s;
+}
+
+// Runs GEMMs `a` (on `st`) and `b` (on the side stream) at the same time, each on its share of the
+// multiprocessors; `b` is ordered after everything enqueued on `st` so far and `st` continues only
+// after both.  share_a: multiprocessors given to `a` (even).
+int run_gemm_pair(const Dims& d, UmmaGemm a, UmmaGemm b, int share_a, int* status, cudaStream_t st) {
+  SideStream* side = side_stream_for_current_device();
+  const int sms = device_sms();
+  if (!side || d.simt || share_a <= 0 || share_a >= sms) {
+    int rc = run_gemm(d, a, status, st);
+    return rc ? rc : run_gemm(d, b, status, st);
+  }
+  a.max_ctas = share_a; b.max_ctas = sms - share_a;
+  if (cudaEventRecord(side->fork, st) != cudaSuccess || cudaStreamWaitEvent(side->stream, side->fork, 0) != cudaSuccess)
+    return GSHARD_ERR_CUDA;
+  int rc = run_gemm(d, a, status, st);
+  if (rc) return rc;
+  rc = run_gemm(d, b, status, side->stream);
+  if (rc) return rc;
+  if (cudaEventRecord(side->join, side->stream) != cudaSuccess || cudaStreamWaitEvent(st, side->join, 0) != cudaSuccess)
+    return GSHARD_ERR_CUDA;
+  return GSHARD_OK;
+}
+
 template <typename T>
 int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, const void* wo, const unsigned char* ctx,
                const void* dy, float k_aux, void* dx, float* dwg, void* dwi, void* dwo, unsigned char* ws,
@@ -224,36 +275,34 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   count_launch(2);
   launch_dispatch(d, x, slot_token, buf, st);
 
-  // expert FFN backward
-  UmmaGemm g{};
+  // expert FFN backward.  dh and dbuf stream the weights (read-heavy), dwo and dwi write a gradient the
+  // size of the weights from short contractions (write-heavy): one of each runs side by side.
+  UmmaGemm g_dh{}, g_dwo{}, g_dwi{}, g_dbuf{};
   // dh = (dout . wo^T) masked by h > 0
-  g.A = dout; g.B = wo; g.C = dh; g.mask = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;
-  g.a_kmajor = true; g.b_kmajor = true;
-  g.a_ld = d.M; g.a_bs = rows * d.M; g.b_ld = d.M; g.b_bs = (long long)d.H * d.M; g.c_ld = d.H; g.c_bs = rows * d.H;
-  g.b_stream = 1; g.prefer_two_sm = 1;
-  int rc = run_gemm(d, g, status, st);
-  if (rc) return rc;
+  g_dh.A = dout; g_dh.B = wo; g_dh.C = dh; g_dh.mask = h; g_dh.rows = d.rows; g_dh.cols = d.H; g_dh.K = d.M; g_dh.batch = d.E;
+  g_dh.a_kmajor = true; g_dh.b_kmajor = true;
+  g_dh.a_ld = d.M; g_dh.a_bs = rows * d.M; g_dh.b_ld = d.M; g_dh.b_bs = (long long)d.H * d.M; g_dh.c_ld = d.H; g_dh.c_bs = rows * d.H;
+  g_dh.b_stream = 1; g_dh.prefer_two_sm = 1;
   // dwo[e] = h[e]^T . dout[e]   [H x M]
-  g = UmmaGemm{};
-  g.A = h; g.B = dout; g.C = dwo; g.rows = d.H; g.cols = d.M; g.K = d.rows; g.batch = d.E;
-  g.a_kmajor = false; g.b_kmajor = false;
-  g.a_ld = d.H; g.a_bs = rows * d.H; g.b_ld = d.M; g.b_bs = rows * d.M; g.c_ld = d.M; g.c_bs = (long long)d.H * d.M;
-  rc = run_gemm(d, g, status, st);
-  if (rc) return rc;
+  g_dwo.A = h; g_dwo.B = dout; g_dwo.C = dwo; g_dwo.rows = d.H; g_dwo.cols = d.M; g_dwo.K = d.rows; g_dwo.batch = d.E;
+  g_dwo.a_kmajor = false; g_dwo.b_kmajor = false;
+  g_dwo.a_ld = d.H; g_dwo.a_bs = rows * d.H; g_dwo.b_ld = d.M; g_dwo.b_bs = rows * d.M; g_dwo.c_ld = d.M; g_dwo.c_bs = (long long)d.H * d.M;
   // dwi[e] = buf[e]^T . dh[e]   [M x H]
-  g = UmmaGemm{};
-  g.A = buf; g.B = dh; g.C = dwi; g.rows = d.M; g.cols = d.H; g.K = d.rows; g.batch = d.E;
-  g.a_kmajor = false; g.b_kmajor = false;
-  g.a_ld = d.M; g.a_bs = rows * d.M; g.b_ld = d.H; g.b_bs = rows * d.H; g.c_ld = d.H; g.c_bs = (long long)d.M * d.H;
-  rc = run_gemm(d, g, status, st);
-  if (rc) return rc;
+  g_dwi.A = buf; g_dwi.B = dh; g_dwi.C = dwi; g_dwi.rows = d.M; g_dwi.cols = d.H; g_dwi.K = d.rows; g_dwi.batch = d.E;
+  g_dwi.a_kmajor = false; g_dwi.b_kmajor = false;
+  g_dwi.a_ld = d.M; g_dwi.a_bs = rows * d.M; g_dwi.b_ld = d.H; g_dwi.b_bs = rows * d.H; g_dwi.c_ld = d.H; g_dwi.c_bs = (long long)d.M * d.H;
   // dbuf = dh . wi^T   [rows x M]
-  g = UmmaGemm{};
-  g.A = dh; g.B = wi; g.C = dbuf; g.rows = d.rows; g.cols = d.M; g.K = d.H; g.batch = d.E;
-  g.a_kmajor = true; g.b_kmajor = true;
-  g.a_ld = d.H; g.a_bs = rows * d.H; g.b_ld = d.H; g.b_bs = (long long)d.M * d.H; g.c_ld = d.M; g.c_bs = rows * d.M;
-  g.b_stream = 1; g.prefer_two_sm = 1;
-  rc = run_gemm(d, g, status, st);
+  g_dbuf.A = dh; g_dbuf.B = wi; g_dbuf.C = dbuf; g_dbuf.rows = d.rows; g_dbuf.cols = d.M; g_dbuf.K = d.H; g_dbuf.batch = d.E;
+  g_dbuf.a_kmajor = true; g_dbuf.b_kmajor = true;
+  g_dbuf.a_ld = d.H; g_dbuf.a_bs = rows * d.H; g_dbuf.b_ld = d.H; g_dbuf.b_bs = (long long)d.M * d.H; g_dbuf.c_ld = d.M; g_dbuf.c_bs = rows * d.M;
+  g_dbuf.b_stream = 1; g_dbuf.prefer_two_sm = 1;
+  // On request each read-heavy GEMM shares the GPU with a write-heavy one (half of the multiprocessors
+  // each, two streams).  Measured at the MoE(512E) training shape this is slower than running the four
+  // one after another on all multiprocessors, so it is not the default.
+  const int share = d.bwd_paired ? (device_sms() / 2) & ~1 : 0;
+  int rc = run_gemm_pair(d, g_dh, g_dwo, share, status, st);
+  if (rc) return rc;
+  rc = run_gemm_pair(d, g_dbuf, g_dwi, share, status, st);
   if (rc) return rc;
 
   // gating backward: recompute the logits, softmax backward, two GEMMs
@@ -264,7 +313,7 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
                                                      aux_coef, dlogits, d.N, d.S, d.E);
   count_launch();
   // dwg = x^T . dlogits   [M x E] fp32
-  g = UmmaGemm{};
+  UmmaGemm g{};
   g.A = x; g.B = dlogits; g.C = dwg; g.rows = d.M; g.cols = d.E; g.K = (int)d.N; g.batch = 1;
   g.a_kmajor = false; g.b_kmajor = false; g.a_ld = d.M; g.b_ld = d.E; g.c_ld = d.E; g.out_f32 = 1;
   // Few output tiles, very long contraction: split the token dimension over the batch index so that

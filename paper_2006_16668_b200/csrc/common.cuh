@@ -101,6 +101,7 @@ struct Dims {
   bool gate_one_sm;     // stored-logits gating kernel on single CTAs instead of CTA pairs
   bool gate_cluster;    // gating on clusters with the mean-gate partial sums fused in (no stored logits)
   bool gather_dispatch; // single-launch FFN gathers its rows from x instead of reading a dispatch buffer
+  bool bwd_paired;      // backward: read-heavy and write-heavy expert GEMMs side by side on half of the SMs each
 };
 
 inline Dims make_dims(const gshard_moe_shape& s) {
@@ -123,6 +124,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.one_sm_mma = (s.flags & GSHARD_FLAG_ONE_SM_MMA) != 0;
   d.add_residual = (s.flags & GSHARD_FLAG_ADD_RESIDUAL) != 0;
   d.chained_ffn = (s.flags & GSHARD_FLAG_CHAINED_FFN) != 0;
+  d.bwd_paired = (s.flags & GSHARD_FLAG_BWD_PAIRED_GEMMS) != 0;
   return d;
 }
 

@@ -54,6 +54,8 @@ struct UmmaGemm {
   int relu;
   int a_stream, b_stream;    // operand is read once: load with an evict-first L2 hint
   int prefer_two_sm;         // run on CTA pairs (cta_group::2) when a problem has more than 128 rows
+  int max_ctas;              // > 0: use at most this many CTAs (persistent grid), leaving the other
+                             // multiprocessors to a kernel running beside this one on another stream
 };
 int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st);
 // umma2_gemm.cu: the same contraction with the two-SM MMA (CTA pairs, 256 x 256 tiles).

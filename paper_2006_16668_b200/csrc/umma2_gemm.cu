@@ -252,6 +252,7 @@ int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   p.status = status;
   const int sms = device_sms();
   int pairs = sms / 2;
+  if (g.max_ctas > 0 && pairs > g.max_ctas / 2) pairs = g.max_ctas / 2 > 0 ? g.max_ctas / 2 : 1;
   if (pairs > p.total_tiles) pairs = p.total_tiles;
 #define GSHARD_DISPATCH2(AK, BKM) \
   (p.mask ? launch2_t<AK, BKM, true>(ma, mb, p, pairs, st) : launch2_t<AK, BKM, false>(ma, mb, p, pairs, st))

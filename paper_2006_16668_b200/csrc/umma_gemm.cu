@@ -396,7 +396,8 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   // stream the larger operand once: walk the tiles that share it back to back
   p.n_fastest = (g.rows > g.cols) ? 1 : 0;
   p.status = status;
-  const int sms = device_sms();
+  int sms = device_sms();
+  if (g.max_ctas > 0 && sms > g.max_ctas) sms = g.max_ctas;
   if (!g.a_kmajor && !g.b_kmajor && !g.mask && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
     // short contraction, several row tiles per column block: keep the B tile resident
     const int n_groups = p.n_tiles * g.batch;

@@ -62,6 +62,8 @@ BWD_CASES = [
     # full four k-blocks
     ("bf16_wgrad_resident_ragged", 2, 256, 512, 640, 16, 40, "bf16", 0, GRAD_TOL),
     ("bf16_wgrad_resident_k256", 2, 1024, 512, 512, 16, 128, "bf16", 0, GRAD_TOL),
+    # dh beside dwo and dbuf beside dwi, half of the multiprocessors each
+    ("bf16_paired_gemms", 2, 1024, 512, 512, 16, 128, "bf16", B.GSHARD_FLAG_BWD_PAIRED_GEMMS, GRAD_TOL),
 ]
 
 
