@@ -270,6 +270,67 @@ int gshard_moe_expert_ffn(const gshard_moe_shape* shape, const void* buf, const 
 int gshard_moe_combine(const gshard_moe_shape* shape, const void* out, const int32_t* expert_idx,
                        const int32_t* slot, const float* weight, void* y, void* cuda_stream);
 
+/* ---- expert-parallel form over several GPUs ------------------------------------------------
+ * The paper's partitioning of the layer (Algorithm 2 and the sharding annotations of the MoE layer
+ * in the section on the SPMD partitioner; AllToAll cost in the performance section): groups G split
+ * over the devices for gating, capacity assignment, dispatch and combine with wg replicated,
+ * experts E split over the devices for the expert FFN, one AllToAll before and one after it.
+ * One process per GPU; rank r of `world` owns groups [r*G/world, (r+1)*G/world) and experts
+ * [r*E/world, (r+1)*E/world); G and E must be multiples of world. */
+
+/* Where a rank's data lives, as computed on the host by gshard_moe_ep_plan (no GPU needed). */
+typedef struct {
+  int32_t rank, world;
+  int32_t groups_local, experts_local;   /* G/world, E/world                                        */
+  int32_t group_begin, expert_begin;     /* first global group / expert of this rank                */
+  int32_t rows_local;                    /* groups_local * C: rows of one expert in one rank's slab  */
+  size_t row_bytes;                      /* M elements                                               */
+  size_t bytes_per_peer;                 /* experts_local * rows_local * row_bytes: one slab         */
+  gshard_moe_shape local;                /* shape of the stages that run on the local groups (G = G/world) */
+  gshard_moe_shape ffn;                  /* shape of the local expert FFN (E = E/world, all G groups' rows) */
+} gshard_moe_ep_layout;
+
+/* The collectives, supplied by the caller (NCCL, torch.distributed, MPI ...).  Both enqueue on
+ * cuda_stream (or order themselves after and before it) and return 0 on success.
+ *   all_to_all: equal splits; bytes [i*bytes_per_peer, (i+1)*bytes_per_peer) of send go to rank i,
+ *     the same range of recv receives from rank i.  send and recv are device buffers inside the
+ *     workspace of the call and never alias.
+ *   all_reduce_sum_f32: in-place sum over the ranks of `count` floats in device memory. */
+typedef struct {
+  int (*all_to_all)(void* user, const void* send, void* recv, size_t bytes_per_peer, void* cuda_stream);
+  int (*all_reduce_sum_f32)(void* user, float* buf, size_t count, void* cuda_stream);
+  void* user;
+} gshard_ep_comm;
+
+/* Host-only: validates the partitioning and fills `layout`.  GSHARD_ERR_UNSUPPORTED_SHAPE when G or
+ * E is not a multiple of world (or SAVE_FOR_BACKWARD is set: the expert-parallel form is forward only). */
+int gshard_moe_ep_plan(const gshard_moe_shape* shape, int rank, int world, gshard_moe_ep_layout* layout);
+
+/* Host-only: the permutation between the layout an AllToAll delivers, [world (source rank)]
+ * [experts_local][rows_local] rows, and the layout the expert FFN reads, [experts_local]
+ * [world * rows_local] rows (one expert's rows from all sources contiguous, in global group order);
+ * inverse != 0 goes back.  src and dst are HOST buffers of world * experts_local * rows_local rows of
+ * row_bytes bytes.  The device-side regroup inside gshard_moe_top2_forward_ep uses the same index
+ * arithmetic; this function lets a CPU-only multi-process test drive it. */
+int gshard_moe_ep_regroup_host(const gshard_moe_ep_layout* layout, const void* src, void* dst, size_t row_bytes,
+                               int inverse);
+
+size_t gshard_moe_ep_workspace_bytes(const gshard_moe_shape* shape, int world);
+
+/* Forward of the layer on rank `rank` of `world` (shape is the GLOBAL shape).
+ *   x_local, y_local [G/world, S, M], u_local [G/world, S]: this rank's groups; wg [M, E] replicated;
+ *   wi_local [E/world, M, H], wo_local [E/world, H, M]: this rank's experts.
+ *   l_aux: the layer's loss (mean over ALL groups), identical on every rank after the call.
+ *   routing_out: optional outputs for the LOCAL groups (shapes as in gshard_moe_routing with
+ *   G = G/world; stats are this rank's).  comm: the collectives; may be NULL when world == 1.
+ * With world == 1 the call runs exactly the kernels of gshard_moe_top2_forward and gives the same
+ * bits.  Every received slab lies in this GPU's own workspace before a kernel reads it. */
+int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int world, const void* x_local,
+                               const void* wg, const void* wi_local, const void* wo_local,
+                               const float* u_local, void* y_local, float* l_aux,
+                               const gshard_moe_routing* routing_out, const gshard_ep_comm* comm,
+                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+
 /* The position-wise feed-forward sub-layer of the ordinary Transformer layers that alternate with
  * the MoE layers (section 2.1: every other feed-forward layer is replaced by a MoE layer; the
  * performance section times "MoE layer + adjacent Transformer layer"): y = relu(x . wi) . wo over

@@ -50,6 +50,21 @@ class gshard_moe_routing(Structure):
                                         "total_count", "slot_token", "m", "l_aux_group", "stats")]
 
 
+class gshard_moe_ep_layout(Structure):
+    _fields_ = [("rank", c_int32), ("world", c_int32), ("groups_local", c_int32), ("experts_local", c_int32),
+                ("group_begin", c_int32), ("expert_begin", c_int32), ("rows_local", c_int32),
+                ("row_bytes", c_size_t), ("bytes_per_peer", c_size_t), ("local", gshard_moe_shape),
+                ("ffn", gshard_moe_shape)]
+
+
+ALL_TO_ALL_FN = ctypes.CFUNCTYPE(c_int, c_void_p, c_void_p, c_void_p, c_size_t, c_void_p)
+ALL_REDUCE_FN = ctypes.CFUNCTYPE(c_int, c_void_p, c_void_p, c_size_t, c_void_p)
+
+
+class gshard_ep_comm(Structure):
+    _fields_ = [("all_to_all", ALL_TO_ALL_FN), ("all_reduce_sum_f32", ALL_REDUCE_FN), ("user", c_void_p)]
+
+
 EXPORTS = {
     # name: (restype, argtypes)
     "gshard_version": (c_int, []),
@@ -74,6 +89,12 @@ EXPORTS = {
     "gshard_moe_dispatch": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 4),
     "gshard_moe_expert_ffn": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 5 + [c_size_t, c_void_p]),
     "gshard_moe_combine": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6),
+    "gshard_moe_ep_plan": (c_int, [POINTER(gshard_moe_shape), c_int, c_int, POINTER(gshard_moe_ep_layout)]),
+    "gshard_moe_ep_regroup_host": (c_int, [POINTER(gshard_moe_ep_layout), c_void_p, c_void_p, c_size_t, c_int]),
+    "gshard_moe_ep_workspace_bytes": (c_size_t, [POINTER(gshard_moe_shape), c_int]),
+    "gshard_moe_top2_forward_ep": (c_int, [POINTER(gshard_moe_shape), c_int, c_int] + [c_void_p] * 7 +
+                                   [POINTER(gshard_moe_routing), POINTER(gshard_ep_comm), c_void_p, c_size_t,
+                                    c_void_p]),
     "gshard_dense_ffn_workspace_bytes": (c_size_t, [ctypes.c_int64, c_int32, c_int32, c_int32]),
     "gshard_dense_ffn_forward": (c_int, [ctypes.c_int64, c_int32, c_int32, c_int32] + [c_void_p] * 5 +
                                  [c_size_t, c_void_p]),
@@ -259,6 +280,38 @@ def gshard_moe_expert_ffn(shape, buf, wi, wo, out, workspace, stream=None):
 def gshard_moe_combine(shape, out, expert_idx, slot, weight, y, stream=None):
     _check(load().gshard_moe_combine(ctypes.byref(shape), _p(out), _p(expert_idx), _p(slot), _p(weight), _p(y),
                                      _stream(stream)), "gshard_moe_combine")
+
+
+def gshard_moe_ep_plan(shape, rank, world) -> gshard_moe_ep_layout:
+    """Host-only partitioning arithmetic of the expert-parallel form (works without a GPU)."""
+    layout = gshard_moe_ep_layout()
+    _check(load().gshard_moe_ep_plan(ctypes.byref(shape), int(rank), int(world), ctypes.byref(layout)),
+           "gshard_moe_ep_plan")
+    return layout
+
+
+def gshard_moe_ep_regroup_host(layout, src, dst, inverse=False):
+    """Permutes HOST tensors (rows of equal byte length) between the AllToAll layout and the expert
+    FFN's layout; src and dst are contiguous CPU tensors of world * experts_local * rows_local rows."""
+    rows = layout.world * layout.experts_local * layout.rows_local
+    row_bytes = src.numel() * src.element_size() // rows
+    assert src.is_contiguous() and dst.is_contiguous() and src.numel() == dst.numel()
+    _check(load().gshard_moe_ep_regroup_host(ctypes.byref(layout), src.data_ptr(), dst.data_ptr(), row_bytes,
+                                             int(bool(inverse))), "gshard_moe_ep_regroup_host")
+
+
+def gshard_moe_ep_workspace_bytes(shape, world) -> int:
+    return int(load().gshard_moe_ep_workspace_bytes(ctypes.byref(shape), int(world)))
+
+
+def gshard_moe_top2_forward_ep(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux,
+                               routing_out=None, comm=None, workspace=None, stream=None):
+    rp = ctypes.byref(routing_out) if routing_out is not None else None
+    cp = ctypes.byref(comm) if comm is not None else None
+    _check(load().gshard_moe_top2_forward_ep(ctypes.byref(shape), int(rank), int(world), _p(x_local), _p(wg),
+                                             _p(wi_local), _p(wo_local), _p(u_local), _p(y_local), _p(l_aux), rp, cp,
+                                             _p(workspace), workspace.numel(), _stream(stream)),
+           "gshard_moe_top2_forward_ep")
 
 
 def _dtype_code(t) -> int:

@@ -19,10 +19,6 @@ static FfnTiming& ffn_timing() {
   return t;
 }
 
-namespace {
-
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
 int check_device() {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return GSHARD_ERR_CUDA; }
@@ -30,6 +26,10 @@ int check_device() {
   if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return GSHARD_ERR_CUDA;
   return major == 10 ? GSHARD_OK : GSHARD_ERR_ARCH;
 }
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 #define GS_REQUIRE_PTR(p)                                          \
   do {                                                             \
@@ -53,8 +53,6 @@ int gate_logits(const Dims& d, const void* x, const void* wg, float* logits, int
   g.out_f32 = 1; g.a_stream = 1;
   return run_gemm(d, g, status, st);
 }
-
-namespace {
 
 int gate_stage(const Dims& d, const FwdPlan& pl, unsigned char* ws, const void* x, const void* wg,
                int32_t* expert_idx, float* gate12, float* m, float* rowmax, float* rowinv, cudaStream_t st) {
@@ -96,8 +94,7 @@ bool ffn_runs_fused(const Dims& d, bool keep_h) {
 
 // With x / slot_token (only where ffn_runs_fused) the rows are gathered from x and buf is not read.
 int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
-              void* fused_scratch, int* status, cudaStream_t st, const void* x = nullptr,
-              const int32_t* slot_token = nullptr) {
+              void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token) {
   const long long rows = d.rows;
   // One persistent launch in which the hidden activations never leave L2: the faster form when
   // the FFN is bound by streaming the expert weights (at most one 128-row tile per expert); with
@@ -127,12 +124,6 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   g2.b_stream = 1; g2.prefer_two_sm = 1;
   return run_gemm(d, g2, status, st);
 }
-
-template <typename T> T* pick(T* user, unsigned char* ws, size_t off) {
-  return user ? user : reinterpret_cast<T*>(ws + off);
-}
-
-}  // namespace
 
 int validate_shape(const gshard_moe_shape* s) {
   if (!s) return GSHARD_ERR_INVALID_ARG;
@@ -435,7 +426,7 @@ int gshard_moe_expert_ffn(const gshard_moe_shape* shape, const void* buf, const 
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   if (cudaMemsetAsync(ws + pl.status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   GS_TRY(ffn_stage(d, buf, wi, wo, ws + pl.h, false, out, ws + pl.ffn_scratch,
-                   reinterpret_cast<int*>(ws + pl.status), st));
+                   reinterpret_cast<int*>(ws + pl.status), st, nullptr, nullptr));
   return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 

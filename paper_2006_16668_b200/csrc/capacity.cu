@@ -180,12 +180,14 @@ __global__ void __launch_bounds__(kCapThreads) capacity_kernel(CapacityArgs a) {
 }
 
 // Layer-level results: l_aux = mean over groups (fixed order), stats summed over groups.
-__global__ void capacity_finalize_kernel(const float* l_aux_group, const int32_t* stats_group, int G,
+// G_mean: the number of groups the mean is taken over (more than G when these G groups are one
+// rank's share of a layer whose groups are spread over several GPUs; the shares are then added).
+__global__ void capacity_finalize_kernel(const float* l_aux_group, const int32_t* stats_group, int G, int G_mean,
                                          float* l_aux, long long* stats) {
   if (threadIdx.x == 0 && l_aux) {
     float acc = 0.f;
     for (int g = 0; g < G; ++g) acc += l_aux_group[g];
-    *l_aux = acc / (float)G;
+    *l_aux = acc / (float)G_mean;
   }
   if (stats && threadIdx.x < 8) {
     long long acc = 0;
@@ -205,7 +207,7 @@ int capacity_warps_for(int E) {
 int launch_capacity(const Dims& d, const int32_t* expert_idx, const float* gate12, const float* u,
                     const float* m, int32_t* slot, float* weight, uint8_t* flags, int32_t* first_count,
                     int32_t* total_count, int32_t* slot_token, float* l_aux_group, int32_t* stats_group,
-                    float* l_aux, long long* stats, cudaStream_t st) {
+                    float* l_aux, long long* stats, cudaStream_t st, int groups_in_mean) {
   CapacityArgs a;
   a.S = d.S; a.E = d.E; a.C = d.C; a.G = d.G;
   a.warps_used = capacity_warps_for(d.E);
@@ -220,7 +222,8 @@ int launch_capacity(const Dims& d, const int32_t* expert_idx, const float* gate1
   if (cudaFuncSetAttribute(capacity_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
     return GSHARD_ERR_CUDA;
   capacity_kernel<<<d.G, kCapThreads, smem, st>>>(a);
-  capacity_finalize_kernel<<<1, 32, 0, st>>>(l_aux_group, stats_group, d.G, l_aux, stats);
+  capacity_finalize_kernel<<<1, 32, 0, st>>>(l_aux_group, stats_group, d.G, groups_in_mean > 0 ? groups_in_mean : d.G,
+                                             l_aux, stats);
   count_launch(2);
   return GSHARD_OK;
 }

@@ -1,0 +1,197 @@
+// Expert-parallel form of the layer (the paper's own partitioning, Algorithm 2 with the sharding
+// annotations of the MoE layer): the groups G are split over the devices for gating, capacity
+// assignment, dispatch and combine (wg replicated), the experts E are split over the devices for
+// the expert FFN, and an AllToAll before and after the FFN changes between the two layouts
+// ("GSEC,GSM->EGCM" is sharded on G on its inputs and on E on its output).
+//
+// Rank r of W holds groups [r*G/W, (r+1)*G/W) of x, u, y and experts [r*E/W, (r+1)*E/W) of wi, wo.
+//   1. gating + capacity + dispatch over the local groups:   send [E, Gl*C, M] = [W][El, Gl*C, M]
+//   2. AllToAll (equal splits): slab d goes to rank d        recv [W(src)][El, Gl*C, M]
+//   3. regroup: rows of one local expert from all sources become contiguous, in global group
+//      order                                                  in   [El, W*Gl*C = G*C, M]
+//   4. expert FFN over the El local experts with G*C rows each (the same kernels as on one GPU)
+//   5. inverse regroup, AllToAll back                         out  [E, Gl*C, M]
+//   6. combine over the local groups; l_aux = sum over ranks of (sum of local group losses) / G
+// The collectives are the caller's: two callbacks (all-to-all, all-reduce of floats) that enqueue
+// on the given stream - NCCL behind torch.distributed in this repository's harness.  Every slab is
+// received into this GPU's own workspace before any kernel or TMA load touches it; no tensor map
+// ever covers another GPU's memory and no load is multicast.
+#include <cstring>
+
+#include "kernels.cuh"
+#include "plan.cuh"
+
+namespace gshard {
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Row of the FFN input [El, G*C, .] that holds row `row_local` (= gl*C + c) of local expert `el` in
+// the slab received from rank `src`: the source's groups are global groups src*Gl + gl.
+__host__ __device__ inline long long ep_ffn_row(int W, int El, int rows_local, int src, int el, int row_local) {
+  return ((long long)el * W + src) * rows_local + row_local;
+}
+__host__ __device__ inline long long ep_slab_row(int El, int rows_local, int src, int el, int row_local) {
+  return ((long long)src * El + el) * rows_local + row_local;
+}
+
+// dst/src as 16-byte vectors, row_vec per row.  inverse == 0: slab order -> FFN order.
+__global__ void __launch_bounds__(256) ep_regroup_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int W,
+                                                         int El, int rows_local, int row_vec, int inverse) {
+  const long long chunk_vec = (long long)rows_local * row_vec;        // one (rank, expert) block is contiguous
+  const long long total = (long long)W * El * chunk_vec;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    const long long blk = i / chunk_vec, off = i % chunk_vec;
+    const int s = (int)(blk / El), el = (int)(blk % El);              // blk indexes the slab order [W][El]
+    const long long slab = ep_slab_row(El, rows_local, s, el, 0) * row_vec + off;
+    const long long ffn = ep_ffn_row(W, El, rows_local, s, el, 0) * row_vec + off;
+    if (inverse) dst[slab] = src[ffn]; else dst[ffn] = src[slab];
+  }
+}
+
+void launch_ep_regroup(const void* src, void* dst, int W, int El, int rows_local, int row_vec, int inverse,
+                       cudaStream_t st) {
+  const long long total = (long long)W * El * rows_local * row_vec;
+  long long blocks = (total + 255) / 256;
+  const long long cap = (long long)device_sms() * 16;
+  if (blocks > cap) blocks = cap;
+  ep_regroup_kernel<<<(int)(blocks > 0 ? blocks : 1), 256, 0, st>>>(static_cast<const uint4*>(src), static_cast<uint4*>(dst),
+                                                                    W, El, rows_local, row_vec, inverse);
+  count_launch();
+}
+
+int make_layout(const gshard_moe_shape* shape, int rank, int world, gshard_moe_ep_layout* out) {
+  const int rc = validate_shape(shape);
+  if (rc != GSHARD_OK) return rc;
+  if (world < 1 || rank < 0 || rank >= world) return GSHARD_ERR_INVALID_ARG;
+  if (shape->G % world || shape->E % world) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  if (shape->flags & GSHARD_FLAG_SAVE_FOR_BACKWARD) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  gshard_moe_ep_layout l;
+  l.rank = rank; l.world = world;
+  l.groups_local = shape->G / world; l.experts_local = shape->E / world;
+  l.group_begin = rank * l.groups_local; l.expert_begin = rank * l.experts_local;
+  l.rows_local = l.groups_local * shape->C;
+  const size_t esize = shape->dtype == GSHARD_BF16 ? 2 : 4;
+  l.row_bytes = (size_t)shape->M * esize;
+  l.bytes_per_peer = (size_t)l.experts_local * l.rows_local * l.row_bytes;
+  l.local = *shape;  l.local.G = l.groups_local;                  // gating, capacity, dispatch, combine
+  l.ffn = *shape;    l.ffn.E = l.experts_local;                   // expert FFN: all G groups' rows of El experts
+  // the local problems must themselves be valid shapes (E stays global for the gating; El >= 1 for the FFN)
+  const int rl = validate_shape(&l.local);
+  if (rl != GSHARD_OK) return rl;
+  *out = l;
+  return GSHARD_OK;
+}
+
+}  // namespace
+
+}  // namespace gshard
+
+using namespace gshard;
+
+extern "C" {
+
+int gshard_moe_ep_plan(const gshard_moe_shape* shape, int rank, int world, gshard_moe_ep_layout* layout) {
+  if (!layout) return GSHARD_ERR_INVALID_ARG;
+  return make_layout(shape, rank, world, layout);
+}
+
+int gshard_moe_ep_regroup_host(const gshard_moe_ep_layout* l, const void* src, void* dst, size_t row_bytes,
+                               int inverse) {
+  if (!l || !src || !dst || row_bytes == 0 || l->world < 1 || l->experts_local < 1 || l->rows_local < 1)
+    return GSHARD_ERR_INVALID_ARG;
+  const unsigned char* s = static_cast<const unsigned char*>(src);
+  unsigned char* d = static_cast<unsigned char*>(dst);
+  for (int r = 0; r < l->world; ++r)
+    for (int el = 0; el < l->experts_local; ++el)
+      for (int row = 0; row < l->rows_local; ++row) {
+        const size_t slab = (size_t)ep_slab_row(l->experts_local, l->rows_local, r, el, row) * row_bytes;
+        const size_t ffn = (size_t)ep_ffn_row(l->world, l->experts_local, l->rows_local, r, el, row) * row_bytes;
+        if (inverse) memcpy(d + slab, s + ffn, row_bytes); else memcpy(d + ffn, s + slab, row_bytes);
+      }
+  return GSHARD_OK;
+}
+
+size_t gshard_moe_ep_workspace_bytes(const gshard_moe_shape* shape, int world) {
+  gshard_moe_ep_layout l;
+  if (make_layout(shape, 0, world, &l) != GSHARD_OK) return 0;
+  const Dims dl = make_dims(l.local);
+  // the local forward plan (its buf / h / out regions have exactly the sizes the FFN over El experts
+  // and G*C rows needs) plus two exchange buffers of one dispatch buffer each
+  return plan_forward(dl).total + 2 * align_up((size_t)dl.R * dl.M * dl.esize);
+}
+
+int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int world, const void* x_local,
+                               const void* wg, const void* wi_local, const void* wo_local, const float* u_local,
+                               void* y_local, float* l_aux, const gshard_moe_routing* routing_out,
+                               const gshard_ep_comm* comm, void* workspace, size_t workspace_bytes,
+                               void* cuda_stream) {
+  launch_counter().n = 0;
+  gshard_moe_ep_layout l;
+  const int rcl = make_layout(shape, rank, world, &l);
+  if (rcl != GSHARD_OK) return rcl;
+  const void* ptrs[] = {x_local, wg, wi_local, wo_local, u_local, y_local, workspace};
+  for (const void* p : ptrs)
+    if (p == nullptr || !aligned16(p)) return GSHARD_ERR_INVALID_ARG;
+  if (l_aux == nullptr) return GSHARD_ERR_INVALID_ARG;
+  if (world > 1 && (!comm || !comm->all_to_all || !comm->all_reduce_sum_f32)) return GSHARD_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  if (workspace_bytes < gshard_moe_ep_workspace_bytes(shape, world)) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  const int rcd = check_device();
+  if (rcd != GSHARD_OK) return rcd;
+
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const Dims dl = make_dims(l.local);          // G = Gl, E global
+  const Dims df = make_dims(l.ffn);            // G global, E = El: rows per expert = G*C
+  const FwdPlan pl = plan_forward(dl);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  const size_t slab_bytes = align_up((size_t)dl.R * dl.M * dl.esize);
+  void* xa = ws + pl.total;                    // exchange buffers
+  void* xb = ws + pl.total + slab_bytes;
+  gshard_moe_routing r{};
+  if (routing_out) r = *routing_out;
+  int* status = reinterpret_cast<int*>(ws + pl.status);
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  int32_t* expert_idx = pick(r.expert_idx, ws, pl.expert_idx);
+  int32_t* slot = pick(r.slot, ws, pl.slot);
+  float* weight = pick(r.weight, ws, pl.weight);
+  int32_t* slot_token = pick(r.slot_token, ws, pl.slot_token);
+  float* gate12 = reinterpret_cast<float*>(ws + pl.gate12);
+  float* m = pick(r.m, ws, pl.m);
+  void* buf = ws + pl.buf;
+  void* h = ws + pl.h;
+  void* out = ws + pl.out;
+
+  int rc = gate_stage(dl, pl, ws, x_local, wg, expert_idx, gate12, m, reinterpret_cast<float*>(ws + pl.rowmax),
+                      reinterpret_cast<float*>(ws + pl.rowinv), st);
+  if (rc != GSHARD_OK) return rc;
+  // l_aux: this rank's group losses over the GLOBAL group count; the all-reduce below adds the shares
+  rc = launch_capacity(dl, expert_idx, gate12, u_local, m, slot, weight, pick(r.flags, ws, pl.flags),
+                       pick(r.first_count, ws, pl.first_count), pick(r.total_count, ws, pl.total_count), slot_token,
+                       pick(r.l_aux_group, ws, pl.l_aux_group), reinterpret_cast<int32_t*>(ws + pl.stats_group), l_aux,
+                       reinterpret_cast<long long*>(r.stats), st, shape->G);
+  if (rc != GSHARD_OK) return rc;
+  launch_dispatch(dl, x_local, slot_token, buf, st);
+
+  const int row_vec = (int)(l.row_bytes / 16);
+  const void* ffn_in = buf;
+  void* ffn_out = out;
+  if (world > 1) {
+    if (comm->all_to_all(comm->user, buf, xa, l.bytes_per_peer, cuda_stream) != 0) return GSHARD_ERR_CUDA;
+    launch_ep_regroup(xa, xb, world, l.experts_local, l.rows_local, row_vec, 0, st);
+    ffn_in = xb;
+    ffn_out = xa;
+  }
+  rc = ffn_stage(df, ffn_in, wi_local, wo_local, h, false, ffn_out, ws + pl.ffn_scratch, status, st, nullptr, nullptr);
+  if (rc != GSHARD_OK) return rc;
+  if (world > 1) {
+    launch_ep_regroup(xa, xb, world, l.experts_local, l.rows_local, row_vec, 1, st);
+    if (comm->all_to_all(comm->user, xb, out, l.bytes_per_peer, cuda_stream) != 0) return GSHARD_ERR_CUDA;
+    if (comm->all_reduce_sum_f32(comm->user, l_aux, 1, cuda_stream) != 0) return GSHARD_ERR_CUDA;
+  }
+  launch_combine(dl, out, expert_idx, slot, weight, y_local, st, dl.add_residual ? x_local : nullptr);
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+}  // extern "C"

@@ -32,7 +32,7 @@ int launch_gate_fused(const Dims& d, const void* x, const void* wg, float* logit
 int launch_capacity(const Dims& d, const int32_t* expert_idx, const float* gate12, const float* u, const float* m,
                     int32_t* slot, float* weight, uint8_t* flags, int32_t* first_count, int32_t* total_count,
                     int32_t* slot_token, float* l_aux_group, int32_t* stats_group, float* l_aux, long long* stats,
-                    cudaStream_t st);
+                    cudaStream_t st, int groups_in_mean = 0);
 int capacity_warps_for(int E);
 
 // dispatch_combine.cu

@@ -104,4 +104,16 @@ inline BwdPlan plan_backward(const Dims& d) {
 
 int validate_shape(const gshard_moe_shape* s);
 
+// api.cu: the stages as launch sequences, shared by the whole-layer, stage and expert-parallel calls.
+template <typename T> inline T* pick(T* user, unsigned char* ws, size_t off) {
+  return user ? user : reinterpret_cast<T*>(ws + off);
+}
+int gate_stage(const Dims& d, const FwdPlan& pl, unsigned char* ws, const void* x, const void* wg,
+               int32_t* expert_idx, float* gate12, float* m, float* rowmax, float* rowinv, cudaStream_t st);
+bool ffn_runs_fused(const Dims& d, bool keep_h);
+// With x / slot_token (only where ffn_runs_fused) the rows are gathered from x and buf is not read.
+int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
+              void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token);
+int check_device();
+
 }  // namespace gshard

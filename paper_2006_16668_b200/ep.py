@@ -1,0 +1,81 @@
+"""Expert-parallel forward over several GPUs, one process per GPU: the collectives of
+``gshard_moe_top2_forward_ep`` backed by ``torch.distributed`` (NCCL over NVLink on GPUs).
+
+The layer itself - gating, capacity, dispatch, the regrouping of received slabs, the expert FFN and
+the combine - runs inside the CUDA library; this module only hands it two callbacks that move bytes
+between ranks (Algorithm 2's AllToAll before and after the expert FFN, and the sum of the per-rank
+shares of l_aux) and slices each rank's share out of global tensors.
+"""
+from __future__ import annotations
+
+import traceback
+
+import torch
+import torch.distributed as dist
+
+from . import binding as B
+
+
+class TorchDistComm:
+    """A ``gshard_ep_comm`` whose all-to-all and all-reduce are torch.distributed collectives.
+
+    The library passes raw device pointers; they always point into the workspace of the call (or at
+    the l_aux scalar), so they are turned back into views of those tensors.  torch's NCCL collectives
+    order themselves after the current stream and make it wait for their completion, which is the
+    contract of the callbacks as long as the library call is made on torch's current stream.
+    """
+
+    def __init__(self, workspace: torch.Tensor, l_aux: torch.Tensor, group=None):
+        self.workspace, self.l_aux, self.group = workspace, l_aux, group
+        self.world = dist.get_world_size(group) if dist.is_initialized() else 1
+        self.error = None
+        self._a2a = B.ALL_TO_ALL_FN(self._all_to_all)        # keep the thunks alive
+        self._ar = B.ALL_REDUCE_FN(self._all_reduce)
+        self.struct = B.gshard_ep_comm(self._a2a, self._ar, None)
+
+    def _view(self, ptr: int, nbytes: int) -> torch.Tensor:
+        off = ptr - self.workspace.data_ptr()
+        if off < 0 or off + nbytes > self.workspace.numel():
+            raise ValueError("collective buffer outside the workspace")
+        return self.workspace[off:off + nbytes]
+
+    def _all_to_all(self, user, send, recv, bytes_per_peer, stream):
+        try:
+            n = bytes_per_peer * self.world
+            dist.all_to_all_single(self._view(recv, n), self._view(send, n), group=self.group)
+            return 0
+        except Exception:                                    # an exception must not cross the C frame
+            self.error = traceback.format_exc()
+            return 1
+
+    def _all_reduce(self, user, buf, count, stream):
+        try:
+            if buf != self.l_aux.data_ptr() or count > self.l_aux.numel():
+                raise ValueError("all-reduce buffer is not the l_aux tensor")
+            dist.all_reduce(self.l_aux[:count], op=dist.ReduceOp.SUM, group=self.group)
+            return 0
+        except Exception:
+            self.error = traceback.format_exc()
+            return 1
+
+
+def local_slices(layout: B.gshard_moe_ep_layout):
+    """(group slice, expert slice) of this rank in the global tensors."""
+    g0, e0 = layout.group_begin, layout.expert_begin
+    return slice(g0, g0 + layout.groups_local), slice(e0, e0 + layout.experts_local)
+
+
+def forward(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux, routing_out=None,
+            workspace=None, group=None):
+    """One expert-parallel forward on this rank (global `shape`); the process group must be
+    initialised when world > 1.  Enqueues on torch's current stream."""
+    comm = None
+    if world > 1:
+        comm = TorchDistComm(workspace, l_aux, group)
+    try:
+        B.gshard_moe_top2_forward_ep(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux,
+                                     routing_out, comm.struct if comm else None, workspace)
+    except B.GshardError:
+        if comm is not None and comm.error:
+            raise RuntimeError("a collective of the expert-parallel forward failed:\n" + comm.error)
+        raise

@@ -1,0 +1,204 @@
+"""gshard_moe_top2_forward_ep on one GPU.
+
+world = 1 must give the bits of gshard_moe_top2_forward.  For world = 2 and 4 the ranks are host
+threads of this process that share the GPU, each with its own stream, inputs slice and workspace,
+and the collectives are emulated on the host side: a rank's callback publishes its send buffer with
+an event, meets the others at a host barrier and copies its slabs out of their buffers on its own
+stream.  No kernel of one rank ever waits for a kernel of another (only streams wait on events), so
+sharing the GPU is safe; what is tested is everything inside the library call: local gating and
+capacity, the slab layout, the device-side regroup, the FFN over all groups' rows of the local
+experts, the way back and the combine.  y and the routing must equal the single-GPU layer bit for
+bit (whose parity with the oracle the other tests establish), l_aux to 1e-6 (the order of the sum
+over groups differs)."""
+import threading
+import traceback
+
+import pytest
+import torch
+
+from paper_2006_16668_b200 import MoEConfig, make_inputs
+from paper_2006_16668_b200 import binding as B
+from paper_2006_16668_b200 import ep
+
+pytestmark = pytest.mark.gpu
+
+
+def _single(cfg, inp, flags=0):
+    shape = B.make_shape(cfg, flags=flags)
+    ws = B.alloc_workspace(shape)
+    rt, rs = B.alloc_routing(shape)
+    y = torch.empty_like(inp["x"])
+    l_aux = torch.zeros(1, device="cuda")
+    B.gshard_moe_top2_forward(shape, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l_aux, rs, None, ws)
+    assert B.gshard_moe_last_device_status(ws) == B.GSHARD_OK
+    return y, l_aux, rt
+
+
+class _World:
+    def __init__(self, n):
+        self.n = n
+        self.barrier = threading.Barrier(n, timeout=60)
+        self.buf = [None] * n
+        self.ready = [None] * n
+        self.done = [None] * n
+
+
+class _ThreadComm:
+    """gshard_ep_comm for one emulated rank (a host thread with its own stream)."""
+
+    def __init__(self, world, rank, workspace, l_aux, stream):
+        self.w, self.rank, self.ws, self.l_aux, self.stream = world, rank, workspace, l_aux, stream
+        self.error = None
+        self._a2a = B.ALL_TO_ALL_FN(self._all_to_all)
+        self._ar = B.ALL_REDUCE_FN(self._all_reduce)
+        self.struct = B.gshard_ep_comm(self._a2a, self._ar, None)
+
+    def _view(self, ptr, n):
+        off = ptr - self.ws.data_ptr()
+        assert 0 <= off and off + n <= self.ws.numel()
+        return self.ws[off:off + n]
+
+    def _exchange(self, mine, consume):
+        """Publish `mine`, wait until every rank has published, run consume(all buffers) on this
+        rank's stream, and do not return before every rank has finished reading."""
+        w, r = self.w, self.rank
+        with torch.cuda.stream(self.stream):
+            ev = torch.cuda.Event()
+            ev.record(self.stream)
+            w.buf[r], w.ready[r] = mine, ev
+            w.barrier.wait()
+            for s in range(w.n):
+                self.stream.wait_event(w.ready[s])
+            result = consume(list(w.buf))
+            d = torch.cuda.Event()
+            d.record(self.stream)
+            w.done[r] = d
+            w.barrier.wait()
+            for s in range(w.n):
+                self.stream.wait_event(w.done[s])
+            w.barrier.wait()
+        return result
+
+    def _all_to_all(self, user, send, recv, bpp, stream):
+        try:
+            n, r = self.w.n, self.rank
+            recv_v = self._view(recv, bpp * n)
+
+            def consume(bufs):
+                for s in range(n):
+                    recv_v[s * bpp:(s + 1) * bpp].copy_(bufs[s][r * bpp:(r + 1) * bpp], non_blocking=True)
+            self._exchange(self._view(send, bpp * n), consume)
+            return 0
+        except Exception:
+            self.error = traceback.format_exc()
+            return 1
+
+    def _all_reduce(self, user, buf, count, stream):
+        try:
+            assert buf == self.l_aux.data_ptr() and count == 1
+            total = self._exchange(self.l_aux, lambda bufs: torch.stack([b.clone() for b in bufs]).sum(0))
+            with torch.cuda.stream(self.stream):
+                self.l_aux.copy_(total)
+            return 0
+        except Exception:
+            self.error = traceback.format_exc()
+            return 1
+
+
+def _run_ranks(cfg, inp, world, flags=0):
+    shape = B.make_shape(cfg, flags=flags)
+    state = _World(world)
+    results, errors = [None] * world, [None] * world
+
+    def rank_main(rank):
+        try:
+            torch.cuda.set_device(0)
+            lay = B.gshard_moe_ep_plan(shape, rank, world)
+            gs, es = ep.local_slices(lay)
+            stream = torch.cuda.Stream()
+            x, u = inp["x"][gs].contiguous(), inp["u"][gs].contiguous()
+            wi, wo = inp["wi"][es].contiguous(), inp["wo"][es].contiguous()
+            ws = torch.empty(B.gshard_moe_ep_workspace_bytes(shape, world), dtype=torch.uint8, device="cuda")
+            rt, rs = B.alloc_routing(lay.local)
+            y = torch.empty_like(x)
+            l_aux = torch.zeros(1, device="cuda")
+            torch.cuda.synchronize()
+            comm = _ThreadComm(state, rank, ws, l_aux, stream)
+            B.gshard_moe_top2_forward_ep(shape, rank, world, x, inp["wg"], wi, wo, u, y, l_aux, rs, comm.struct, ws,
+                                         stream)
+            assert comm.error is None, comm.error
+            assert B.gshard_moe_last_device_status(ws, stream) == B.GSHARD_OK
+            stream.synchronize()
+            results[rank] = (y, l_aux, rt)
+        except Exception:
+            errors[rank] = traceback.format_exc()
+            state.barrier.abort()
+
+    threads = [threading.Thread(target=rank_main, args=(r,)) for r in range(world)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=180)
+    assert not any(errors), "\n".join(e for e in errors if e)
+    assert all(r is not None for r in results)
+    return results
+
+
+CASES = [
+    # name, G, S, M, H, E, C, dtype, flags
+    ("f32", 4, 64, 32, 64, 8, 12, "f32", 0),
+    ("bf16_single_launch_ffn", 8, 256, 256, 1024, 32, 16, "bf16", 0),          # 128 rows per expert
+    ("bf16_cta_pairs", 8, 256, 256, 512, 16, 40, "bf16", 0),                   # 320 rows per expert
+    ("bf16_variant_a", 4, 384, 128, 256, 64, 10, "bf16", B.GSHARD_FLAG_SECOND_SKIP_FREES_SLOT),
+]
+
+
+@pytest.mark.parametrize("name,G,S,M,H,E,C,dtype,flags", CASES, ids=[c[0] for c in CASES])
+@pytest.mark.parametrize("world", [1, 2, 4])
+def test_expert_parallel_equals_single_gpu(world, name, G, S, M, H, E, C, dtype, flags):
+    cfg = MoEConfig(name, G=G, S=S, M=M, H=H, E=E, C=C, dtype=dtype, seed=4321)
+    inp = make_inputs(cfg, "cuda")
+    y_ref, l_ref, rt_ref = _single(cfg, inp, flags)
+    results = _run_ranks(cfg, inp, world, flags)
+    y = torch.cat([r[0] for r in results])
+    assert torch.equal(y.view(torch.uint8), y_ref.view(torch.uint8)), "y differs from the single-GPU layer"
+    for k in ("expert_idx", "slot", "weight", "flags", "first_count", "total_count", "m", "l_aux_group"):
+        got = torch.cat([r[2][k] for r in results])
+        assert torch.equal(got, rt_ref[k]), k
+    st = torch.cat([r[2]["slot_token"] for r in results], dim=1)             # [E, Gl, C] per rank -> [E, G, C]
+    assert torch.equal(st, rt_ref["slot_token"])
+    assert int(sum(int(r[2]["stats"][4]) for r in results)) == int(rt_ref["stats"][4])
+    for r in results:                                                          # the same l_aux on every rank
+        if world == 1:
+            assert torch.equal(r[1], l_ref)
+        else:
+            assert float(r[1]) == pytest.approx(float(l_ref), rel=1e-6)
+            assert torch.equal(r[1], results[0][1])
+
+
+def test_world_one_at_full_size_is_the_single_gpu_layer():
+    from paper_2006_16668_b200 import CONFIGS
+    cfg = CONFIGS["c3_512e_skew"]
+    inp = make_inputs(cfg, "cuda")
+    y_ref, l_ref, _ = _single(cfg, inp)
+    shape = B.make_shape(cfg)
+    ws = torch.empty(B.gshard_moe_ep_workspace_bytes(shape, 1), dtype=torch.uint8, device="cuda")
+    y = torch.empty_like(inp["x"])
+    l_aux = torch.zeros(1, device="cuda")
+    ep.forward(shape, 0, 1, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l_aux, None, ws)
+    assert B.gshard_moe_last_device_status(ws) == B.GSHARD_OK
+    assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16)) and torch.equal(l_aux, l_ref)
+
+
+def test_bad_arguments():
+    cfg = MoEConfig("bad", G=4, S=64, M=32, H=64, E=8, C=12, dtype="f32", seed=1)
+    shape = B.make_shape(cfg)
+    lib = B.load()
+    fake = 0x10000
+    import ctypes
+    args = [fake] * 6
+    assert lib.gshard_moe_top2_forward_ep(ctypes.byref(shape), 0, 3, *args, fake, None, None, fake, 1 << 40, None) == B.GSHARD_ERR_UNSUPPORTED_SHAPE
+    assert lib.gshard_moe_top2_forward_ep(ctypes.byref(shape), 2, 2, *args, fake, None, None, fake, 1 << 40, None) == B.GSHARD_ERR_INVALID_ARG
+    # world > 1 needs the collectives
+    assert lib.gshard_moe_top2_forward_ep(ctypes.byref(shape), 0, 2, *args, fake, None, None, fake, 1 << 40, None) == B.GSHARD_ERR_INVALID_ARG
+    assert lib.gshard_moe_top2_forward_ep(ctypes.byref(shape), 0, 1, *args, fake, None, None, fake, 16, None) == B.GSHARD_ERR_WORKSPACE_TOO_SMALL
