@@ -108,7 +108,20 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  that HBM sees reads and writes mixed.  Measured
                                                  slower than the default (one after another on all
                                                  multiprocessors); kept for measurement */
-#define GSHARD_FLAG_ALL 8191u
+#define GSHARD_FLAG_TF32_EXPERTS 8192u        /* dtype GSHARD_F32 only (ignored for bf16): the two expert
+                                                 FFN contractions of the forward run on the tensor cores
+                                                 with the fp32 operands read as TF32 (10-bit mantissa,
+                                                 fp32 accumulation), the way the paper's float32
+                                                 training would run on this hardware; gating, softmax,
+                                                 top-2 and the combine stay exact fp32, so the routing
+                                                 does not change.  y then agrees with the fp32 result to
+                                                 about 1e-3 relative instead of 1e-6.  The tensor core
+                                                 reads 32-bit operands only when they are contiguous
+                                                 along the contraction, which wi [E,M,H] and wo [E,H,M]
+                                                 are not: each call first writes transposed copies of
+                                                 both into the workspace (its size grows by their
+                                                 size) */
+#define GSHARD_FLAG_ALL 16383u
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,
@@ -337,11 +350,13 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
  * all tokens, no bias - eq. (2) with a single expert that sees every token, run by the same two
  * grouped tensor-core GEMMs as the expert FFN.
  *   x, y [n_tokens, M], wi [M, H], wo [H, M]: dtype (gshard_dtype); bf16 needs M % 64 == 0 and
- *   H % 64 == 0.  workspace: gshard_dense_ffn_workspace_bytes() bytes, 256-byte aligned; it holds a
+ *   H % 64 == 0.  flags: 0, or GSHARD_FLAG_TF32_EXPERTS (fp32 on the tensor cores),
+ *   GSHARD_FLAG_ONE_SM_MMA, GSHARD_FLAG_SIMT_CONTRACTIONS with their meaning above.
+ *   workspace: gshard_dense_ffn_workspace_bytes() bytes, 256-byte aligned; it holds a
  *   status word (read with gshard_moe_last_device_status) and the hidden activations [n_tokens, H]. */
 size_t gshard_dense_ffn_workspace_bytes(int64_t n_tokens, int32_t M, int32_t H, int32_t dtype);
-int gshard_dense_ffn_forward(int64_t n_tokens, int32_t M, int32_t H, int32_t dtype, const void* x,
-                             const void* wi, const void* wo, void* y, void* workspace,
+int gshard_dense_ffn_forward(int64_t n_tokens, int32_t M, int32_t H, int32_t dtype, uint32_t flags,
+                             const void* x, const void* wi, const void* wo, void* y, void* workspace,
                              size_t workspace_bytes, void* cuda_stream);
 
 /* Self-test of the give-up path shared by every bounded device-side wait (the paper has no

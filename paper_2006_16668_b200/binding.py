@@ -38,6 +38,7 @@ GSHARD_FLAG_ONE_SM_MMA = 512
 GSHARD_FLAG_ADD_RESIDUAL = 1024
 GSHARD_FLAG_CHAINED_FFN = 2048
 GSHARD_FLAG_BWD_PAIRED_GEMMS = 4096
+GSHARD_FLAG_TF32_EXPERTS = 8192
 
 
 class gshard_moe_shape(Structure):
@@ -96,7 +97,7 @@ EXPORTS = {
                                    [POINTER(gshard_moe_routing), POINTER(gshard_ep_comm), c_void_p, c_size_t,
                                     c_void_p]),
     "gshard_dense_ffn_workspace_bytes": (c_size_t, [ctypes.c_int64, c_int32, c_int32, c_int32]),
-    "gshard_dense_ffn_forward": (c_int, [ctypes.c_int64, c_int32, c_int32, c_int32] + [c_void_p] * 5 +
+    "gshard_dense_ffn_forward": (c_int, [ctypes.c_int64, c_int32, c_int32, c_int32, c_uint32] + [c_void_p] * 5 +
                                  [c_size_t, c_void_p]),
     "gshard_moe_debug_wait_timeout": (c_int, [c_void_p, c_uint32, c_void_p]),
     "gshard_moe_last_device_status": (c_int, [c_void_p, c_void_p]),
@@ -322,11 +323,11 @@ def gshard_dense_ffn_workspace_bytes(n_tokens, M, H, dtype_code) -> int:
     return int(load().gshard_dense_ffn_workspace_bytes(int(n_tokens), int(M), int(H), int(dtype_code)))
 
 
-def gshard_dense_ffn_forward(x, wi, wo, y, workspace, stream=None):
+def gshard_dense_ffn_forward(x, wi, wo, y, workspace, stream=None, flags=0):
     """y = relu(x . wi) . wo for x [n, M], wi [M, H], wo [H, M] (the dense Transformer FFN)."""
     n, M = x.shape
     H = wi.shape[1]
-    _check(load().gshard_dense_ffn_forward(n, M, H, _dtype_code(x), _p(x), _p(wi), _p(wo), _p(y), _p(workspace),
+    _check(load().gshard_dense_ffn_forward(n, M, H, _dtype_code(x), flags, _p(x), _p(wi), _p(wo), _p(y), _p(workspace),
                                            workspace.numel(), _stream(stream)), "gshard_dense_ffn_forward")
 
 

@@ -94,7 +94,8 @@ bool ffn_runs_fused(const Dims& d, bool keep_h) {
 
 // With x / slot_token (only where ffn_runs_fused) the rows are gathered from x and buf is not read.
 int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
-              void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token) {
+              void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token,
+              void* wt) {
   const long long rows = d.rows;
   // One persistent launch in which the hidden activations never leave L2: the faster form when
   // the FFN is bound by streaming the expert weights (at most one 128-row tile per expert); with
@@ -116,12 +117,22 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   g.a_kmajor = true; g.b_kmajor = false;
   g.a_ld = d.M; g.a_bs = rows * d.M; g.b_ld = d.H; g.b_bs = (long long)d.M * d.H; g.c_ld = d.H; g.c_bs = rows * d.H;
   g.relu = 1; g.b_stream = 1; g.prefer_two_sm = 1;
-  GS_TRY(run_gemm(d, g, status, st));
   UmmaGemm g2{};
   g2.A = h; g2.B = wo; g2.C = out; g2.rows = d.rows; g2.cols = d.M; g2.K = d.H; g2.batch = d.E;
   g2.a_kmajor = true; g2.b_kmajor = false;
   g2.a_ld = d.H; g2.a_bs = rows * d.H; g2.b_ld = d.M; g2.b_bs = (long long)d.H * d.M; g2.c_ld = d.M; g2.c_bs = rows * d.M;
   g2.b_stream = 1; g2.prefer_two_sm = 1;
+  if (d.tf32_experts && wt) {
+    // The tensor core reads 32-bit operands K-major only, and the weights are contiguous along the
+    // other dimension: transposed copies first (wi[e] [M,H] -> [H,M], wo[e] [H,M] -> [M,H]).
+    float* wi_t = static_cast<float*>(wt);
+    float* wo_t = wi_t + (size_t)d.E * d.M * d.H;
+    launch_transpose_f32(static_cast<const float*>(wi), wi_t, d.E, d.M, d.H, st);
+    launch_transpose_f32(static_cast<const float*>(wo), wo_t, d.E, d.H, d.M, st);
+    g.B = wi_t; g.b_kmajor = true; g.b_ld = d.M; g.tf32 = 1; g.out_f32 = 1;
+    g2.B = wo_t; g2.b_kmajor = true; g2.b_ld = d.H; g2.tf32 = 1; g2.out_f32 = 1;
+  }
+  GS_TRY(run_gemm(d, g, status, st));
   return run_gemm(d, g2, status, st);
 }
 
@@ -193,7 +204,8 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
   FfnTiming& ft = ffn_timing();
   const bool timed = ft.start != nullptr && ft.stop != nullptr;
   if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.start), st) != cudaSuccess) return GSHARD_ERR_CUDA;
-  GS_TRY(ffn_stage(d, buf, wi, wo, h, save, out, ws + pl.ffn_scratch, status, st, gather ? x : nullptr, slot_token));
+  GS_TRY(ffn_stage(d, buf, wi, wo, h, save, out, ws + pl.ffn_scratch, status, st, gather ? x : nullptr, slot_token,
+                   ws + pl.wt));
   if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.stop), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   ft.start = ft.stop = nullptr;
   launch_combine(d, out, expert_idx, slot, weight, y, st, d.add_residual ? x : nullptr);
@@ -426,7 +438,7 @@ int gshard_moe_expert_ffn(const gshard_moe_shape* shape, const void* buf, const 
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   if (cudaMemsetAsync(ws + pl.status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   GS_TRY(ffn_stage(d, buf, wi, wo, ws + pl.h, false, out, ws + pl.ffn_scratch,
-                   reinterpret_cast<int*>(ws + pl.status), st, nullptr, nullptr));
+                   reinterpret_cast<int*>(ws + pl.status), st, nullptr, nullptr, ws + pl.wt));
   return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
@@ -445,12 +457,17 @@ size_t gshard_dense_ffn_workspace_bytes(int64_t n_tokens, int32_t M, int32_t H, 
   if (dtype != GSHARD_F32 && dtype != GSHARD_BF16) return 0;
   if (dtype == GSHARD_BF16 && (M % 64 || H % 64)) return 0;
   if (dtype == GSHARD_F32 && (n_tokens + 63) / 64 > 65535) return 0;
-  return kAlign + align_up((size_t)n_tokens * H * (dtype == GSHARD_BF16 ? 2 : 4));
+  // status word, hidden activations, and (fp32, for the TF32 option) the transposed weights
+  return kAlign + align_up((size_t)n_tokens * H * (dtype == GSHARD_BF16 ? 2 : 4)) +
+         (dtype == GSHARD_F32 ? align_up(2 * (size_t)M * H * 4) : 0);
 }
 
-int gshard_dense_ffn_forward(int64_t n_tokens, int32_t M, int32_t H, int32_t dtype, const void* x, const void* wi,
-                             const void* wo, void* y, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+int gshard_dense_ffn_forward(int64_t n_tokens, int32_t M, int32_t H, int32_t dtype, uint32_t flags, const void* x,
+                             const void* wi, const void* wo, void* y, void* workspace, size_t workspace_bytes,
+                             void* cuda_stream) {
   launch_counter().n = 0;
+  if (flags & ~(GSHARD_FLAG_TF32_EXPERTS | GSHARD_FLAG_ONE_SM_MMA | GSHARD_FLAG_SIMT_CONTRACTIONS))
+    return GSHARD_ERR_INVALID_ARG;
   const size_t need = gshard_dense_ffn_workspace_bytes(n_tokens, M, H, dtype);
   if (need == 0) return (n_tokens <= 0 || M <= 0 || H <= 0) ? GSHARD_ERR_INVALID_ARG : GSHARD_ERR_UNSUPPORTED_SHAPE;
   GS_REQUIRE_PTR(x); GS_REQUIRE_PTR(wi); GS_REQUIRE_PTR(wo); GS_REQUIRE_PTR(y); GS_REQUIRE_PTR(workspace);
@@ -463,7 +480,7 @@ int gshard_dense_ffn_forward(int64_t n_tokens, int32_t M, int32_t H, int32_t dty
   if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   // the expert FFN's two grouped GEMMs with a single problem of n_tokens rows
   gshard_moe_shape one{};
-  one.G = 1; one.S = 1; one.C = 1; one.E = 2; one.M = M; one.H = H; one.dtype = dtype;
+  one.G = 1; one.S = 1; one.C = 1; one.E = 2; one.M = M; one.H = H; one.dtype = dtype; one.flags = flags;
   Dims d = make_dims(one);
   d.rows = (int)n_tokens;
   void* h = ws + kAlign;
@@ -471,11 +488,19 @@ int gshard_dense_ffn_forward(int64_t n_tokens, int32_t M, int32_t H, int32_t dty
   g.A = x; g.B = wi; g.C = h; g.rows = d.rows; g.cols = H; g.K = M; g.batch = 1;
   g.a_kmajor = true; g.b_kmajor = false; g.a_ld = M; g.b_ld = H; g.c_ld = H;
   g.relu = 1; g.a_stream = 1; g.prefer_two_sm = 1;
-  GS_TRY(run_gemm(d, g, status, st));
   UmmaGemm g2{};
   g2.A = h; g2.B = wo; g2.C = y; g2.rows = d.rows; g2.cols = M; g2.K = H; g2.batch = 1;
   g2.a_kmajor = true; g2.b_kmajor = false; g2.a_ld = H; g2.b_ld = M; g2.c_ld = M;
   g2.a_stream = 1; g2.prefer_two_sm = 1;
+  if (d.tf32_experts) {          // K-major (transposed) copies of the weights, as in the expert FFN
+    float* wi_t = reinterpret_cast<float*>(ws + kAlign + align_up((size_t)n_tokens * H * 4));
+    float* wo_t = wi_t + (size_t)M * H;
+    launch_transpose_f32(static_cast<const float*>(wi), wi_t, 1, M, H, st);
+    launch_transpose_f32(static_cast<const float*>(wo), wo_t, 1, H, M, st);
+    g.B = wi_t; g.b_kmajor = true; g.b_ld = M; g.tf32 = 1; g.out_f32 = 1;
+    g2.B = wo_t; g2.b_kmajor = true; g2.b_ld = H; g2.tf32 = 1; g2.out_f32 = 1;
+  }
+  GS_TRY(run_gemm(d, g, status, st));
   GS_TRY(run_gemm(d, g2, status, st));
   return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }

@@ -101,6 +101,7 @@ struct Dims {
   bool gate_one_sm;     // stored-logits gating kernel on single CTAs instead of CTA pairs
   bool gate_cluster;    // gating on clusters with the mean-gate partial sums fused in (no stored logits)
   bool gather_dispatch; // single-launch FFN gathers its rows from x instead of reading a dispatch buffer
+  bool tf32_experts;    // fp32 dtype: expert FFN contractions on the tensor cores in TF32
   bool bwd_paired;      // backward: read-heavy and write-heavy expert GEMMs side by side on half of the SMs each
 };
 
@@ -125,6 +126,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.add_residual = (s.flags & GSHARD_FLAG_ADD_RESIDUAL) != 0;
   d.chained_ffn = (s.flags & GSHARD_FLAG_CHAINED_FFN) != 0;
   d.bwd_paired = (s.flags & GSHARD_FLAG_BWD_PAIRED_GEMMS) != 0;
+  d.tf32_experts = !d.bf16 && (s.flags & GSHARD_FLAG_TF32_EXPERTS) != 0;
   return d;
 }
 

@@ -84,6 +84,32 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
   }
 }
 
+// Batched fp32 matrix transpose through a padded 32 x 32 shared-memory tile (coalesced both ways).
+__global__ void __launch_bounds__(256) transpose_f32_kernel(const float* __restrict__ src, float* __restrict__ dst,
+                                                            int rows, int cols) {
+  __shared__ float tile[32][33];
+  const long long base = (long long)blockIdx.z * rows * cols;
+  const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;          // 32 x 8 threads
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int r = r0 + ty + 8 * i, c = c0 + tx;
+    if (r < rows && c < cols) tile[ty + 8 * i][tx] = src[base + (long long)r * cols + c];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int c = c0 + ty + 8 * i, r = r0 + tx;
+    if (r < rows && c < cols) dst[base + (long long)c * rows + r] = tile[tx][ty + 8 * i];
+  }
+}
+
+void launch_transpose_f32(const float* src, float* dst, int batch, int rows, int cols, cudaStream_t st) {
+  const dim3 grid(ceil_div(cols, 32), ceil_div(rows, 32), batch);
+  transpose_f32_kernel<<<grid, 256, 0, st>>>(src, dst, rows, cols);
+  count_launch();
+}
+
 void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st) {
   const int row_vec = (int)((size_t)d.M * d.esize / 16);
   dispatch_kernel<<<grid_for_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(x), slot_token,

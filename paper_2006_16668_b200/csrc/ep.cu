@@ -183,7 +183,8 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
     ffn_in = xb;
     ffn_out = xa;
   }
-  rc = ffn_stage(df, ffn_in, wi_local, wo_local, h, false, ffn_out, ws + pl.ffn_scratch, status, st, nullptr, nullptr);
+  rc = ffn_stage(df, ffn_in, wi_local, wo_local, h, false, ffn_out, ws + pl.ffn_scratch, status, st, nullptr, nullptr,
+                 ws + pl.wt);
   if (rc != GSHARD_OK) return rc;
   if (world > 1) {
     launch_ep_regroup(xa, xb, world, l.experts_local, l.rows_local, row_vec, 1, st);

@@ -14,12 +14,15 @@ inline int run_gemm(const Dims& d, const UmmaGemm& g, int* status, cudaStream_t 
     // holds its tensor pipe near 65 %.  Callers mark the GEMMs that measured faster on pairs (the two
     // forward expert GEMMs); the flags force either form everywhere.  A single row tile would leave
     // the second CTA of a pair without rows.
+    if (g.tf32) return GSHARD_ERR_INTERNAL;   // bf16 operands cannot be read as TF32
     if (g.rows > 128 && !d.one_sm_mma && (d.two_sm_mma || g.prefer_two_sm)) {
       const int rc = launch_umma2_gemm(g, status, st);
       if (rc == GSHARD_OK) return rc;       // a refused cluster launch ran nothing: single CTAs take over
     }
     return launch_umma_gemm(g, status, st);
   }
+  // fp32 dtype with the TF32 option: the GEMMs marked by their caller run on the tensor cores
+  if (!d.bf16 && d.tf32_experts && g.tf32) return launch_umma_gemm(g, status, st);
   SimtGemm s{};
   s.A = g.A; s.B = g.B; s.C = g.C; s.mask = g.mask;
   s.rows = g.rows; s.cols = g.cols; s.K = g.K; s.batch = g.batch;

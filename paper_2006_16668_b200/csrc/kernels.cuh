@@ -40,6 +40,9 @@ void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, vo
 void launch_combine(const Dims& d, const void* out, const int32_t* expert_idx, const int32_t* slot,
                     const float* weight, void* y, cudaStream_t st, const void* residual = nullptr);
 
+// dispatch_combine.cu: dst[b][c][r] = src[b][r][c] for a batch of fp32 matrices [rows, cols].
+void launch_transpose_f32(const float* src, float* dst, int batch, int rows, int cols, cudaStream_t st);
+
 // umma_gemm.cu: batched bf16 GEMM on tcgen05, C[b] = act(A[b] . B[b]).
 struct UmmaGemm {
   const void* A; const void* B; void* C;
@@ -54,6 +57,8 @@ struct UmmaGemm {
   int relu;
   int a_stream, b_stream;    // operand is read once: load with an evict-first L2 hint
   int prefer_two_sm;         // run on CTA pairs (cta_group::2) when a problem has more than 128 rows
+  int tf32;                  // A and B hold float: contraction on the tensor cores in TF32 (both operands
+                             // K-major, float output)
   int max_ctas;              // > 0: use at most this many CTAs (persistent grid), leaving the other
                              // multiprocessors to a kernel running beside this one on another stream
 };

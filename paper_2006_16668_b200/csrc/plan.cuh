@@ -14,7 +14,7 @@ struct Carver {
 
 struct FwdPlan {
   size_t status, logits, rowmax, rowinv, partial, gate12, m, expert_idx, slot, weight, flags, first_count,
-      total_count, slot_token, l_aux_group, stats_group, ffn_scratch, buf, h, out, total;
+      total_count, slot_token, l_aux_group, stats_group, ffn_scratch, buf, h, out, wt, total;
 };
 
 inline FwdPlan plan_forward(const Dims& d) {
@@ -42,6 +42,8 @@ inline FwdPlan plan_forward(const Dims& d) {
   p.buf = c.take(R * d.M * d.esize);
   p.h = c.take(R * d.H * d.esize);
   p.out = c.take(R * d.M * d.esize);
+  // TF32 expert contractions: transposed copies of both weight tensors (K-major B operands)
+  p.wt = c.take(d.tf32_experts ? 2 * (size_t)d.E * d.M * d.H * 4 : 0);
   p.total = c.off;
   return p;
 }
@@ -112,8 +114,10 @@ int gate_stage(const Dims& d, const FwdPlan& pl, unsigned char* ws, const void* 
                int32_t* expert_idx, float* gate12, float* m, float* rowmax, float* rowinv, cudaStream_t st);
 bool ffn_runs_fused(const Dims& d, bool keep_h);
 // With x / slot_token (only where ffn_runs_fused) the rows are gathered from x and buf is not read.
+// wt: with d.tf32_experts, room for the transposed copies of wi and wo (2 * E * M * H floats).
 int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
-              void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token);
+              void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token,
+              void* wt = nullptr);
 int check_device();
 
 }  // namespace gshard

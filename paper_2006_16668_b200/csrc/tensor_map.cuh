@@ -25,15 +25,17 @@ inline EncodeTiledFn encode_fn() {
 // 3-D bf16 tensor map {inner, outer, batch} with a {box_inner, box_outer, 1} box, 128-byte swizzle;
 // out-of-range elements read as zero.  ld_elems / bs_elems: elements between consecutive outer
 // rows / batches.
+// esize 2: bfloat16 elements; esize 4: float elements (the box's inner extent stays 128 bytes).
 inline bool make_map(CUtensorMap* map, const void* base, long long inner, long long outer, long long batch,
-                     long long ld_elems, long long bs_elems, int box_inner, int box_outer) {
+                     long long ld_elems, long long bs_elems, int box_inner, int box_outer, int esize = 2) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[3] = {(cuuint64_t)inner, (cuuint64_t)outer, (cuuint64_t)batch};
-  cuuint64_t strides[2] = {(cuuint64_t)ld_elems * 2, (cuuint64_t)(batch > 1 ? bs_elems : ld_elems * outer) * 2};
+  cuuint64_t strides[2] = {(cuuint64_t)ld_elems * esize, (cuuint64_t)(batch > 1 ? bs_elems : ld_elems * outer) * esize};
   cuuint32_t box[3] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(map, esize == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3,
+            const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }

@@ -65,7 +65,11 @@ __device__ __forceinline__ TileCoord decode(const Params& p, int tile) {
   return t;
 }
 
-template <bool A_K, bool B_K, int BN, bool MASK>
+// TF32: A and B hold fp32 values that the tensor core reads as TF32 (K-major operands only: with a
+// 32-bit MN-major operand the instruction returns zeros).  A shared-memory row is still 128 bytes,
+// i.e. 32 elements: a k-block is 32 deep and an MMA contracts 8; stage sizes in bytes are those of
+// the bf16 form.
+template <bool A_K, bool B_K, int BN, bool MASK, bool TF32 = false>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                  const Params p) {
@@ -81,6 +85,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int BKE = TF32 ? 32 : 64;                  // elements per k-block (128 bytes)
+  constexpr int kBoxMN = TF32 ? 32 : 64;               // MN extent of one box of an MN-major operand
+  constexpr int kBoxB = kBoxMN * BKE * (TF32 ? 4 : 2); // its bytes
+  constexpr int kStepMN = TF32 ? 1024 : 2048;          // bytes of the K rows one MMA contracts (8 or 16 x 128)
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C_::stages; ++s) { ptx::mbar_init(full + s, 1); ptx::mbar_init(empty + s, 1); }
@@ -114,18 +122,18 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
           unsigned char* sb = sa + kABytes;
           ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)C_::stage_bytes);
           if (A_K) {
-            ptx::tma_load_3d(sa, &map_a, full + stage, kb * BK, t.mt * BM, t.b, pol_a);
+            ptx::tma_load_3d(sa, &map_a, full + stage, kb * BKE, t.mt * BM, t.b, pol_a);
           } else {
 #pragma unroll
-            for (int j = 0; j < BM / 64; ++j)
-              ptx::tma_load_3d(sa + j * kBoxBytes, &map_a, full + stage, t.mt * BM + j * 64, kb * BK, t.b, pol_a);
+            for (int j = 0; j < BM / kBoxMN; ++j)
+              ptx::tma_load_3d(sa + j * kBoxB, &map_a, full + stage, t.mt * BM + j * kBoxMN, kb * BKE, t.b, pol_a);
           }
           if (B_K) {
-            ptx::tma_load_3d(sb, &map_b, full + stage, kb * BK, t.nt * BN, t.b, pol_b);
+            ptx::tma_load_3d(sb, &map_b, full + stage, kb * BKE, t.nt * BN, t.b, pol_b);
           } else {
 #pragma unroll
-            for (int j = 0; j < BN / 64; ++j)
-              ptx::tma_load_3d(sb + j * kBoxBytes, &map_b, full + stage, t.nt * BN + j * 64, kb * BK, t.b, pol_b);
+            for (int j = 0; j < BN / kBoxMN; ++j)
+              ptx::tma_load_3d(sb + j * kBoxB, &map_b, full + stage, t.nt * BN + j * kBoxMN, kb * BKE, t.b, pol_b);
           }
           if (++stage == C_::stages) { stage = 0; phase ^= 1u; }
         }
@@ -134,7 +142,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------------------
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::make_idesc_bf16(BM, BN, !A_K, !B_K);
+      constexpr uint32_t idesc = TF32 ? ptx::make_idesc_tf32(BM, BN, !A_K, !B_K) : ptx::make_idesc_bf16(BM, BN, !A_K, !B_K);
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
       for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
@@ -147,12 +155,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
           const uint32_t sa = ptx::smem_u32(smem + stage * C_::stage_bytes);
           const uint32_t sb = sa + kABytes;
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
+          for (int k = 0; k < 4; ++k) {              // 4 MMAs per k-block: 4 x 16 bf16 or 4 x 8 tf32
             const uint64_t da = A_K ? ptx::make_smem_desc(sa + k * 32, 16, 1024)
-                                    : ptx::make_smem_desc(sa + k * 2048, kBoxBytes, 1024);
+                                    : ptx::make_smem_desc(sa + k * kStepMN, kBoxB, 1024);
             const uint64_t db = B_K ? ptx::make_smem_desc(sb + k * 32, 16, 1024)
-                                    : ptx::make_smem_desc(sb + k * 2048, kBoxBytes, 1024);
-            ptx::umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+                                    : ptx::make_smem_desc(sb + k * kStepMN, kBoxB, 1024);
+            if (TF32) ptx::umma_tf32(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
+            else ptx::umma_bf16(d_tmem, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
           }
           ptx::umma_commit(empty + stage);           // stage reusable once these MMAs have read it
           if (++stage == C_::stages) { stage = 0; phase ^= 1u; }
@@ -363,9 +372,9 @@ umma_gemm_resident_b_kernel(const __grid_constant__ CUtensorMap map_a, const __g
 
 // ---- host side ------------------------------------------------------------------------------
 
-template <bool A_K, bool B_K, int BN, bool MASK>
+template <bool A_K, bool B_K, int BN, bool MASK, bool TF32 = false>
 int launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int grid, cudaStream_t st) {
-  auto kern = umma_gemm_kernel<A_K, B_K, BN, MASK>;
+  auto kern = umma_gemm_kernel<A_K, B_K, BN, MASK, TF32>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::smem_bytes) != cudaSuccess)
     return GSHARD_ERR_CUDA;
   kern<<<grid, kThreads, Cfg<BN>::smem_bytes, st>>>(ma, mb, p);
@@ -379,26 +388,31 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (g.rows <= 0 || g.cols <= 0 || g.K <= 0 || g.batch <= 0) return GSHARD_OK;
   if (g.mask && g.out_f32) return GSHARD_ERR_INTERNAL;   // the mask is staged as bf16 rows
   const int BN = g.cols > 128 ? 256 : 128;
+  // fp32 operands read as TF32: the tensor core takes 32-bit operands K-major only (an MN-major
+  // one yields zeros), so both operands must be contiguous along the contraction
+  if (g.tf32 && (!g.a_kmajor || !g.b_kmajor || g.mask || !g.out_f32)) return GSHARD_ERR_INTERNAL;
+  const int esz = g.tf32 ? 4 : 2;
+  const int bke = 128 / esz;                     // elements per 128-byte k-block row
   CUtensorMap ma, mb;
   bool okm;
-  if (g.a_kmajor) okm = make_map(&ma, g.A, g.K, g.rows, g.batch, g.a_ld, g.a_bs, BK, BM);
-  else            okm = make_map(&ma, g.A, g.rows, g.K, g.batch, g.a_ld, g.a_bs, 64, BK);
-  if (g.b_kmajor) okm = okm && make_map(&mb, g.B, g.K, g.cols, g.batch, g.b_ld, g.b_bs, BK, BN);
-  else            okm = okm && make_map(&mb, g.B, g.cols, g.K, g.batch, g.b_ld, g.b_bs, 64, BK);
+  if (g.a_kmajor) okm = make_map(&ma, g.A, g.K, g.rows, g.batch, g.a_ld, g.a_bs, bke, BM, esz);
+  else            okm = make_map(&ma, g.A, g.rows, g.K, g.batch, g.a_ld, g.a_bs, bke, bke, esz);
+  if (g.b_kmajor) okm = okm && make_map(&mb, g.B, g.K, g.cols, g.batch, g.b_ld, g.b_bs, bke, BN, esz);
+  else            okm = okm && make_map(&mb, g.B, g.cols, g.K, g.batch, g.b_ld, g.b_bs, bke, bke, esz);
   if (!okm) return GSHARD_ERR_CUDA;
   Params p;
   p.C = g.C; p.mask = g.mask; p.rows = g.rows; p.cols = g.cols; p.K = g.K; p.batch = g.batch;
   p.c_ld = g.c_ld; p.c_bs = g.c_bs;
   p.m_tiles = ceil_div(g.rows, BM); p.n_tiles = ceil_div(g.cols, BN);
   p.total_tiles = p.m_tiles * p.n_tiles * g.batch;
-  p.k_blocks = ceil_div(g.K, BK);
+  p.k_blocks = ceil_div(g.K, bke);
   p.out_f32 = g.out_f32; p.relu = g.relu; p.a_stream = g.a_stream; p.b_stream = g.b_stream;
   // stream the larger operand once: walk the tiles that share it back to back
   p.n_fastest = (g.rows > g.cols) ? 1 : 0;
   p.status = status;
   int sms = device_sms();
   if (g.max_ctas > 0 && sms > g.max_ctas) sms = g.max_ctas;
-  if (!g.a_kmajor && !g.b_kmajor && !g.mask && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
+  if (!g.tf32 && !g.a_kmajor && !g.b_kmajor && !g.mask && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
     // short contraction, several row tiles per column block: keep the B tile resident
     const int n_groups = p.n_tiles * g.batch;
     if (cudaFuncSetAttribute(umma_gemm_resident_b_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -409,6 +423,9 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
     return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
   }
   const int grid = p.total_tiles < sms ? p.total_tiles : sms;
+  if (g.tf32)
+    return BN == 256 ? launch_t<true, true, 256, false, true>(ma, mb, p, grid, st)
+                     : launch_t<true, true, 128, false, true>(ma, mb, p, grid, st);
 #define GSHARD_DISPATCH(AK, BKM)                                                                    \
   (p.mask ? (BN == 256 ? launch_t<AK, BKM, 256, true>(ma, mb, p, grid, st)                          \
                        : launch_t<AK, BKM, 128, true>(ma, mb, p, grid, st))                         \

@@ -33,6 +33,27 @@ def test_dense_ffn_against_oracle(n, M, H, dtype):
     assert err < (1e-5 if dtype == "f32" else 1e-2), err
 
 
+@pytest.mark.parametrize("n,M,H", [(50, 64, 256), (300, 40, 72), (1000, 256, 1024), (4100, 1024, 2048)])
+def test_dense_ffn_tf32_against_oracle(n, M, H):
+    """fp32 tensors with both contractions on the tensor cores in TF32: within 1e-2 of the oracle
+    (the achieved error, a few 1e-4, is printed), and much closer to it than bf16 would be."""
+    gen = torch.Generator(device="cuda").manual_seed(n + M + 1)
+    x = torch.randn(n, M, generator=gen, device="cuda")
+    wi = torch.randn(M, H, generator=gen, device="cuda") * M ** -0.5
+    wo = torch.randn(H, M, generator=gen, device="cuda") * H ** -0.5
+    y = torch.empty_like(x)
+    ws = torch.empty(B.gshard_dense_ffn_workspace_bytes(n, M, H, B.GSHARD_F32), dtype=torch.uint8, device="cuda")
+    B.gshard_dense_ffn_forward(x, wi, wo, y, ws, flags=B.GSHARD_FLAG_TF32_EXPERTS)
+    assert B.gshard_moe_last_device_status(ws) == B.GSHARD_OK
+    assert B.gshard_moe_last_launch_count() == 4          # two weight transposes, two tensor-core GEMMs
+    rows = np.unique(np.concatenate([np.arange(min(n, 40)), np.arange(max(0, n - 40), n),
+                                     np.random.default_rng(n).integers(0, n, 64)]))
+    ref = orc.ffn_rows(to_np(x)[rows], to_np(wi), to_np(wo))
+    err = rel_fro(to_np(y)[rows], ref)
+    print(f"\n[dense FFN tf32 n={n} M={M} H={H}] rel. Frobenius error {err:.3e}")
+    assert 1e-6 < err < 2e-3, err
+
+
 def test_dense_ffn_full_size_sampled_rows():
     """The adjacent Transformer layer's FFN at the MoE(2048E) batch: 131072 tokens, M=1024, H=8192."""
     n, M, H = 131072, 1024, 8192
@@ -57,7 +78,7 @@ def test_dense_ffn_bad_arguments():
     assert B.gshard_dense_ffn_workspace_bytes(8, 60, 64, B.GSHARD_F32) == 0
     assert B.gshard_dense_ffn_workspace_bytes(8, 72, 64, B.GSHARD_BF16) == 0
     fake = 0x10000
-    assert lib.gshard_dense_ffn_forward(0, 64, 64, 0, fake, fake, fake, fake, fake, 1 << 30, None) == B.GSHARD_ERR_INVALID_ARG
-    assert lib.gshard_dense_ffn_forward(8, 72, 64, 1, fake, fake, fake, fake, fake, 1 << 30, None) == B.GSHARD_ERR_UNSUPPORTED_SHAPE
-    assert lib.gshard_dense_ffn_forward(8, 64, 64, 0, fake, fake, None, fake, fake, 1 << 30, None) == B.GSHARD_ERR_INVALID_ARG
-    assert lib.gshard_dense_ffn_forward(8, 64, 64, 0, fake, fake, fake, fake, fake, 16, None) == B.GSHARD_ERR_WORKSPACE_TOO_SMALL
+    assert lib.gshard_dense_ffn_forward(0, 64, 64, 0, 0, fake, fake, fake, fake, fake, 1 << 30, None) == B.GSHARD_ERR_INVALID_ARG
+    assert lib.gshard_dense_ffn_forward(8, 72, 64, 1, 0, fake, fake, fake, fake, fake, 1 << 30, None) == B.GSHARD_ERR_UNSUPPORTED_SHAPE
+    assert lib.gshard_dense_ffn_forward(8, 64, 64, 0, 0, fake, fake, None, fake, fake, 1 << 30, None) == B.GSHARD_ERR_INVALID_ARG
+    assert lib.gshard_dense_ffn_forward(8, 64, 64, 0, 0, fake, fake, fake, fake, fake, 16, None) == B.GSHARD_ERR_WORKSPACE_TOO_SMALL
