@@ -403,12 +403,16 @@ class Bench:
         ffn_bytes, ffn_flops = ffn_work(cfg.M, cfg.H, cfg.E, rows, es)
         fused = (cfg.dtype == "bf16" and not self.train and
                  (args.fused_ffn or (not args.unfused_ffn and rows <= 128)))
-        pairs = rows > 128 and not args.one_sm_mma
+        compact = (args.flags & 16384) or (rows >= 768 and not (args.one_sm_mma or args.two_sm_mma or args.chained_ffn
+                                                            or args.fused_ffn or self.train))
+        pairs = rows > 128 and not args.one_sm_mma and not compact
         if fused:
             kernel, label, n_launch = "ffn_group4_kernel", "expert FFN, both GEMMs in 1 launch", 1
         else:
             kernel = "umma2_gemm_kernel" if pairs else "umma_gemm_kernel"
             label, n_launch = "expert FFN, 2 grouped-GEMM launches (sum of both)", 2
+            if compact:
+                label += ", compacted slots: only row tiles that hold kept rows"
         roof = kernel_roofline(ffn_bytes, ffn_flops, rec["ffn_ms"], peaks)
         roof.update({"kernel": f"{kernel} ({label})", "launches_per_step": n_launch, "launch_ms": rec["ffn_ms"] / n_launch,
                      "algorithmic_bytes": ffn_bytes, "algorithmic_flops": ffn_flops,

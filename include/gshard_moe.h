@@ -121,7 +121,20 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  are not: each call first writes transposed copies of
                                                  both into the workspace (its size grows by their
                                                  size) */
-#define GSHARD_FLAG_ALL 16383u
+#define GSHARD_FLAG_COMPACT_SLOTS 16384u      /* forward, bf16, grouped-GEMM form of the expert FFN
+                                                 (more than 128 rows per expert): the filled slots of
+                                                 each expert are compacted to the front of its block,
+                                                 the GEMMs run only the 128-row tiles that hold kept
+                                                 rows (13 to 30 % of the slots are empty at the
+                                                 paper's shapes), empty rows are neither zero-filled
+                                                 nor multiplied, and the combine finds its rows through
+                                                 the compaction index.  Kept rows get the same bits.
+                                                 This is already the default where an expert has 768
+                                                 rows or more (unless ONE_SM_MMA, TWO_SM_MMA, FUSED_FFN
+                                                 or CHAINED_FFN names another form); the flag extends it
+                                                 to fewer rows.  Ignored with SAVE_FOR_BACKWARD and
+                                                 where the single-launch FFN runs */
+#define GSHARD_FLAG_ALL 32767u
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

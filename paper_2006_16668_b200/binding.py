@@ -39,6 +39,7 @@ GSHARD_FLAG_ADD_RESIDUAL = 1024
 GSHARD_FLAG_CHAINED_FFN = 2048
 GSHARD_FLAG_BWD_PAIRED_GEMMS = 4096
 GSHARD_FLAG_TF32_EXPERTS = 8192
+GSHARD_FLAG_COMPACT_SLOTS = 16384
 
 
 class gshard_moe_shape(Structure):

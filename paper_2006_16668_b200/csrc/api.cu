@@ -95,7 +95,7 @@ bool ffn_runs_fused(const Dims& d, bool keep_h) {
 // With x / slot_token (only where ffn_runs_fused) the rows are gathered from x and buf is not read.
 int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
               void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token,
-              void* wt) {
+              void* wt, const int* tile_base) {
   const long long rows = d.rows;
   // One persistent launch in which the hidden activations never leave L2: the faster form when
   // the FFN is bound by streaming the expert weights (at most one 128-row tile per expert); with
@@ -104,11 +104,11 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   // Both single-launch forms need their whole grid resident at once and are launched cooperatively;
   // when the runtime refuses that (GSHARD_ERR_UNSUPPORTED_SHAPE, nothing launched) the two
   // grouped-GEMM launches below take over.
-  if (ffn_runs_fused(d, keep_h)) {
+  if (!tile_base && ffn_runs_fused(d, keep_h)) {
     const int rc = launch_ffn_fused(d, buf, wi, wo, fused_scratch, out, status, st, x, slot_token);
     if (rc != GSHARD_ERR_UNSUPPORTED_SHAPE) return rc;
     if (x) launch_dispatch(d, x, slot_token, const_cast<void*>(buf), st);   // rows were to be gathered in the launch
-  } else if (d.chained_ffn && ffn_chained_supported(d)) {
+  } else if (!tile_base && d.chained_ffn && ffn_chained_supported(d)) {
     const int rc = launch_ffn_chained(d, buf, wi, wo, h, out, fused_scratch, status, st);
     if (rc != GSHARD_ERR_UNSUPPORTED_SHAPE) return rc;
   }
@@ -122,6 +122,12 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   g2.a_kmajor = true; g2.b_kmajor = false;
   g2.a_ld = d.H; g2.a_bs = rows * d.H; g2.b_ld = d.M; g2.b_bs = (long long)d.H * d.M; g2.c_ld = d.M; g2.c_bs = rows * d.M;
   g2.b_stream = 1; g2.prefer_two_sm = 1;
+  if (tile_base) {
+    // compacted rows: each expert's row-tile count comes from the device-side prefix; 128-row tiles on
+    // single CTAs (a 256-row pair tile would round the kept rows up further)
+    g.tile_base = tile_base; g.prefer_two_sm = 0;
+    g2.tile_base = tile_base; g2.prefer_two_sm = 0;
+  }
   if (d.tf32_experts && wt) {
     // The tensor core reads 32-bit operands K-major only, and the weights are contiguous along the
     // other dimension: transposed copies first (wi[e] [M,H] -> [H,M], wo[e] [H,M] -> [M,H]).
@@ -199,16 +205,27 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
   GS_TRY(launch_capacity(d, expert_idx, gate12, u, m, slot, weight, flags, first_count, total_count, slot_token,
                          l_aux_group, stats_group, l_aux, reinterpret_cast<long long*>(r.stats), st));
   const bool gather = d.gather_dispatch && ffn_runs_fused(d, save);
-  if (!gather) launch_dispatch(d, x, slot_token, buf, st);
+  // compacted slots apply to the grouped-GEMM form of the FFN only
+  const bool compact = d.compact_slots && !ffn_runs_fused(d, save);
+  int32_t* crow_token = reinterpret_cast<int32_t*>(ws + pl.crow_token);
+  int32_t* slot_crow = reinterpret_cast<int32_t*>(ws + pl.slot_crow);
+  int32_t* kept = reinterpret_cast<int32_t*>(ws + pl.kept);
+  int32_t* tile_base = reinterpret_cast<int32_t*>(ws + pl.tile_base);
+  if (compact) {
+    launch_compact(d, slot_token, crow_token, slot_crow, kept, tile_base, st);
+    launch_dispatch_compact(d, x, crow_token, kept, buf, st);
+  } else if (!gather) {
+    launch_dispatch(d, x, slot_token, buf, st);
+  }
   // optional event pair around the expert FFN, armed for one call by gshard_moe_time_expert_ffn
   FfnTiming& ft = ffn_timing();
   const bool timed = ft.start != nullptr && ft.stop != nullptr;
   if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.start), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   GS_TRY(ffn_stage(d, buf, wi, wo, h, save, out, ws + pl.ffn_scratch, status, st, gather ? x : nullptr, slot_token,
-                   ws + pl.wt));
+                   ws + pl.wt, compact ? tile_base : nullptr));
   if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.stop), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   ft.start = ft.stop = nullptr;
-  launch_combine(d, out, expert_idx, slot, weight, y, st, d.add_residual ? x : nullptr);
+  launch_combine(d, out, expert_idx, slot, weight, y, st, d.add_residual ? x : nullptr, compact ? slot_crow : nullptr);
 
   if (save) {   // hand the caller the routing tensors it asked for
     struct { void* dst; const void* src; size_t n; } cps[] = {

@@ -41,7 +41,8 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
                                                       const float* __restrict__ weight,
                                                       const uint4* __restrict__ residual,
                                                       uint4* __restrict__ y, long long N, int G, int S,
-                                                      int C, int E, int row_vec) {
+                                                      int C, int E, int row_vec,
+                                                      const int32_t* __restrict__ slot_crow) {
   constexpr int n = Vec16<T>::n;
   const int lane = threadIdx.x & 31;
   const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -52,8 +53,13 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
     const float w0 = weight[2 * t], w1 = weight[2 * t + 1];
     const int x0 = expert_idx[2 * t], x1 = expert_idx[2 * t + 1];
     const bool k0 = s0 >= 0 && s0 < C && x0 >= 0 && x0 < E, k1 = s1 >= 0 && s1 < C && x1 >= 0 && x1 < E;
-    const uint4* r0 = k0 ? out + (((long long)x0 * G + g) * C + s0) * row_vec : nullptr;
-    const uint4* r1 = k1 ? out + (((long long)x1 * G + g) * C + s1) * row_vec : nullptr;
+    long long row0 = k0 ? ((long long)x0 * G + g) * C + s0 : 0, row1 = k1 ? ((long long)x1 * G + g) * C + s1 : 0;
+    if (slot_crow) {                      // outputs stored by compacted row within the expert's block
+      if (k0) row0 = (long long)x0 * G * C + slot_crow[row0];
+      if (k1) row1 = (long long)x1 * G * C + slot_crow[row1];
+    }
+    const uint4* r0 = k0 ? out + row0 * row_vec : nullptr;
+    const uint4* r1 = k1 ? out + row1 * row_vec : nullptr;
     uint4* dst = y + t * row_vec;
     // four 16-byte pieces per lane and row at a time, every load issued before the first use (the
     // rows are scattered in HBM)
@@ -110,6 +116,34 @@ void launch_transpose_f32(const float* src, float* dst, int batch, int rows, int
   count_launch();
 }
 
+// Dispatch into compacted rows: row j of expert e is the token crow_token[e, j] (j < kept[e]).
+__global__ void __launch_bounds__(256) dispatch_compact_kernel(const uint4* __restrict__ x,
+                                                               const int32_t* __restrict__ crow_token,
+                                                               const int32_t* __restrict__ kept,
+                                                               uint4* __restrict__ buf, long long R, int rows,
+                                                               long long N, int row_vec) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long r = warp; r < R; r += nwarps) {
+    const int e = (int)(r / rows), j = (int)(r % rows);
+    if (j >= kept[e]) continue;
+    const long long t = crow_token[r];
+    if (t < 0 || t >= N) continue;
+    const uint4* src = x + t * row_vec;
+    uint4* dst = buf + r * row_vec;
+    for (int i = lane; i < row_vec; i += 32) dst[i] = __ldg(src + i);
+  }
+}
+
+void launch_dispatch_compact(const Dims& d, const void* x, const int32_t* crow_token, const int32_t* kept, void* buf,
+                             cudaStream_t st) {
+  const int row_vec = (int)((size_t)d.M * d.esize / 16);
+  dispatch_compact_kernel<<<grid_for_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(x), crow_token, kept,
+                                                              reinterpret_cast<uint4*>(buf), d.R, d.rows, d.N, row_vec);
+  count_launch();
+}
+
 void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st) {
   const int row_vec = (int)((size_t)d.M * d.esize / 16);
   dispatch_kernel<<<grid_for_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(x), slot_token,
@@ -118,16 +152,16 @@ void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, vo
 }
 
 void launch_combine(const Dims& d, const void* out, const int32_t* expert_idx, const int32_t* slot,
-                    const float* weight, void* y, cudaStream_t st, const void* residual) {
+                    const float* weight, void* y, cudaStream_t st, const void* residual, const int32_t* slot_crow) {
   const int row_vec = (int)((size_t)d.M * d.esize / 16);
   if (d.bf16)
     combine_kernel<__nv_bfloat16><<<grid_for_rows(d.N), 256, 0, st>>>(
         reinterpret_cast<const uint4*>(out), expert_idx, slot, weight, reinterpret_cast<const uint4*>(residual),
-        reinterpret_cast<uint4*>(y), d.N, d.G, d.S, d.C, d.E, row_vec);
+        reinterpret_cast<uint4*>(y), d.N, d.G, d.S, d.C, d.E, row_vec, slot_crow);
   else
     combine_kernel<float><<<grid_for_rows(d.N), 256, 0, st>>>(
         reinterpret_cast<const uint4*>(out), expert_idx, slot, weight, reinterpret_cast<const uint4*>(residual),
-        reinterpret_cast<uint4*>(y), d.N, d.G, d.S, d.C, d.E, row_vec);
+        reinterpret_cast<uint4*>(y), d.N, d.G, d.S, d.C, d.E, row_vec, slot_crow);
   count_launch();
 }
 

@@ -15,7 +15,7 @@ inline int run_gemm(const Dims& d, const UmmaGemm& g, int* status, cudaStream_t 
     // forward expert GEMMs); the flags force either form everywhere.  A single row tile would leave
     // the second CTA of a pair without rows.
     if (g.tf32) return GSHARD_ERR_INTERNAL;   // bf16 operands cannot be read as TF32
-    if (g.rows > 128 && !d.one_sm_mma && (d.two_sm_mma || g.prefer_two_sm)) {
+    if (g.rows > 128 && !g.tile_base && !d.one_sm_mma && (d.two_sm_mma || g.prefer_two_sm)) {
       const int rc = launch_umma2_gemm(g, status, st);
       if (rc == GSHARD_OK) return rc;       // a refused cluster launch ran nothing: single CTAs take over
     }

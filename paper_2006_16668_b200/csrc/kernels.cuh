@@ -37,8 +37,20 @@ int capacity_warps_for(int E);
 
 // dispatch_combine.cu
 void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st);
+// slot_crow (optional): the expert outputs are stored by compacted row; slot_crow[e, g*C+c] is the row.
 void launch_combine(const Dims& d, const void* out, const int32_t* expert_idx, const int32_t* slot,
-                    const float* weight, void* y, cudaStream_t st, const void* residual = nullptr);
+                    const float* weight, void* y, cudaStream_t st, const void* residual = nullptr,
+                    const int32_t* slot_crow = nullptr);
+
+// compact.cu: per expert, the filled slots in (group, position) order become rows 0 .. kept-1.
+//   crow_token [E, G*C]  global token index (g*S + s) of compacted row j, j < kept[e]
+//   slot_crow  [E, G*C]  compacted row of slot (g, c), or -1 for an empty slot
+//   kept [E], tile_base [E+1]: exclusive prefix of ceil(kept / 128)
+void launch_compact(const Dims& d, const int32_t* slot_token, int32_t* crow_token, int32_t* slot_crow, int32_t* kept,
+                    int32_t* tile_base, cudaStream_t st);
+// buf[e, j, :] = x[crow_token[e, j], :] for j < kept[e]; other rows are left untouched
+void launch_dispatch_compact(const Dims& d, const void* x, const int32_t* crow_token, const int32_t* kept, void* buf,
+                             cudaStream_t st);
 
 // dispatch_combine.cu: dst[b][c][r] = src[b][r][c] for a batch of fp32 matrices [rows, cols].
 void launch_transpose_f32(const float* src, float* dst, int batch, int rows, int cols, cudaStream_t st);
@@ -59,6 +71,8 @@ struct UmmaGemm {
   int prefer_two_sm;         // run on CTA pairs (cta_group::2) when a problem has more than 128 rows
   int tf32;                  // A and B hold float: contraction on the tensor cores in TF32 (both operands
                              // K-major, float output)
+  const int* tile_base;      // ragged batch (device pointer, batch + 1 ints): problem b has
+                             // tile_base[b+1] - tile_base[b] row tiles of 128 rows; single-CTA kernel only
   int max_ctas;              // > 0: use at most this many CTAs (persistent grid), leaving the other
                              // multiprocessors to a kernel running beside this one on another stream
 };

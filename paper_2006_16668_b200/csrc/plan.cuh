@@ -14,7 +14,8 @@ struct Carver {
 
 struct FwdPlan {
   size_t status, logits, rowmax, rowinv, partial, gate12, m, expert_idx, slot, weight, flags, first_count,
-      total_count, slot_token, l_aux_group, stats_group, ffn_scratch, buf, h, out, wt, total;
+      total_count, slot_token, l_aux_group, stats_group, ffn_scratch, buf, h, out, wt, crow_token, slot_crow, kept,
+      tile_base, total;
 };
 
 inline FwdPlan plan_forward(const Dims& d) {
@@ -44,6 +45,11 @@ inline FwdPlan plan_forward(const Dims& d) {
   p.out = c.take(R * d.M * d.esize);
   // TF32 expert contractions: transposed copies of both weight tensors (K-major B operands)
   p.wt = c.take(d.tf32_experts ? 2 * (size_t)d.E * d.M * d.H * 4 : 0);
+  // compacted slots: row lists both ways, kept counts, row-tile prefix
+  p.crow_token = c.take(d.compact_slots ? R * 4 : 0);
+  p.slot_crow = c.take(d.compact_slots ? R * 4 : 0);
+  p.kept = c.take(d.compact_slots ? (size_t)d.E * 4 : 0);
+  p.tile_base = c.take(d.compact_slots ? ((size_t)d.E + 1) * 4 : 0);
   p.total = c.off;
   return p;
 }
@@ -117,7 +123,7 @@ bool ffn_runs_fused(const Dims& d, bool keep_h);
 // wt: with d.tf32_experts, room for the transposed copies of wi and wo (2 * E * M * H floats).
 int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
               void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token,
-              void* wt = nullptr);
+              void* wt = nullptr, const int* tile_base = nullptr);
 int check_device();
 
 }  // namespace gshard

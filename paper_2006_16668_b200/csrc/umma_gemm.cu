@@ -55,15 +55,35 @@ struct Params {
   int a_stream, b_stream;
   int n_fastest;   // tile order: column tiles fastest (A is the larger operand) instead of row tiles
   int* status;
+  // Ragged batches (compacted expert rows): problem b owns the row tiles [tile_base[b], tile_base[b+1])
+  // of a device-side prefix array with batch + 1 entries; nullptr = every problem has m_tiles row tiles.
+  const int* tile_base;
 };
 
-__device__ __forceinline__ TileCoord decode(const Params& p, int tile) {
-  TileCoord t;
-  t.mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
-  t.nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
-  t.b = tile / (p.m_tiles * p.n_tiles);
-  return t;
-}
+// Tile index -> (row tile, column tile, problem).  A thread walks its tiles in increasing order, so
+// for ragged batches it keeps the problem index of its last tile and moves forward from there
+// instead of searching the prefix array.
+struct TileWalk {
+  int b = 0;
+  __device__ __forceinline__ int total(const Params& p) const {
+    return p.tile_base ? __ldg(p.tile_base + p.batch) * p.n_tiles : p.total_tiles;
+  }
+  __device__ __forceinline__ TileCoord decode(const Params& p, int tile) {
+    TileCoord t;
+    if (p.tile_base) {
+      while (b + 1 < p.batch && __ldg(p.tile_base + b + 1) * p.n_tiles <= tile) ++b;
+      const int first = __ldg(p.tile_base + b);
+      const int m_b = __ldg(p.tile_base + b + 1) - first;           // row tiles of this problem (>= 1 here)
+      const int i = tile - first * p.n_tiles;
+      t.mt = i % m_b; t.nt = i / m_b; t.b = b;                      // row tiles fastest: they share the B tile
+      return t;
+    }
+    t.mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
+    t.nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
+    t.b = tile / (p.m_tiles * p.n_tiles);
+    return t;
+  }
+};
 
 // TF32: A and B hold fp32 values that the tensor core reads as TF32 (K-major operands only: with a
 // 32-bit MN-major operand the instruction returns zeros).  A shared-memory row is still 128 bytes,
@@ -114,8 +134,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       const uint64_t pol_a = p.a_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
       const uint64_t pol_b = p.b_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
       int stage = 0; uint32_t phase = 0;
-      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-        const TileCoord t = decode(p, tile);
+      TileWalk walk;
+      const int total_tiles = walk.total(p);
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+        const TileCoord t = walk.decode(p, tile);
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!ptx::mbar_wait(empty + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
           unsigned char* sa = smem + stage * C_::stage_bytes;
@@ -145,7 +167,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       constexpr uint32_t idesc = TF32 ? ptx::make_idesc_tf32(BM, BN, !A_K, !B_K) : ptx::make_idesc_bf16(BM, BN, !A_K, !B_K);
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
-      for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
+      const int total_tiles = TileWalk().total(p);
+      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         if (!ptx::mbar_wait(acc_empty + acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
@@ -178,8 +201,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int half = ew >> 2;                        // which half of the tile's columns
     unsigned char* stg = smem + C_::stg_off + ew * kStgWarpBytes;
     int acc = 0; uint32_t acc_phase = 0;
-    for (int tile = blockIdx.x; tile < p.total_tiles && ok; tile += gridDim.x) {
-      const TileCoord t = decode(p, tile);
+    TileWalk walk;
+    const int total_tiles = walk.total(p);
+    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+      const TileCoord t = walk.decode(p, tile);
       uint4 mreg[MASK ? 8 : 1];
       if (MASK) load_mask_block(p, t.b, t.mt * BM + q * 32, round_col0<BN>(t, half, 0), lane, mreg);
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
@@ -410,9 +435,12 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   // stream the larger operand once: walk the tiles that share it back to back
   p.n_fastest = (g.rows > g.cols) ? 1 : 0;
   p.status = status;
+  p.tile_base = g.tile_base;
+  if (g.tile_base && g.tf32) return GSHARD_ERR_INTERNAL;
+  if (g.tile_base) p.n_fastest = 0;            // ragged lists are walked with the row tiles fastest
   int sms = device_sms();
   if (g.max_ctas > 0 && sms > g.max_ctas) sms = g.max_ctas;
-  if (!g.tf32 && !g.a_kmajor && !g.b_kmajor && !g.mask && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
+  if (!g.tf32 && !g.tile_base && !g.a_kmajor && !g.b_kmajor && !g.mask && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
     // short contraction, several row tiles per column block: keep the B tile resident
     const int n_groups = p.n_tiles * g.batch;
     if (cudaFuncSetAttribute(umma_gemm_resident_b_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -422,7 +450,7 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
     count_launch();
     return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
   }
-  const int grid = p.total_tiles < sms ? p.total_tiles : sms;
+  const int grid = (p.total_tiles < sms && !g.tile_base) ? p.total_tiles : sms;   // ragged: count known on the device only
   if (g.tf32)
     return BN == 256 ? launch_t<true, true, 256, false, true>(ma, mb, p, grid, st)
                      : launch_t<true, true, 128, false, true>(ma, mb, p, grid, st);

@@ -143,6 +143,12 @@ SMALL = [
     # 160 rows per expert: expert GEMMs on CTA pairs (default) and on single CTAs
     ("bf16_two_sm_default", 2, 512, 256, 512, 16, 80, "bf16", 0),
     ("bf16_one_sm_forced", 2, 512, 256, 512, 16, 80, "bf16", B.GSHARD_FLAG_ONE_SM_MMA),
+    # compacted slots: ragged row-tile lists (160 slots per expert, about 100 of them filled), and a
+    # shape where some experts keep nothing
+    ("bf16_compact_slots", 2, 512, 256, 512, 16, 80, "bf16", B.GSHARD_FLAG_COMPACT_SLOTS),
+    ("bf16_compact_slots_four_tiles", 4, 1024, 128, 256, 16, 150, "bf16", B.GSHARD_FLAG_COMPACT_SLOTS),
+    ("bf16_compact_slots_by_default", 8, 512, 128, 256, 16, 100, "bf16", 0),
+    ("bf16_compact_slots_sparse", 3, 64, 128, 256, 64, 50, "bf16", B.GSHARD_FLAG_COMPACT_SLOTS),
     # far more experts than tokens per group (16 column tiles in the gating kernel, almost all experts empty)
     ("bf16_many_experts", 2, 96, 64, 64, 4096, 1, "bf16", 0),
     # gating on clusters with the mean-gate partial sums fused in (no stored logits)
@@ -188,6 +194,30 @@ def test_gather_dispatch_matches_dispatch_buffer_bitwise():
     y_g, l_g, rt_g = run_forward(cfg, inp, B.GSHARD_FLAG_GATHER_DISPATCH)
     assert torch.equal(y_b.view(torch.int16), y_g.view(torch.int16)) and torch.equal(l_b, l_g)
     assert torch.equal(rt_b["slot_token"], rt_g["slot_token"])
+
+
+def test_compact_slots_matches_dispatch_buffer_bitwise():
+    # a kept row meets the same MMAs whether its tile also holds empty rows or not
+    cfg = MoEConfig("cs", G=4, S=1024, M=256, H=1024, E=16, C=100, dtype="bf16", seed=80)
+    inp = make_inputs(cfg, "cuda")
+    y_b, l_b, rt_b = run_forward(cfg, inp, B.GSHARD_FLAG_ONE_SM_MMA)
+    y_c, l_c, rt_c = run_forward(cfg, inp, B.GSHARD_FLAG_COMPACT_SLOTS)
+    assert torch.equal(y_b.view(torch.int16), y_c.view(torch.int16)) and torch.equal(l_b, l_c)
+    for k in rt_b:
+        assert torch.equal(rt_b[k], rt_c[k]), k
+    assert 0.3 < int(rt_c["stats"][4]) / (cfg.E * cfg.G * cfg.C) < 0.98      # some slots are empty
+
+
+@pytest.mark.parametrize("name", ["c2_128e", "c3_512e_skew"])
+def test_compact_slots_full_size(name):
+    """Paper-shaped layers with compacted slots: bitwise the single-CTA grouped-GEMM form, and the
+    oracle on two groups' routing and sampled tokens."""
+    cfg = CONFIGS[name]
+    inp = make_inputs(cfg, "cuda")
+    y_c, l_c, rt_c = run_forward(cfg, inp, B.GSHARD_FLAG_COMPACT_SLOTS)
+    check_forward(cfg, inp, y_c, l_c, rt_c, [0, cfg.G - 1], 6)
+    y_b, l_b, _ = run_forward(cfg, inp, B.GSHARD_FLAG_ONE_SM_MMA)
+    assert torch.equal(y_b.view(torch.int16), y_c.view(torch.int16)) and torch.equal(l_b, l_c)
 
 
 def test_gather_dispatch_full_size_bitwise():
