@@ -403,8 +403,8 @@ class Bench:
         ffn_bytes, ffn_flops = ffn_work(cfg.M, cfg.H, cfg.E, rows, es)
         fused = (cfg.dtype == "bf16" and not self.train and
                  (args.fused_ffn or (not args.unfused_ffn and rows <= 128)))
-        compact = (args.flags & 16384) or (rows >= 768 and not (args.one_sm_mma or args.two_sm_mma or args.chained_ffn
-                                                            or args.fused_ffn or self.train))
+        compact = (args.flags & 16384) or (rows >= 768 and not (args.one_sm_mma or args.two_sm_mma or args.fused_ffn
+                                                            or self.train))
         pairs = rows > 128 and not args.one_sm_mma and not compact
         if fused:
             kernel, label, n_launch = "ffn_group4_kernel", "expert FFN, both GEMMs in 1 launch", 1
@@ -527,7 +527,6 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra-configs", action="store_true", help="measure only --config")
     ap.add_argument("--sustained-seconds", type=float, default=2.0, help="0 skips the sustained run")
-    ap.add_argument("--chained-ffn", action="store_true", help="both expert GEMMs in one launch (rows > 128)")
     ap.add_argument("--one-sm-mma", action="store_true", help="ablation: no grouped GEMM on CTA pairs")
     ap.add_argument("--gate-one-sm", action="store_true", help="ablation: gating GEMM on single CTAs, row-major logits")
     ap.add_argument("--gate-cluster", action="store_true",
@@ -575,8 +574,7 @@ def main():
              (B.GSHARD_FLAG_GATHER_DISPATCH if args.gather_dispatch else 0) |
              (B.GSHARD_FLAG_GATE_CLUSTER if args.gate_cluster else 0) |
              (B.GSHARD_FLAG_GATE_ONE_SM if args.gate_one_sm else 0) |
-             (B.GSHARD_FLAG_ONE_SM_MMA if args.one_sm_mma else 0) |
-             (B.GSHARD_FLAG_CHAINED_FFN if args.chained_ffn else 0) | args.flags)
+             (B.GSHARD_FLAG_ONE_SM_MMA if args.one_sm_mma else 0) | args.flags)
 
     sampler = ClockSampler(local_rank)
     sampler.start()

@@ -63,10 +63,10 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  handed over through L2, never written to HBM) where
                                                  the shape allows it; by default it is used when an
                                                  expert has at most 128 rows */
-/* The single-launch forms (FUSED_FFN, its GATHER_DISPATCH mode, CHAINED_FFN) are persistent grids
- * whose CTAs wait on one another, one CTA per multiprocessor.  They are launched cooperatively: the
- * runtime starts them only when the whole grid can be resident, so work of other streams that holds
- * multiprocessors delays them instead of breaking them; if the runtime refuses the launch, the two
+/* The single-launch form (FUSED_FFN and its GATHER_DISPATCH mode) is a persistent grid whose CTAs
+ * wait on one another, one CTA per multiprocessor.  It is launched cooperatively: the runtime
+ * starts it only when the whole grid can be resident, so work of other streams that holds
+ * multiprocessors delays it instead of breaking it; if the runtime refuses the launch, the two
  * grouped-GEMM launches run instead. */
 #define GSHARD_FLAG_UNFUSED_FFN 16u           /* force the two grouped-GEMM launches instead (hidden
                                                  activations make a round trip through HBM) */
@@ -98,10 +98,7 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  overflowed tokens pass through it) folded into the
                                                  combine; backward: dx also receives dy.  Not applied
                                                  by the stage call gshard_moe_combine */
-#define GSHARD_FLAG_CHAINED_FFN 2048u         /* experts with more than 128 rows: both expert GEMMs in
-                                                 one persistent launch of CTA pairs, GEMM-2 reading
-                                                 the hidden activations from L2 (they are still written
-                                                 once) */
+/* bit 2048 is not in use */
 #define GSHARD_FLAG_BWD_PAIRED_GEMMS 4096u    /* backward: the GEMM that computes dh runs beside the one
                                                  for dwo, and dbuf beside dwi, each on half of the
                                                  multiprocessors (second, library-owned stream), so
@@ -130,11 +127,11 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  nor multiplied, and the combine finds its rows through
                                                  the compaction index.  Kept rows get the same bits.
                                                  This is already the default where an expert has 768
-                                                 rows or more (unless ONE_SM_MMA, TWO_SM_MMA, FUSED_FFN
-                                                 or CHAINED_FFN names another form); the flag extends it
+                                                 rows or more (unless ONE_SM_MMA, TWO_SM_MMA or FUSED_FFN
+                                                 names another form); the flag extends it
                                                  to fewer rows.  Ignored with SAVE_FOR_BACKWARD and
                                                  where the single-launch FFN runs */
-#define GSHARD_FLAG_ALL 32767u
+#define GSHARD_FLAG_ALL (32767u & ~2048u)
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

@@ -16,7 +16,7 @@
  * the caller) and every sum is accumulated in double.  There is no blocking,
  * fusion or reordering beyond what the paper's steps state.
  *
- * Readings where the paper is silent (all listed in the design notes):
+ * Readings where the paper is silent:
  *   - top_2 ties: the lowest expert index wins, for both picks.
  *   - the pass-2 counters continue from the (unclipped) pass-1 counts;
  *     Algorithm 1 initialises c_E once.

@@ -101,16 +101,13 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   // the FFN is bound by streaming the expert weights (at most one 128-row tile per expert); with
   // more rows per expert the two grouped-GEMM launches keep the tensor pipe busier.  Not available
   // when the caller keeps h for the backward pass.
-  // Both single-launch forms need their whole grid resident at once and are launched cooperatively;
-  // when the runtime refuses that (GSHARD_ERR_UNSUPPORTED_SHAPE, nothing launched) the two
-  // grouped-GEMM launches below take over.
+  // The single-launch form needs its whole grid resident at once and is launched cooperatively; when
+  // the runtime refuses that (GSHARD_ERR_UNSUPPORTED_SHAPE, nothing launched) the two grouped-GEMM
+  // launches below take over.
   if (!tile_base && ffn_runs_fused(d, keep_h)) {
     const int rc = launch_ffn_fused(d, buf, wi, wo, fused_scratch, out, status, st, x, slot_token);
     if (rc != GSHARD_ERR_UNSUPPORTED_SHAPE) return rc;
     if (x) launch_dispatch(d, x, slot_token, const_cast<void*>(buf), st);   // rows were to be gathered in the launch
-  } else if (!tile_base && d.chained_ffn && ffn_chained_supported(d)) {
-    const int rc = launch_ffn_chained(d, buf, wi, wo, h, out, fused_scratch, status, st);
-    if (rc != GSHARD_ERR_UNSUPPORTED_SHAPE) return rc;
   }
   UmmaGemm g{};
   g.A = buf; g.B = wi; g.C = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;

@@ -95,7 +95,6 @@ struct Dims {
   bool fused_ffn;       // force the single-launch FFN (h handed over through L2)
   bool unfused_ffn;     // force the two grouped-GEMM launches (h through HBM)
   bool two_sm_mma;      // grouped GEMMs on CTA pairs (tcgen05 cta_group::2) where rows > 128
-  bool chained_ffn;     // more than 128 rows per expert: both GEMMs in one launch, h consumed from L2
   bool add_residual;    // y = x + layer(x); dx gains dy
   bool one_sm_mma;      // never use CTA pairs for the grouped GEMMs
   bool gate_one_sm;     // stored-logits gating kernel on single CTAs instead of CTA pairs
@@ -125,7 +124,6 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.gate_one_sm = (s.flags & GSHARD_FLAG_GATE_ONE_SM) != 0;
   d.one_sm_mma = (s.flags & GSHARD_FLAG_ONE_SM_MMA) != 0;
   d.add_residual = (s.flags & GSHARD_FLAG_ADD_RESIDUAL) != 0;
-  d.chained_ffn = (s.flags & GSHARD_FLAG_CHAINED_FFN) != 0;
   d.bwd_paired = (s.flags & GSHARD_FLAG_BWD_PAIRED_GEMMS) != 0;
   d.tf32_experts = !d.bf16 && (s.flags & GSHARD_FLAG_TF32_EXPERTS) != 0;
   // Compacted slots: on request, and by default where an expert has at least six 128-row tiles, so
@@ -133,8 +131,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   // 3.68 against 3.74 ms for a burst of steps, 4.08 against 4.62 ms sustained under the power cap; at
   // 256 rows per expert nothing is saved and the CTA-pair GEMM is faster).  A flag that names
   // another GEMM form switches the default off.
-  const bool other_form = (s.flags & (GSHARD_FLAG_ONE_SM_MMA | GSHARD_FLAG_TWO_SM_MMA | GSHARD_FLAG_CHAINED_FFN |
-                                      GSHARD_FLAG_FUSED_FFN)) != 0;
+  const bool other_form = (s.flags & (GSHARD_FLAG_ONE_SM_MMA | GSHARD_FLAG_TWO_SM_MMA | GSHARD_FLAG_FUSED_FFN)) != 0;
   d.compact_slots = d.bf16 && !d.simt && !(s.flags & GSHARD_FLAG_SAVE_FOR_BACKWARD) &&
                     ((s.flags & GSHARD_FLAG_COMPACT_SLOTS) != 0 || (d.rows >= 768 && !other_form));
   return d;

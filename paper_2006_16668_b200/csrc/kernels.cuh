@@ -90,12 +90,4 @@ int launch_ffn_fused(const Dims& d, const void* buf, const void* wi, const void*
                      int* status, cudaStream_t st, const void* x_gather = nullptr,
                      const int32_t* slot_token = nullptr);
 
-// ffn_chained.cu: both expert GEMMs in one persistent launch of CTA pairs for experts with more than
-// 128 rows; GEMM-2 tiles wait on per-expert counters and read h while it is still in L2.  h is
-// written in full (the caller may keep it).  scratch: ffn_chained_scratch_bytes, zeroed by the call.
-bool ffn_chained_supported(const Dims& d);
-size_t ffn_chained_scratch_bytes(const Dims& d);
-int launch_ffn_chained(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, void* out,
-                       void* scratch, int* status, cudaStream_t st);
-
 }  // namespace gshard

@@ -122,11 +122,6 @@ FFN_CASES = [
     (2, 2, 100, 1024, 2048, "bf16", 0),          # 200 rows: ragged second row tile
     (3, 1, 24, 192, 448, "bf16", 0),             # fewer rows than a tile, ragged column tile
     (1, 4, 96, 512, 1024, "bf16", 0),            # 384 rows
-    # both GEMMs chained in one launch (GEMM-2 waits on per-expert counters)
-    (2, 2, 100, 1024, 2048, "bf16", B.GSHARD_FLAG_CHAINED_FFN),   # 200 rows: ragged second CTA
-    (5, 8, 128, 256, 1536, "bf16", B.GSHARD_FLAG_CHAINED_FFN),    # 1024 rows: four row tiles per expert
-    (150, 2, 80, 256, 2048, "bf16", B.GSHARD_FLAG_CHAINED_FFN),   # 150 experts in three waves
-    (3, 4, 96, 448, 1088, "bf16", B.GSHARD_FLAG_CHAINED_FFN),     # ragged column tiles in both GEMMs
     # more than 128 rows run on CTA pairs by default: the same shapes on single CTAs
     (2, 2, 100, 1024, 2048, "bf16", B.GSHARD_FLAG_ONE_SM_MMA),
     (1, 4, 96, 512, 1024, "bf16", B.GSHARD_FLAG_ONE_SM_MMA),

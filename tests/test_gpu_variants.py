@@ -1,5 +1,5 @@
 """Consistency of the kernel forms: on seeded random shapes every switchable form of the bf16
-tensor-core path (single-launch / chained / two-launch FFN, single CTAs / CTA pairs, the three gating
+tensor-core path (single-launch / two-launch FFN, single CTAs / CTA pairs, the three gating
 kernels, dispatch fused into the FFN) must agree with the CUDA-core form of the same layer - identical
 routing, y / l_aux / gradients within the tolerances of the oracle tests.  The oracle parity of the
 default forms is established elsewhere; this guards the alternatives and the ragged shapes."""
@@ -13,10 +13,10 @@ from paper_2006_16668_b200 import binding as B
 
 pytestmark = pytest.mark.gpu
 
-FORMS = [0, B.GSHARD_FLAG_FUSED_FFN, B.GSHARD_FLAG_CHAINED_FFN, B.GSHARD_FLAG_ONE_SM_MMA, B.GSHARD_FLAG_TWO_SM_MMA,
+FORMS = [0, B.GSHARD_FLAG_FUSED_FFN, B.GSHARD_FLAG_COMPACT_SLOTS, B.GSHARD_FLAG_ONE_SM_MMA, B.GSHARD_FLAG_TWO_SM_MMA,
          B.GSHARD_FLAG_GATE_CLUSTER, B.GSHARD_FLAG_GATE_ONE_SM, B.GSHARD_FLAG_GATHER_DISPATCH,
          B.GSHARD_FLAG_GATHER_DISPATCH | B.GSHARD_FLAG_FUSED_FFN, B.GSHARD_FLAG_SECOND_SKIP_FREES_SLOT,
-         B.GSHARD_FLAG_GATE_CLUSTER | B.GSHARD_FLAG_CHAINED_FFN]
+         B.GSHARD_FLAG_GATE_CLUSTER | B.GSHARD_FLAG_COMPACT_SLOTS]
 
 
 def _cases(n, seed):
