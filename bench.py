@@ -514,6 +514,50 @@ def measure(cfg, args, flags, dev, world, rank, sampler, *, e2e: bool, sustained
     return out
 
 
+def measure_dense_ffn(args, dev, sampler, n_tokens=131072, M=1024, H=8192) -> dict:
+    """The dense feed-forward sub-layer of the adjacent Transformer layer (section 2.1) at the headline
+    batch: y = relu(x . wi) . wo over all tokens, bf16, through gshard_dense_ffn_forward."""
+    import torch
+    from paper_2006_16668_b200 import binding as B
+    peaks = load_peaks()
+    gen = torch.Generator(device=dev).manual_seed(20200640)
+    x = torch.randn(n_tokens, M, generator=gen, device=dev).bfloat16()
+    wi = (torch.randn(M, H, generator=gen, device=dev) * M ** -0.5).bfloat16()
+    wo = (torch.randn(H, M, generator=gen, device=dev) * H ** -0.5).bfloat16()
+    y = torch.empty_like(x)
+    ws = torch.empty(B.gshard_dense_ffn_workspace_bytes(n_tokens, M, H, B.GSHARD_BF16), dtype=torch.uint8, device=dev)
+    flops = 4.0 * n_tokens * M * H
+
+    def region(steps):
+        torch.cuda.synchronize()
+        c0 = sampler.mark()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            B.gshard_dense_ffn_forward(x, wi, wo, y, ws)
+        e1.record()
+        torch.cuda.synchronize()
+        time.sleep(0.06)
+        if B.gshard_moe_last_device_status(ws) != B.GSHARD_OK:
+            raise SystemExit("dense FFN: device status is not OK")
+        return e0.elapsed_time(e1) / steps, sampler.summary(c0)
+
+    for _ in range(args.warmup):
+        B.gshard_dense_ffn_forward(x, wi, wo, y, ws)
+    ms, clocks = region(args.steps)
+    rec = {"workload": f"dense FFN of the adjacent Transformer layer, {n_tokens} x {M} x {H}, bf16",
+           "ms_per_step": ms, "value": n_tokens / (ms * 1e-3), "unit": UNIT, "tflops": flops / (ms * 1e-3) / 1e12,
+           "bound": "tensor", "frac": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"], "clocks": clocks,
+           "launches_per_step": B.gshard_moe_last_launch_count(), "kernel": "umma2_gemm_kernel, 2 launches"}
+    if args.sustained_seconds > 0:
+        steps = int(math.ceil(args.sustained_seconds * 1e3 / ms * 1.1))
+        sms, sclk = region(steps)
+        rec["sustained"] = {"steps": steps, "ms_per_step": sms, "tflops": flops / (sms * 1e-3) / 1e12,
+                            "frac_of_sustained_peak": flops / (sms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+                            "sm_mhz": sclk["sm_mhz"], "reasons": sclk["reasons"]}
+    return rec
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -602,6 +646,7 @@ def main():
                 if k in r:
                     keep[k] = r[k]
             extra[name] = keep
+        extra["dense_ffn"] = measure_dense_ffn(args, dev, sampler)
     sampler.stop()
     clocks["reasons_whole_run"] = sampler.summary()["reasons"]
 
