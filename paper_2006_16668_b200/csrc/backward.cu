@@ -352,7 +352,7 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
                                                d.add_residual ? reinterpret_cast<const uint4*>(dy) : nullptr,
                                                reinterpret_cast<uint4*>(dx), d.N, d.G, d.S, d.C, row_vec);
   count_launch();
-  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
 }  // namespace

@@ -346,7 +346,7 @@ int launch_gate_fused(const Dims& d, const void* x, const void* wg, float* logit
     return GSHARD_ERR_CUDA;
   gate_fused_kernel<<<grid, kThreads, kSmemBytes, st>>>(mx, mw, p);
   count_launch();
-  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
 }  // namespace gshard

@@ -404,7 +404,7 @@ int launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int 
     return GSHARD_ERR_CUDA;
   kern<<<grid, kThreads, Cfg<BN>::smem_bytes, st>>>(ma, mb, p);
   count_launch();
-  return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
 }  // namespace
@@ -448,7 +448,7 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
       return GSHARD_ERR_CUDA;
     umma_gemm_resident_b_kernel<<<n_groups < sms ? n_groups : sms, kThreads, resb::smem_bytes, st>>>(ma, mb, p);
     count_launch();
-    return cudaPeekAtLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
   }
   const int grid = (p.total_tiles < sms && !g.tile_base) ? p.total_tiles : sms;   // ragged: count known on the device only
   if (g.tf32)
