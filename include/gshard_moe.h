@@ -98,7 +98,10 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  overflowed tokens pass through it) folded into the
                                                  combine; backward: dx also receives dy.  Not applied
                                                  by the stage call gshard_moe_combine */
-/* bit 2048 is not in use */
+#define GSHARD_FLAG_PLAIN_STORES 2048u        /* the grouped GEMMs write their output tiles with 16-byte
+                                                 stores from the epilogue warps instead of bulk tensor
+                                                 (TMA) stores out of the staging rows; same bits, for
+                                                 comparisons */
 #define GSHARD_FLAG_BWD_PAIRED_GEMMS 4096u    /* backward: the GEMM that computes dh runs beside the one
                                                  for dwo, and dbuf beside dwi, each on half of the
                                                  multiprocessors (second, library-owned stream), so
@@ -131,7 +134,7 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  names another form); the flag extends it
                                                  to fewer rows.  Ignored with SAVE_FOR_BACKWARD and
                                                  where the single-launch FFN runs */
-#define GSHARD_FLAG_ALL (32767u & ~2048u)
+#define GSHARD_FLAG_ALL 32767u
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

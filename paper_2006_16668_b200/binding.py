@@ -36,6 +36,7 @@ GSHARD_FLAG_GATE_CLUSTER = 128
 GSHARD_FLAG_GATE_ONE_SM = 256
 GSHARD_FLAG_ONE_SM_MMA = 512
 GSHARD_FLAG_ADD_RESIDUAL = 1024
+GSHARD_FLAG_PLAIN_STORES = 2048
 GSHARD_FLAG_BWD_PAIRED_GEMMS = 4096
 GSHARD_FLAG_TF32_EXPERTS = 8192
 GSHARD_FLAG_COMPACT_SLOTS = 16384

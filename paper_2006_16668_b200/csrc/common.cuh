@@ -102,6 +102,7 @@ struct Dims {
   bool gather_dispatch; // single-launch FFN gathers its rows from x instead of reading a dispatch buffer
   bool tf32_experts;    // fp32 dtype: expert FFN contractions on the tensor cores in TF32
   bool compact_slots;   // grouped-GEMM expert FFN over compacted rows (empty slots skipped)
+  bool plain_stores;    // GEMM epilogues write with 16-byte stores instead of bulk tensor (TMA) stores
   bool bwd_paired;      // backward: read-heavy and write-heavy expert GEMMs side by side on half of the SMs each
 };
 
@@ -125,6 +126,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.one_sm_mma = (s.flags & GSHARD_FLAG_ONE_SM_MMA) != 0;
   d.add_residual = (s.flags & GSHARD_FLAG_ADD_RESIDUAL) != 0;
   d.bwd_paired = (s.flags & GSHARD_FLAG_BWD_PAIRED_GEMMS) != 0;
+  d.plain_stores = (s.flags & GSHARD_FLAG_PLAIN_STORES) != 0;
   d.tf32_experts = !d.bf16 && (s.flags & GSHARD_FLAG_TF32_EXPERTS) != 0;
   // Compacted slots: on request, and by default where an expert has at least six 128-row tiles, so
   // that the usual 13-30 % of empty slots free at least one of them (measured at the MoE(128E) shape:

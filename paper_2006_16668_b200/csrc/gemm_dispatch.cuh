@@ -6,7 +6,9 @@
 namespace gshard {
 
 // A and B hold the configuration dtype; C holds float when g.out_f32, else the dtype.
-inline int run_gemm(const Dims& d, const UmmaGemm& g, int* status, cudaStream_t st) {
+inline int run_gemm(const Dims& d, const UmmaGemm& g_in, int* status, cudaStream_t st) {
+  UmmaGemm g = g_in;
+  if (d.plain_stores) g.plain_stores = 1;
   if (!d.simt) {
     // CTA pairs with the two-SM MMA read only half of the B tile from their own shared memory per
     // MMA and load a third fewer operand bytes per SM; the one-SM kernel's 128 x 256 tiles keep the

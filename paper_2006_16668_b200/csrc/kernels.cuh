@@ -73,6 +73,7 @@ struct UmmaGemm {
                              // K-major, float output)
   const int* tile_base;      // ragged batch (device pointer, batch + 1 ints): problem b has
                              // tile_base[b+1] - tile_base[b] row tiles of 128 rows; single-CTA kernel only
+  int plain_stores;          // epilogue writes C with 16-byte stores instead of bulk tensor (TMA) stores
   int max_ctas;              // > 0: use at most this many CTAs (persistent grid), leaving the other
                              // multiprocessors to a kernel running beside this one on another stream
 };

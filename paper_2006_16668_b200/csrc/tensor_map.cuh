@@ -4,6 +4,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include "kernels.cuh"
+
 namespace gshard {
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -38,6 +40,23 @@ inline bool make_map(CUtensorMap* map, const void* base, long long inner, long l
             const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tensor map of an output matrix batch C [batch][rows][cols] (row pitch c_ld, batch pitch c_bs elements)
+// for the epilogue's 32-row x 128-byte stores.
+inline bool make_store_map(CUtensorMap* map, void* base, long long cols, long long rows, long long batch,
+                           long long c_ld, long long c_bs, int esize) {
+  return make_map(map, base, cols, rows, batch, c_ld, c_bs, 128 / esize, 32, esize);
+}
+
+// The store map of a GEMM's output, when its layout allows bulk stores (16-byte aligned base and row
+// pitch) and the caller did not ask for plain stores; false = use plain 16-byte stores.
+inline bool store_map_for(const UmmaGemm& g, CUtensorMap* mc) {
+  const int esize = g.out_f32 ? 4 : 2;
+  if (g.plain_stores || (reinterpret_cast<uintptr_t>(g.C) & 15u) || (g.c_ld * esize) % 16 ||
+      (g.batch > 1 && (g.c_bs * esize) % 16))
+    return false;
+  return make_store_map(mc, g.C, g.cols, g.rows, g.batch, g.c_ld, g.c_bs, esize);
 }
 
 }  // namespace gshard

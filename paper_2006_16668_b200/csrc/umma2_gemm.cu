@@ -40,7 +40,7 @@ constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kStages = 6;
 constexpr int kTmemCols = 2 * BN;
 constexpr int kBarOff = kStages * kStageBytes;
-constexpr int kStgOff = kBarOff + 256;
+constexpr int kStgOff = kBarOff + 1024;        // 1024-byte aligned: the staging rows leave by swizzled TMA stores
 constexpr int kSmemBytes = kStgOff + kEpiWarps * kStgWarpBytes + 1024;
 
 struct Params2 {
@@ -53,6 +53,7 @@ struct Params2 {
   int a_stream, b_stream;
   int n_fastest;
   int* status;
+  int tma_store;   // epilogue rows leave by bulk tensor stores through map_c
 };
 
 __device__ __forceinline__ TileCoord decode(const Params2& p, int tile) {
@@ -67,7 +68,7 @@ __device__ __forceinline__ TileCoord decode(const Params2& p, int tile) {
 template <bool A_K, bool B_K, bool MASK>
 __global__ void __launch_bounds__(kThreads, 1)
 umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                  const Params2 p) {
+                  const __grid_constant__ CUtensorMap map_c, const Params2 p) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kBarOff);
@@ -180,12 +181,14 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       if (MASK) load_mask_block(p, t.b, tile_row0 + q * 32, round_col0<BN>(t, half, 0), lane, mreg);
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      epilogue_tile<BN, MASK>(p, t, tile_row0, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, mreg);
+      epilogue_tile<BN, MASK>(p, p.tma_store ? &map_c : nullptr, t, tile_row0, tmem_base + (uint32_t)(acc * BN), q, half,
+                              stg, lane, mreg);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_remote_relaxed(ptx::map_to_cta(ptx::smem_u32(acc_empty + acc), 0));   // the leader's barrier
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    epilogue_finish(p.tma_store ? &map_c : nullptr, lane);
   }
 
   // ------------------------------ teardown ---------------------------------------------------
@@ -206,7 +209,8 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 }
 
 template <bool A_K, bool B_K, bool MASK>
-int launch2_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params2& p, int pairs, cudaStream_t st) {
+int launch2_t(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const Params2& p, int pairs,
+              cudaStream_t st) {
   auto kern = umma2_gemm_kernel<A_K, B_K, MASK>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
     return GSHARD_ERR_CUDA;
@@ -222,7 +226,7 @@ int launch2_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params2& p, in
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  if (cudaLaunchKernelEx(&cfg, kern, ma, mb, p) != cudaSuccess) { cudaGetLastError(); return GSHARD_ERR_CUDA; }
+  if (cudaLaunchKernelEx(&cfg, kern, ma, mb, mc, p) != cudaSuccess) { cudaGetLastError(); return GSHARD_ERR_CUDA; }
   count_launch();
   return GSHARD_OK;
 }
@@ -241,7 +245,10 @@ int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (g.b_kmajor) okm = okm && make_map(&mb, g.B, g.K, g.cols, g.batch, g.b_ld, g.b_bs, BK, BNH);
   else            okm = okm && make_map(&mb, g.B, g.cols, g.K, g.batch, g.b_ld, g.b_bs, 64, BK);
   if (!okm) return GSHARD_ERR_CUDA;
+  CUtensorMap mc;
+  const bool tma_store = store_map_for(g, &mc);
   Params2 p;
+  p.tma_store = tma_store ? 1 : 0;
   p.C = g.C; p.mask = g.mask; p.rows = g.rows; p.cols = g.cols; p.K = g.K; p.batch = g.batch;
   p.c_ld = g.c_ld; p.c_bs = g.c_bs;
   p.m_tiles = ceil_div(g.rows, 2 * BM); p.n_tiles = ceil_div(g.cols, BN);
@@ -255,7 +262,7 @@ int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (g.max_ctas > 0 && pairs > g.max_ctas / 2) pairs = g.max_ctas / 2 > 0 ? g.max_ctas / 2 : 1;
   if (pairs > p.total_tiles) pairs = p.total_tiles;
 #define GSHARD_DISPATCH2(AK, BKM) \
-  (p.mask ? launch2_t<AK, BKM, true>(ma, mb, p, pairs, st) : launch2_t<AK, BKM, false>(ma, mb, p, pairs, st))
+  (p.mask ? launch2_t<AK, BKM, true>(ma, mb, mc, p, pairs, st) : launch2_t<AK, BKM, false>(ma, mb, mc, p, pairs, st))
   if (g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH2(true, true);
   if (g.a_kmajor && !g.b_kmajor) return GSHARD_DISPATCH2(true, false);
   if (!g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH2(false, true);

@@ -49,6 +49,25 @@ __device__ __forceinline__ void flush_rows(const unsigned char* stg, const P& p,
   __syncwarp();
 }
 
+// The same block through the TMA unit: the warp's 32 staged rows x 128 bytes (already in the 128-byte
+// swizzle a tensor map expects, the staging block being 1024-byte aligned) leave as one bulk tensor
+// store; rows and columns beyond the matrix are clipped by the tensor map.  Compared with flush_rows
+// this takes the re-read of the staging rows and the global stores off the load/store pipe.  The
+// staging block may be rewritten only after store_wait().
+__device__ __forceinline__ void flush_rows_tma(const unsigned char* stg, const CUtensorMap* map_c, int b, int row0,
+                                               int col0, int lane) {
+  ptx::fence_proxy_async();          // this lane's staged bytes visible to the async proxy
+  __syncwarp();
+  if (lane == 0) {
+    ptx::tma_store_3d(map_c, stg, col0, row0, b);
+    ptx::tma_store_commit();
+  }
+}
+__device__ __forceinline__ void store_wait(int lane) {
+  if (lane == 0) ptx::tma_store_wait_read();
+  __syncwarp();
+}
+
 // Coalesced load of a warp's 32 x 64 block of the bf16 mask (128 bytes per row): lane l takes piece
 // (l & 7) of rows 4*i + (l >> 3), the pattern of flush_rows.  Pieces outside the matrix read as zero.
 template <typename P>
@@ -130,9 +149,11 @@ __device__ __forceinline__ int round_col0(const TileCoord& t, int half, int c) {
 // With a mask (bf16 output only) `mreg` holds the mask block of round 0, loaded by the caller
 // before it waited for the accumulator; the block of round c + 1 is fetched while round c is
 // processed, so the mask's global-memory latency stays off the accumulator's critical path.
+// map_c: tensor map of C for bulk stores, or nullptr for plain 16-byte stores.
 template <int BN, bool MASK, typename P>
-__device__ __forceinline__ void epilogue_tile(const P& p, const TileCoord& t, int tile_row0, uint32_t tmem_acc, int q, int half,
-                                              unsigned char* stg, int lane, uint4* mreg) {
+__device__ __forceinline__ void epilogue_tile(const P& p, const CUtensorMap* map_c, const TileCoord& t, int tile_row0,
+                                              uint32_t tmem_acc, int q, int half, unsigned char* stg, int lane,
+                                              uint4* mreg) {
   constexpr int kHalfCols = BN / 2;
   unsigned char* srow = stg + lane * kStgRowBytes;
   const int row0 = tile_row0 + q * 32;
@@ -144,6 +165,7 @@ __device__ __forceinline__ void epilogue_tile(const P& p, const TileCoord& t, in
     uint32_t r0[32], r1[32];
     ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r0);
     ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r1);
+    if (map_c) store_wait(lane);                 // the previous bulk store has read the staging block
     if (MASK) {
       stage_mask_block(stg, lane, mreg);
       if (c + 1 < kHalfCols / 64) load_mask_block(p, t.b, row0, col0 + 64, lane, mreg);
@@ -151,15 +173,24 @@ __device__ __forceinline__ void epilogue_tile(const P& p, const TileCoord& t, in
     ptx::tmem_ld_wait();
     if (p.out_f32) {                             // 32 fp32 columns = one 128-byte staging row
       process_chunk<MASK>(r0, p, srow, lane, 0);
-      flush_rows(stg, p, t.b, row0, col0, lane);
+      if (map_c) { flush_rows_tma(stg, map_c, t.b, row0, col0, lane); store_wait(lane); }
+      else flush_rows(stg, p, t.b, row0, col0, lane);
       process_chunk<MASK>(r1, p, srow, lane, 0);
-      flush_rows(stg, p, t.b, row0, col0 + 32, lane);
+      if (map_c) flush_rows_tma(stg, map_c, t.b, row0, col0 + 32, lane);
+      else flush_rows(stg, p, t.b, row0, col0 + 32, lane);
     } else {                                     // 64 bf16 columns = one 128-byte staging row
       process_chunk<MASK>(r0, p, srow, lane, 0);
       process_chunk<MASK>(r1, p, srow, lane, 4);
-      flush_rows(stg, p, t.b, row0, col0, lane);
+      if (map_c) flush_rows_tma(stg, map_c, t.b, row0, col0, lane);
+      else flush_rows(stg, p, t.b, row0, col0, lane);
     }
   }
+}
+
+// After a warp's last tile: its bulk stores have left shared memory and reached global memory.
+__device__ __forceinline__ void epilogue_finish(const CUtensorMap* map_c, int lane) {
+  if (map_c && lane == 0) ptx::tma_store_wait_all();
+  __syncwarp();
 }
 
 }  // namespace umma_epi

@@ -41,7 +41,7 @@ template <int BN> struct Cfg {
   static constexpr int stages = (BN == 256) ? 4 : 6;
   static constexpr int tmem_cols = 2 * BN;   // two accumulators
   static constexpr int bar_off = stages * stage_bytes;
-  static constexpr int stg_off = bar_off + 256;
+  static constexpr int stg_off = bar_off + 1024;     // 1024-byte aligned: the staging rows leave by swizzled TMA stores
   static constexpr int smem_bytes = stg_off + kEpiWarps * kStgWarpBytes + 1024 /*alignment slack*/;
 };
 
@@ -58,6 +58,7 @@ struct Params {
   // Ragged batches (compacted expert rows): problem b owns the row tiles [tile_base[b], tile_base[b+1])
   // of a device-side prefix array with batch + 1 entries; nullptr = every problem has m_tiles row tiles.
   const int* tile_base;
+  int tma_store;   // epilogue rows leave by bulk tensor stores through map_c
 };
 
 // Tile index -> (row tile, column tile, problem).  A thread walks its tiles in increasing order, so
@@ -92,7 +93,7 @@ struct TileWalk {
 template <bool A_K, bool B_K, int BN, bool MASK, bool TF32 = false>
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                 const Params p) {
+                 const __grid_constant__ CUtensorMap map_c, const Params p) {
   using C_ = Cfg<BN>;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -209,12 +210,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       if (MASK) load_mask_block(p, t.b, t.mt * BM + q * 32, round_col0<BN>(t, half, 0), lane, mreg);
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
-      epilogue_tile<BN, MASK>(p, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, mreg);
+      epilogue_tile<BN, MASK>(p, p.tma_store ? &map_c : nullptr, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q, half,
+                              stg, lane, mreg);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_relaxed(acc_empty + acc);
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    epilogue_finish(p.tma_store ? &map_c : nullptr, lane);
   }
 
   // ------------------------------ teardown ---------------------------------------------------
@@ -253,14 +256,14 @@ constexpr int kBBlockBytes = BN * BK * 2;                        // 32 KB per k-
 constexpr int kAStages = 4;
 constexpr int a_off = kMaxKBlocks * kBBlockBytes;                // 128 KB
 constexpr int bar_off = a_off + kAStages * kABytes;              // + 64 KB
-constexpr int stg_off = bar_off + 256;
+constexpr int stg_off = bar_off + 1024;
 constexpr int smem_bytes = stg_off + kEpiWarps * kStgWarpBytes + 1024;
 constexpr int tmem_cols = 2 * BN;
 }  // namespace resb
 
 __global__ void __launch_bounds__(kThreads, 1)
 umma_gemm_resident_b_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                            const Params p) {
+                            const __grid_constant__ CUtensorMap map_c, const Params p) {
   using namespace resb;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -371,13 +374,15 @@ umma_gemm_resident_b_kernel(const __grid_constant__ CUtensorMap map_a, const __g
       for (t.mt = 0; t.mt < p.m_tiles; ++t.mt) {
         if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
         ptx::tc_fence_after_sync();
-        epilogue_tile<BN, false>(p, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q, half, stg, lane, nullptr);
+        epilogue_tile<BN, false>(p, p.tma_store ? &map_c : nullptr, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q,
+                                 half, stg, lane, nullptr);
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive_relaxed(acc_empty + acc);
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
     }
+    epilogue_finish(p.tma_store ? &map_c : nullptr, lane);
   }
 
   if (!ok) {
@@ -398,11 +403,12 @@ umma_gemm_resident_b_kernel(const __grid_constant__ CUtensorMap map_a, const __g
 // ---- host side ------------------------------------------------------------------------------
 
 template <bool A_K, bool B_K, int BN, bool MASK, bool TF32 = false>
-int launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const Params& p, int grid, cudaStream_t st) {
+int launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc, const Params& p, int grid,
+             cudaStream_t st) {
   auto kern = umma_gemm_kernel<A_K, B_K, BN, MASK, TF32>;
   if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<BN>::smem_bytes) != cudaSuccess)
     return GSHARD_ERR_CUDA;
-  kern<<<grid, kThreads, Cfg<BN>::smem_bytes, st>>>(ma, mb, p);
+  kern<<<grid, kThreads, Cfg<BN>::smem_bytes, st>>>(ma, mb, mc, p);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
@@ -425,7 +431,10 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (g.b_kmajor) okm = okm && make_map(&mb, g.B, g.K, g.cols, g.batch, g.b_ld, g.b_bs, bke, BN, esz);
   else            okm = okm && make_map(&mb, g.B, g.cols, g.K, g.batch, g.b_ld, g.b_bs, bke, bke, esz);
   if (!okm) return GSHARD_ERR_CUDA;
+  CUtensorMap mc;
+  const bool tma_store = store_map_for(g, &mc);
   Params p;
+  p.tma_store = tma_store ? 1 : 0;
   p.C = g.C; p.mask = g.mask; p.rows = g.rows; p.cols = g.cols; p.K = g.K; p.batch = g.batch;
   p.c_ld = g.c_ld; p.c_bs = g.c_bs;
   p.m_tiles = ceil_div(g.rows, BM); p.n_tiles = ceil_div(g.cols, BN);
@@ -446,19 +455,19 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
     if (cudaFuncSetAttribute(umma_gemm_resident_b_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              resb::smem_bytes) != cudaSuccess)
       return GSHARD_ERR_CUDA;
-    umma_gemm_resident_b_kernel<<<n_groups < sms ? n_groups : sms, kThreads, resb::smem_bytes, st>>>(ma, mb, p);
+    umma_gemm_resident_b_kernel<<<n_groups < sms ? n_groups : sms, kThreads, resb::smem_bytes, st>>>(ma, mb, mc, p);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
   }
   const int grid = (p.total_tiles < sms && !g.tile_base) ? p.total_tiles : sms;   // ragged: count known on the device only
   if (g.tf32)
-    return BN == 256 ? launch_t<true, true, 256, false, true>(ma, mb, p, grid, st)
-                     : launch_t<true, true, 128, false, true>(ma, mb, p, grid, st);
+    return BN == 256 ? launch_t<true, true, 256, false, true>(ma, mb, mc, p, grid, st)
+                     : launch_t<true, true, 128, false, true>(ma, mb, mc, p, grid, st);
 #define GSHARD_DISPATCH(AK, BKM)                                                                    \
-  (p.mask ? (BN == 256 ? launch_t<AK, BKM, 256, true>(ma, mb, p, grid, st)                          \
-                       : launch_t<AK, BKM, 128, true>(ma, mb, p, grid, st))                         \
-          : (BN == 256 ? launch_t<AK, BKM, 256, false>(ma, mb, p, grid, st)                         \
-                       : launch_t<AK, BKM, 128, false>(ma, mb, p, grid, st)))
+  (p.mask ? (BN == 256 ? launch_t<AK, BKM, 256, true>(ma, mb, mc, p, grid, st)                          \
+                       : launch_t<AK, BKM, 128, true>(ma, mb, mc, p, grid, st))                         \
+          : (BN == 256 ? launch_t<AK, BKM, 256, false>(ma, mb, mc, p, grid, st)                         \
+                       : launch_t<AK, BKM, 128, false>(ma, mb, mc, p, grid, st)))
   if (g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH(true, true);
   if (g.a_kmajor && !g.b_kmajor) return GSHARD_DISPATCH(true, false);
   if (!g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH(false, true);
