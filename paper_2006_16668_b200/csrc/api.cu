@@ -95,7 +95,7 @@ bool ffn_runs_fused(const Dims& d, bool keep_h) {
 // With x / slot_token (only where ffn_runs_fused) the rows are gathered from x and buf is not read.
 int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
               void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token,
-              void* wt, const int* tile_base) {
+              void* wt, const int* tile_base, uint32_t* relu_bits_out) {
   const long long rows = d.rows;
   // One persistent launch in which the hidden activations never leave L2: the faster form when
   // the FFN is bound by streaming the expert weights (at most one 128-row tile per expert); with
@@ -114,6 +114,7 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   g.a_kmajor = true; g.b_kmajor = false;
   g.a_ld = d.M; g.a_bs = rows * d.M; g.b_ld = d.H; g.b_bs = (long long)d.M * d.H; g.c_ld = d.H; g.c_bs = rows * d.H;
   g.relu = 1; g.b_stream = 1; g.prefer_two_sm = 1;
+  if (!d.simt) g.mask_bits_out = relu_bits_out;   // the backward's ReLU mask, one bit per hidden activation
   UmmaGemm g2{};
   g2.A = h; g2.B = wo; g2.C = out; g2.rows = d.rows; g2.cols = d.M; g2.K = d.H; g2.batch = d.E;
   g2.a_kmajor = true; g2.b_kmajor = false;
@@ -196,7 +197,7 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
   float* m = pick(r.m, ws, pl.m);
   float* l_aux_group = pick(r.l_aux_group, ws, pl.l_aux_group);
   int32_t* stats_group = reinterpret_cast<int32_t*>(ws + pl.stats_group);
-  void* buf = ws + pl.buf;
+  void* buf = save ? static_cast<void*>(ctx + cp.buf) : static_cast<void*>(ws + pl.buf);
 
   GS_TRY(gate_stage(d, pl, ws, x, wg, expert_idx, gate12, m, rowmax, rowinv, st));
   GS_TRY(launch_capacity(d, expert_idx, gate12, u, m, slot, weight, flags, first_count, total_count, slot_token,
@@ -219,7 +220,8 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
   const bool timed = ft.start != nullptr && ft.stop != nullptr;
   if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.start), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   GS_TRY(ffn_stage(d, buf, wi, wo, h, save, out, ws + pl.ffn_scratch, status, st, gather ? x : nullptr, slot_token,
-                   ws + pl.wt, compact ? tile_base : nullptr));
+                   ws + pl.wt, compact ? tile_base : nullptr,
+                   (save && !d.simt) ? reinterpret_cast<uint32_t*>(ctx + cp.hbits) : nullptr));
   if (timed && cudaEventRecord(static_cast<cudaEvent_t>(ft.stop), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   ft.start = ft.stop = nullptr;
   launch_combine(d, out, expert_idx, slot, weight, y, st, d.add_residual ? x : nullptr, compact ? slot_crow : nullptr);

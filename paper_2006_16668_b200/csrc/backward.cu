@@ -254,11 +254,12 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   const float* rowmax = reinterpret_cast<const float*>(ctx + cp.rowmax);
   const float* rowinv = reinterpret_cast<const float*>(ctx + cp.rowinv);
   const void* h = ctx + cp.h;
+  const uint32_t* hbits = d.simt ? nullptr : reinterpret_cast<const uint32_t*>(ctx + cp.hbits);
   const void* out = ctx + cp.out;
   float* logits = reinterpret_cast<float*>(ws + bp.logits);
   T* dlogits = reinterpret_cast<T*>(ws + bp.dlogits);
   float* dw = reinterpret_cast<float*>(ws + bp.dw);
-  void* buf = ws + bp.buf;
+  const void* buf = ctx + cp.buf;              // dispatched inputs, as the forward wrote them
   void* dout = ws + bp.dout;
   void* dh = ws + bp.dh;
   void* dbuf = ws + bp.dbuf;
@@ -273,13 +274,12 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   dout_kernel<T><<<grid_for_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(dy), slot_token, expert_idx, slot,
                                                  weight, reinterpret_cast<uint4*>(dout), d.R, d.G, d.S, d.C, row_vec);
   count_launch(2);
-  launch_dispatch(d, x, slot_token, buf, st);
 
   // expert FFN backward.  dh and dbuf stream the weights (read-heavy), dwo and dwi write a gradient the
   // size of the weights from short contractions (write-heavy): one of each runs side by side.
   UmmaGemm g_dh{}, g_dwo{}, g_dwi{}, g_dbuf{};
   // dh = (dout . wo^T) masked by h > 0
-  g_dh.A = dout; g_dh.B = wo; g_dh.C = dh; g_dh.mask = h; g_dh.rows = d.rows; g_dh.cols = d.H; g_dh.K = d.M; g_dh.batch = d.E;
+  g_dh.A = dout; g_dh.B = wo; g_dh.C = dh; g_dh.mask = h; g_dh.mask_bits = hbits; g_dh.rows = d.rows; g_dh.cols = d.H; g_dh.K = d.M; g_dh.batch = d.E;
   g_dh.a_kmajor = true; g_dh.b_kmajor = true;
   g_dh.a_ld = d.M; g_dh.a_bs = rows * d.M; g_dh.b_ld = d.M; g_dh.b_bs = (long long)d.H * d.M; g_dh.c_ld = d.H; g_dh.c_bs = rows * d.H;
   g_dh.b_stream = 1; g_dh.prefer_two_sm = 1;

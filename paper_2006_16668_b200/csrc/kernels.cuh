@@ -58,7 +58,9 @@ void launch_transpose_f32(const float* src, float* dst, int batch, int rows, int
 // umma_gemm.cu: batched bf16 GEMM on tcgen05, C[b] = act(A[b] . B[b]).
 struct UmmaGemm {
   const void* A; const void* B; void* C;
-  const void* mask;          // optional bf16 tensor laid out like C: output zeroed where mask <= 0
+  const void* mask;          // CUDA-core path: optional tensor laid out like C, output zeroed where mask <= 0
+  const uint32_t* mask_bits; // tensor-core path: the same as bits, [batch][rows][cols/32] words
+  uint32_t* mask_bits_out;   // tensor-core path: write bit = (accumulator value > 0) in that layout
   int rows, cols, K, batch;
   bool a_kmajor;             // A stored [rows, K] (K contiguous); else stored [K, rows]
   bool b_kmajor;             // B stored [cols, K] (K contiguous); else stored [K, cols]

@@ -54,10 +54,10 @@ inline FwdPlan plan_forward(const Dims& d) {
   return p;
 }
 
-// Saved by the forward for the backward: routing, softmax row statistics, hidden activations
-// and expert outputs.
+// Saved by the forward for the backward: routing, softmax row statistics, dispatched inputs, hidden
+// activations (and their ReLU mask as bits) and expert outputs.
 struct CtxPlan {
-  size_t expert_idx, slot, weight, first_count, slot_token, gate12, rowmax, rowinv, h, out, total;
+  size_t expert_idx, slot, weight, first_count, slot_token, gate12, rowmax, rowinv, h, out, hbits, buf, total;
 };
 
 inline CtxPlan plan_context(const Dims& d) {
@@ -73,6 +73,8 @@ inline CtxPlan plan_context(const Dims& d) {
   p.rowinv = c.take(N * 4);
   p.h = c.take(R * d.H * d.esize);
   p.out = c.take(R * d.M * d.esize);
+  p.hbits = c.take(d.simt ? 0 : R * (size_t)d.H / 8);   // ReLU mask as bits, written by the forward's GEMM-1
+  p.buf = c.take(R * d.M * d.esize);                    // dispatched expert inputs (dwi contracts over them)
   p.total = c.off;
   return p;
 }
@@ -89,9 +91,10 @@ inline StagePlan plan_staging(const Dims& d) {
   return p;
 }
 
-// Backward scratch: logits / dlogits [N,E], dispatched inputs, dout, dh, dbuf, per-token dw.
+// Backward scratch: logits / dlogits [N,E], dout, dh, dbuf, per-token dw (the dispatched inputs come
+// from the context).
 struct BwdPlan {
-  size_t status, logits, dlogits, dw, buf, dout, dh, dbuf, dxg, total;
+  size_t status, logits, dlogits, dw, dout, dh, dbuf, dxg, total;
 };
 
 inline BwdPlan plan_backward(const Dims& d) {
@@ -101,7 +104,6 @@ inline BwdPlan plan_backward(const Dims& d) {
   p.logits = c.take(N * d.E * 4);
   p.dlogits = c.take(N * d.E * d.esize);
   p.dw = c.take(N * 2 * 4);
-  p.buf = c.take(R * d.M * d.esize);
   p.dout = c.take(R * d.M * d.esize);
   p.dh = c.take(R * d.H * d.esize);
   p.dbuf = c.take(R * d.M * d.esize);
@@ -123,7 +125,7 @@ bool ffn_runs_fused(const Dims& d, bool keep_h);
 // wt: with d.tf32_experts, room for the transposed copies of wi and wo (2 * E * M * H floats).
 int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
               void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token,
-              void* wt = nullptr, const int* tile_base = nullptr);
+              void* wt = nullptr, const int* tile_base = nullptr, uint32_t* relu_bits_out = nullptr);
 int check_device();
 
 }  // namespace gshard

@@ -45,7 +45,8 @@ constexpr int kSmemBytes = kStgOff + kEpiWarps * kStgWarpBytes + 1024;
 
 struct Params2 {
   void* C;
-  const void* mask;
+  const uint32_t* mask_bits;   // optional [batch][rows][cols/32]: output zeroed where the bit is clear
+  uint32_t* mask_bits_out;     // optional, same layout: bit = accumulator value positive
   int rows, cols, K, batch;
   long long c_ld, c_bs;
   int m_tiles, n_tiles, total_tiles, k_blocks;   // tiles of 256 x 256
@@ -177,12 +178,10 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     for (int tile = pair; tile < p.total_tiles && ok; tile += n_pairs) {
       const TileCoord t = decode(p, tile);
       const int tile_row0 = t.mt * 2 * BM + (int)rank * BM;     // this CTA's 128 rows of the 256-row tile
-      uint4 mreg[MASK ? 8 : 1];
-      if (MASK) load_mask_block(p, t.b, tile_row0 + q * 32, round_col0<BN>(t, half, 0), lane, mreg);
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       epilogue_tile<BN, MASK>(p, p.tma_store ? &map_c : nullptr, t, tile_row0, tmem_base + (uint32_t)(acc * BN), q, half,
-                              stg, lane, mreg);
+                              stg, lane);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_remote_relaxed(ptx::map_to_cta(ptx::smem_u32(acc_empty + acc), 0));   // the leader's barrier
@@ -237,7 +236,7 @@ int launch2_t(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& m
 // launch_umma_gemm.  Worth it when a problem has more than one 128-row tile.
 int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (g.rows <= 0 || g.cols <= 0 || g.K <= 0 || g.batch <= 0) return GSHARD_OK;
-  if (g.mask && g.out_f32) return GSHARD_ERR_INTERNAL;   // the mask is staged as bf16 rows
+  if ((g.mask_bits || g.mask_bits_out) && g.cols % 32) return GSHARD_ERR_INTERNAL;   // one word per 32 columns
   CUtensorMap ma, mb;
   bool okm;
   if (g.a_kmajor) okm = make_map(&ma, g.A, g.K, g.rows, g.batch, g.a_ld, g.a_bs, BK, BM);
@@ -249,7 +248,7 @@ int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   const bool tma_store = store_map_for(g, &mc);
   Params2 p;
   p.tma_store = tma_store ? 1 : 0;
-  p.C = g.C; p.mask = g.mask; p.rows = g.rows; p.cols = g.cols; p.K = g.K; p.batch = g.batch;
+  p.C = g.C; p.mask_bits = g.mask_bits; p.mask_bits_out = g.mask_bits_out; p.rows = g.rows; p.cols = g.cols; p.K = g.K; p.batch = g.batch;
   p.c_ld = g.c_ld; p.c_bs = g.c_bs;
   p.m_tiles = ceil_div(g.rows, 2 * BM); p.n_tiles = ceil_div(g.cols, BN);
   p.total_tiles = p.m_tiles * p.n_tiles * g.batch;
@@ -262,7 +261,7 @@ int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (g.max_ctas > 0 && pairs > g.max_ctas / 2) pairs = g.max_ctas / 2 > 0 ? g.max_ctas / 2 : 1;
   if (pairs > p.total_tiles) pairs = p.total_tiles;
 #define GSHARD_DISPATCH2(AK, BKM) \
-  (p.mask ? launch2_t<AK, BKM, true>(ma, mb, mc, p, pairs, st) : launch2_t<AK, BKM, false>(ma, mb, mc, p, pairs, st))
+  (p.mask_bits ? launch2_t<AK, BKM, true>(ma, mb, mc, p, pairs, st) : launch2_t<AK, BKM, false>(ma, mb, mc, p, pairs, st))
   if (g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH2(true, true);
   if (g.a_kmajor && !g.b_kmajor) return GSHARD_DISPATCH2(true, false);
   if (!g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH2(false, true);

@@ -68,56 +68,18 @@ __device__ __forceinline__ void store_wait(int lane) {
   __syncwarp();
 }
 
-// Coalesced load of a warp's 32 x 64 block of the bf16 mask (128 bytes per row): lane l takes piece
-// (l & 7) of rows 4*i + (l >> 3), the pattern of flush_rows.  Pieces outside the matrix read as zero.
-template <typename P>
-__device__ __forceinline__ void load_mask_block(const P& p, int b, int row0, int col0, int lane, uint4* m) {
-  const int piece = lane & 7;
-  const int col = col0 + piece * 8;
-  const unsigned char* base = reinterpret_cast<const unsigned char*>(p.mask) + ((long long)b * p.c_bs + col) * 2;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int row = row0 + 4 * i + (lane >> 3);
-    m[i] = (row < p.rows && col < p.cols) ? __ldg(reinterpret_cast<const uint4*>(base + (long long)row * p.c_ld * 2))
-                                          : make_uint4(0u, 0u, 0u, 0u);
-  }
-}
-
-__device__ __forceinline__ void stage_mask_block(unsigned char* stg, int lane, const uint4* m) {
-  const int piece = lane & 7;
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int r = 4 * i + (lane >> 3);
-    *reinterpret_cast<uint4*>(stg + r * kStgRowBytes + ((piece ^ (r & 7)) * 16)) = m[i];
-  }
-  __syncwarp();
-}
-
 // ReLU / mask on one 32-column chunk of this thread's row, then into the staging row (XOR-swizzled
 // 16-byte pieces: conflict-free for the row-wise writes here and the piece-wise reads of the flush).
+// mword: with MASK, bit i set = keep column i of the chunk.
 template <bool MASK, typename P>
 __device__ __forceinline__ void process_chunk(const uint32_t* r, const P& p, unsigned char* srow, int lane,
-                                              int piece0) {
+                                              int piece0, uint32_t mword) {
   float v[32];
 #pragma unroll
   for (int i = 0; i < 32; ++i) {
     v[i] = __uint_as_float(r[i]);
     if (p.relu) v[i] = fmaxf(v[i], 0.f);
-  }
-  if (MASK) {
-    // the mask block was staged into this row's pieces (same swizzle as the output written below)
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const uint4 mv = *reinterpret_cast<const uint4*>(srow + (((piece0 + i) ^ (lane & 7)) * 16));
-      const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        // bf16 > 0  <=>  sign bit clear and magnitude bits non-zero
-        const uint32_t lo = w[j] & 0xffffu, hi = w[j] >> 16;
-        if (!(lo != 0u && lo < 0x8000u)) v[8 * i + 2 * j] = 0.f;
-        if (!(hi != 0u && hi < 0x8000u)) v[8 * i + 2 * j + 1] = 0.f;
-      }
-    }
+    if (MASK && !((mword >> i) & 1u)) v[i] = 0.f;
   }
   if (p.out_f32) {
 #pragma unroll
@@ -144,19 +106,28 @@ __device__ __forceinline__ int round_col0(const TileCoord& t, int half, int c) {
   return t.nt * BN + half * (BN / 2) + c * 64;
 }
 
+// Bit i of the result: accumulator value i of the chunk is positive (the ReLU passes it).
+__device__ __forceinline__ uint32_t positive_bits(const uint32_t* r) {
+  uint32_t w = 0;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) w |= (__uint_as_float(r[i]) > 0.f ? 1u : 0u) << i;
+  return w;
+}
+
 // One epilogue warp's share of a finished 128 x BN accumulator whose first row is tile_row0: lane
-// quarter q, column half `half`.
-// With a mask (bf16 output only) `mreg` holds the mask block of round 0, loaded by the caller
-// before it waited for the accumulator; the block of round c + 1 is fetched while round c is
-// processed, so the mask's global-memory latency stays off the accumulator's critical path.
-// map_c: tensor map of C for bulk stores, or nullptr for plain 16-byte stores.
+// quarter q, column half `half`.  map_c: tensor map of C for bulk stores, or nullptr for plain 16-byte
+// stores.  With MASK (bf16 output only) the output is zeroed where the bit of p.mask_bits
+// ([batch][rows][cols/32] words, bit = column mod 32) is clear; the two words of a thread's row and
+// round are fetched while the accumulator load is in flight.  With p.mask_bits_out the same layout is
+// WRITTEN: bit = accumulator value positive (the ReLU mask the backward pass needs).
 template <int BN, bool MASK, typename P>
 __device__ __forceinline__ void epilogue_tile(const P& p, const CUtensorMap* map_c, const TileCoord& t, int tile_row0,
-                                              uint32_t tmem_acc, int q, int half, unsigned char* stg, int lane,
-                                              uint4* mreg) {
+                                              uint32_t tmem_acc, int q, int half, unsigned char* stg, int lane) {
   constexpr int kHalfCols = BN / 2;
   unsigned char* srow = stg + lane * kStgRowBytes;
   const int row0 = tile_row0 + q * 32;
+  const int row = row0 + lane;
+  const long long word_row = ((long long)t.b * p.rows + row) * (p.cols >> 5);
   const uint32_t t_acc = tmem_acc + (uint32_t)(half * kHalfCols) + ((uint32_t)(q * 32) << 16);
 #pragma unroll 1
   for (int c = 0; c < kHalfCols / 64; ++c) {     // 64 columns per round: two TMEM loads in flight
@@ -165,22 +136,27 @@ __device__ __forceinline__ void epilogue_tile(const P& p, const CUtensorMap* map
     uint32_t r0[32], r1[32];
     ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64), r0);
     ptx::tmem_ld_32x32(t_acc + (uint32_t)(c * 64 + 32), r1);
-    if (map_c) store_wait(lane);                 // the previous bulk store has read the staging block
-    if (MASK) {
-      stage_mask_block(stg, lane, mreg);
-      if (c + 1 < kHalfCols / 64) load_mask_block(p, t.b, row0, col0 + 64, lane, mreg);
+    uint32_t m0 = 0, m1 = 0;
+    if (MASK && row < p.rows) {
+      m0 = __ldg(p.mask_bits + word_row + (col0 >> 5));
+      if (col0 + 32 < p.cols) m1 = __ldg(p.mask_bits + word_row + (col0 >> 5) + 1);
     }
+    if (map_c) store_wait(lane);                 // the previous bulk store has read the staging block
     ptx::tmem_ld_wait();
+    if (p.mask_bits_out && row < p.rows) {
+      p.mask_bits_out[word_row + (col0 >> 5)] = positive_bits(r0);
+      if (col0 + 32 < p.cols) p.mask_bits_out[word_row + (col0 >> 5) + 1] = positive_bits(r1);
+    }
     if (p.out_f32) {                             // 32 fp32 columns = one 128-byte staging row
-      process_chunk<MASK>(r0, p, srow, lane, 0);
+      process_chunk<MASK>(r0, p, srow, lane, 0, m0);
       if (map_c) { flush_rows_tma(stg, map_c, t.b, row0, col0, lane); store_wait(lane); }
       else flush_rows(stg, p, t.b, row0, col0, lane);
-      process_chunk<MASK>(r1, p, srow, lane, 0);
+      process_chunk<MASK>(r1, p, srow, lane, 0, m1);
       if (map_c) flush_rows_tma(stg, map_c, t.b, row0, col0 + 32, lane);
       else flush_rows(stg, p, t.b, row0, col0 + 32, lane);
     } else {                                     // 64 bf16 columns = one 128-byte staging row
-      process_chunk<MASK>(r0, p, srow, lane, 0);
-      process_chunk<MASK>(r1, p, srow, lane, 4);
+      process_chunk<MASK>(r0, p, srow, lane, 0, m0);
+      process_chunk<MASK>(r1, p, srow, lane, 4, m1);
       if (map_c) flush_rows_tma(stg, map_c, t.b, row0, col0, lane);
       else flush_rows(stg, p, t.b, row0, col0, lane);
     }

@@ -47,7 +47,8 @@ template <int BN> struct Cfg {
 
 struct Params {
   void* C;
-  const void* mask;
+  const uint32_t* mask_bits;   // optional [batch][rows][cols/32]: output zeroed where the bit is clear
+  uint32_t* mask_bits_out;     // optional, same layout: bit = accumulator value positive
   int rows, cols, K, batch;
   long long c_ld, c_bs;
   int m_tiles, n_tiles, total_tiles, k_blocks;
@@ -206,12 +207,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int total_tiles = walk.total(p);
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
       const TileCoord t = walk.decode(p, tile);
-      uint4 mreg[MASK ? 8 : 1];
-      if (MASK) load_mask_block(p, t.b, t.mt * BM + q * 32, round_col0<BN>(t, half, 0), lane, mreg);
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       epilogue_tile<BN, MASK>(p, p.tma_store ? &map_c : nullptr, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q, half,
-                              stg, lane, mreg);
+                              stg, lane);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_relaxed(acc_empty + acc);
@@ -375,7 +374,7 @@ umma_gemm_resident_b_kernel(const __grid_constant__ CUtensorMap map_a, const __g
         if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         epilogue_tile<BN, false>(p, p.tma_store ? &map_c : nullptr, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q,
-                                 half, stg, lane, nullptr);
+                                 half, stg, lane);
         ptx::tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive_relaxed(acc_empty + acc);
@@ -417,11 +416,11 @@ int launch_t(const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc
 
 int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (g.rows <= 0 || g.cols <= 0 || g.K <= 0 || g.batch <= 0) return GSHARD_OK;
-  if (g.mask && g.out_f32) return GSHARD_ERR_INTERNAL;   // the mask is staged as bf16 rows
+  if ((g.mask_bits || g.mask_bits_out) && g.cols % 32) return GSHARD_ERR_INTERNAL;   // one word per 32 columns
   const int BN = g.cols > 128 ? 256 : 128;
   // fp32 operands read as TF32: the tensor core takes 32-bit operands K-major only (an MN-major
   // one yields zeros), so both operands must be contiguous along the contraction
-  if (g.tf32 && (!g.a_kmajor || !g.b_kmajor || g.mask || !g.out_f32)) return GSHARD_ERR_INTERNAL;
+  if (g.tf32 && (!g.a_kmajor || !g.b_kmajor || g.mask_bits || !g.out_f32)) return GSHARD_ERR_INTERNAL;
   const int esz = g.tf32 ? 4 : 2;
   const int bke = 128 / esz;                     // elements per 128-byte k-block row
   CUtensorMap ma, mb;
@@ -435,7 +434,7 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   const bool tma_store = store_map_for(g, &mc);
   Params p;
   p.tma_store = tma_store ? 1 : 0;
-  p.C = g.C; p.mask = g.mask; p.rows = g.rows; p.cols = g.cols; p.K = g.K; p.batch = g.batch;
+  p.C = g.C; p.mask_bits = g.mask_bits; p.mask_bits_out = g.mask_bits_out; p.rows = g.rows; p.cols = g.cols; p.K = g.K; p.batch = g.batch;
   p.c_ld = g.c_ld; p.c_bs = g.c_bs;
   p.m_tiles = ceil_div(g.rows, BM); p.n_tiles = ceil_div(g.cols, BN);
   p.total_tiles = p.m_tiles * p.n_tiles * g.batch;
@@ -449,7 +448,7 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   if (g.tile_base) p.n_fastest = 0;            // ragged lists are walked with the row tiles fastest
   int sms = device_sms();
   if (g.max_ctas > 0 && sms > g.max_ctas) sms = g.max_ctas;
-  if (!g.tf32 && !g.tile_base && !g.a_kmajor && !g.b_kmajor && !g.mask && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
+  if (!g.tf32 && !g.tile_base && !g.a_kmajor && !g.b_kmajor && !g.mask_bits && BN == 256 && p.k_blocks <= resb::kMaxKBlocks && p.m_tiles >= 4) {
     // short contraction, several row tiles per column block: keep the B tile resident
     const int n_groups = p.n_tiles * g.batch;
     if (cudaFuncSetAttribute(umma_gemm_resident_b_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -464,7 +463,7 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
     return BN == 256 ? launch_t<true, true, 256, false, true>(ma, mb, mc, p, grid, st)
                      : launch_t<true, true, 128, false, true>(ma, mb, mc, p, grid, st);
 #define GSHARD_DISPATCH(AK, BKM)                                                                    \
-  (p.mask ? (BN == 256 ? launch_t<AK, BKM, 256, true>(ma, mb, mc, p, grid, st)                          \
+  (p.mask_bits ? (BN == 256 ? launch_t<AK, BKM, 256, true>(ma, mb, mc, p, grid, st)                          \
                        : launch_t<AK, BKM, 128, true>(ma, mb, mc, p, grid, st))                         \
           : (BN == 256 ? launch_t<AK, BKM, 256, false>(ma, mb, mc, p, grid, st)                         \
                        : launch_t<AK, BKM, 128, false>(ma, mb, mc, p, grid, st)))
