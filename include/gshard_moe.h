@@ -26,6 +26,8 @@
  *     tcgen05 tensor cores with fp32 accumulation; softmax, top-2, weights, l_aux are fp32.
  *     u, l_aux, weight, m, dwg are always float.
  *   - Outputs are bit-reproducible from run to run (no atomics in any reduction).
+ *   - Every stage's launches sit inside an NVTX range (gshard.gate, .capacity, .dispatch,
+ *     .expert_ffn, .combine, .backward.*), visible to a profiler that injects NVTX.
  */
 #ifndef GSHARD_MOE_H_
 #define GSHARD_MOE_H_
@@ -134,7 +136,12 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  names another form); the flag extends it
                                                  to fewer rows.  Ignored with SAVE_FOR_BACKWARD and
                                                  where the single-launch FFN runs */
-#define GSHARD_FLAG_ALL 32767u
+#define GSHARD_FLAG_DEBUG_CHECKS 32768u       /* forward: after the capacity stage a kernel verifies the
+                                                 routing tensors (expert ids, positions, flags, weights,
+                                                 the inverse slot list; every access bounds-checked) and
+                                                 records GSHARD_ERR_INTERNAL in the status word on a
+                                                 violation - nothing traps */
+#define GSHARD_FLAG_ALL 65535u
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,
@@ -371,6 +378,14 @@ size_t gshard_dense_ffn_workspace_bytes(int64_t n_tokens, int32_t M, int32_t H, 
 int gshard_dense_ffn_forward(int64_t n_tokens, int32_t M, int32_t H, int32_t dtype, uint32_t flags,
                              const void* x, const void* wi, const void* wo, void* y, void* workspace,
                              size_t workspace_bytes, void* cuda_stream);
+
+/* The check that GSHARD_FLAG_DEBUG_CHECKS runs inside the forward, callable on its own: verifies
+ * the invariants Algorithm 1 implies for routing->expert_idx, slot, weight, flags and slot_token
+ * (all five required) and records GSHARD_ERR_INTERNAL in the status word of `workspace` (its first
+ * word; at least 256 bytes, 256-byte aligned) when one does not hold; read it with
+ * gshard_moe_last_device_status.  Indices are bounds-checked before they are used. */
+int gshard_moe_check_routing(const gshard_moe_shape* shape, const gshard_moe_routing* routing, void* workspace,
+                             void* cuda_stream);
 
 /* Self-test of the give-up path shared by every bounded device-side wait (the paper has no
  * counterpart; this is robustness plumbing).  Launches one small CTA that allocates tensor

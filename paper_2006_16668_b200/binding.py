@@ -40,6 +40,7 @@ GSHARD_FLAG_PLAIN_STORES = 2048
 GSHARD_FLAG_BWD_PAIRED_GEMMS = 4096
 GSHARD_FLAG_TF32_EXPERTS = 8192
 GSHARD_FLAG_COMPACT_SLOTS = 16384
+GSHARD_FLAG_DEBUG_CHECKS = 32768
 
 
 class gshard_moe_shape(Structure):
@@ -101,6 +102,7 @@ EXPORTS = {
     "gshard_dense_ffn_forward": (c_int, [ctypes.c_int64, c_int32, c_int32, c_int32, c_uint32] + [c_void_p] * 5 +
                                  [c_size_t, c_void_p]),
     "gshard_moe_debug_wait_timeout": (c_int, [c_void_p, c_uint32, c_void_p]),
+    "gshard_moe_check_routing": (c_int, [POINTER(gshard_moe_shape), POINTER(gshard_moe_routing), c_void_p, c_void_p]),
     "gshard_moe_last_device_status": (c_int, [c_void_p, c_void_p]),
     "gshard_moe_last_launch_count": (c_int, []),
     "gshard_moe_time_expert_ffn": (c_int, [c_void_p, c_void_p]),
@@ -335,6 +337,11 @@ def gshard_dense_ffn_forward(x, wi, wo, y, workspace, stream=None, flags=0):
 def gshard_moe_debug_wait_timeout(workspace, limit_us=200, stream=None):
     _check(load().gshard_moe_debug_wait_timeout(_p(workspace), int(limit_us), _stream(stream)),
            "gshard_moe_debug_wait_timeout")
+
+
+def gshard_moe_check_routing(shape, routing, workspace, stream=None):
+    _check(load().gshard_moe_check_routing(ctypes.byref(shape), ctypes.byref(routing), _p(workspace), _stream(stream)),
+           "gshard_moe_check_routing")
 
 
 def gshard_moe_last_device_status(workspace, stream=None) -> int:

@@ -56,6 +56,7 @@ int gate_logits(const Dims& d, const void* x, const void* wg, float* logits, int
 
 int gate_stage(const Dims& d, const FwdPlan& pl, unsigned char* ws, const void* x, const void* wg,
                int32_t* expert_idx, float* gate12, float* m, float* rowmax, float* rowinv, cudaStream_t st) {
+  NvtxRange range("gshard.gate");
   float* logits = reinterpret_cast<float*>(ws + pl.logits);
   int* status = reinterpret_cast<int*>(ws + pl.status);
   if (d.simt) {
@@ -96,6 +97,7 @@ bool ffn_runs_fused(const Dims& d, bool keep_h) {
 int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, void* h, bool keep_h, void* out,
               void* fused_scratch, int* status, cudaStream_t st, const void* x, const int32_t* slot_token,
               void* wt, const int* tile_base, uint32_t* relu_bits_out) {
+  NvtxRange range("gshard.expert_ffn");
   const long long rows = d.rows;
   // One persistent launch in which the hidden activations never leave L2: the faster form when
   // the FFN is bound by streaming the expert weights (at most one 128-row tile per expert); with
@@ -202,6 +204,7 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
   GS_TRY(gate_stage(d, pl, ws, x, wg, expert_idx, gate12, m, rowmax, rowinv, st));
   GS_TRY(launch_capacity(d, expert_idx, gate12, u, m, slot, weight, flags, first_count, total_count, slot_token,
                          l_aux_group, stats_group, l_aux, reinterpret_cast<long long*>(r.stats), st));
+  if (d.debug_checks) launch_routing_check(d, expert_idx, slot, weight, flags, slot_token, status, st);
   const bool gather = d.gather_dispatch && ffn_runs_fused(d, save);
   // compacted slots apply to the grouped-GEMM form of the FFN only
   const bool compact = d.compact_slots && !ffn_runs_fused(d, save);
@@ -528,6 +531,22 @@ int gshard_moe_last_device_status(void* workspace, void* cuda_stream) {
   int status = 0;
   if (cudaMemcpy(&status, workspace, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return GSHARD_ERR_CUDA;
   return status;
+}
+
+int gshard_moe_check_routing(const gshard_moe_shape* shape, const gshard_moe_routing* routing, void* workspace,
+                             void* cuda_stream) {
+  launch_counter().n = 0;
+  GS_TRY(validate_shape(shape));
+  if (!routing || !workspace || reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  GS_REQUIRE_PTR(routing->expert_idx); GS_REQUIRE_PTR(routing->slot); GS_REQUIRE_PTR(routing->weight);
+  GS_REQUIRE_PTR(routing->flags); GS_REQUIRE_PTR(routing->slot_token);
+  GS_TRY(check_device());
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  int* status = static_cast<int*>(workspace);
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  launch_routing_check(make_dims(*shape), routing->expert_idx, routing->slot, routing->weight, routing->flags,
+                       routing->slot_token, status, st);
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
 int gshard_moe_last_launch_count(void) { return launch_counter().n; }

@@ -241,6 +241,7 @@ template <typename T>
 int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, const void* wo, const unsigned char* ctx,
                const void* dy, float k_aux, void* dx, float* dwg, void* dwi, void* dwo, unsigned char* ws,
                cudaStream_t st) {
+  NvtxRange range("gshard.backward");
   const BwdPlan bp = plan_backward(d);
   const CtxPlan cp = plan_context(d);
   int* status = reinterpret_cast<int*>(ws + bp.status);
@@ -268,6 +269,7 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   const long long rows = d.rows;
 
   // combine backward
+  nvtxRangePushA("gshard.backward.combine");
   combine_bwd_kernel<T><<<grid_for_rows(d.N), 256, 0, st>>>(reinterpret_cast<const uint4*>(dy),
                                                         reinterpret_cast<const uint4*>(out), expert_idx, slot, dw, d.N,
                                                         d.G, d.S, d.C, row_vec);
@@ -275,6 +277,8 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
                                                  weight, reinterpret_cast<uint4*>(dout), d.R, d.G, d.S, d.C, row_vec);
   count_launch(2);
 
+  nvtxRangePop();
+  nvtxRangePushA("gshard.backward.expert_ffn");
   // expert FFN backward.  dh and dbuf stream the weights (read-heavy), dwo and dwi write a gradient the
   // size of the weights from short contractions (write-heavy): one of each runs side by side.
   UmmaGemm g_dh{}, g_dwo{}, g_dwi{}, g_dbuf{};
@@ -305,6 +309,8 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
   rc = run_gemm_pair(d, g_dbuf, g_dwi, share, status, st);
   if (rc) return rc;
 
+  nvtxRangePop();
+  NvtxRange gate_range("gshard.backward.gate");
   // gating backward: recompute the logits, softmax backward, two GEMMs
   rc = gate_logits(d, x, wg, logits, status, st);
   if (rc) return rc;

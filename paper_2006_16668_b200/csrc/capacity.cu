@@ -196,6 +196,57 @@ __global__ void capacity_finalize_kernel(const float* l_aux_group, const int32_t
   }
 }
 
+// Debug check (GSHARD_FLAG_DEBUG_CHECKS, gshard_moe_check_routing): what Algorithm 1 implies for the
+// routing tensors.  Per token: two distinct experts in [0, E), positions in [-1, C), flag bits that
+// agree with the positions, normalised weights that sum to one, and the slot a kept choice names
+// holds this token.  Per slot: a token index in [-1, S), and the token it names lists this slot.
+// A violation records GSHARD_ERR_INTERNAL in the status word; every access is bounds-checked first.
+__global__ void __launch_bounds__(256) routing_check_kernel(const int32_t* __restrict__ expert_idx,
+                                                            const int32_t* __restrict__ slot,
+                                                            const float* __restrict__ weight,
+                                                            const uint8_t* __restrict__ flags,
+                                                            const int32_t* __restrict__ slot_token, long long N,
+                                                            long long R, int G, int S, int E, int C, int* status) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  bool bad = false;
+  if (i < N) {
+    const int g = (int)(i / S), s = (int)(i % S);
+    const int e[2] = {expert_idx[2 * i], expert_idx[2 * i + 1]};
+    const int p[2] = {slot[2 * i], slot[2 * i + 1]};
+    const float w1 = weight[2 * i], w2 = weight[2 * i + 1];
+    const unsigned f = flags[i];
+    bad |= e[0] < 0 || e[0] >= E || e[1] < 0 || e[1] >= E || e[0] == e[1];
+    bad |= !(w1 >= 0.5f - 1e-6f) || !(w2 >= 0.f) || !(fabsf(w1 + w2 - 1.f) <= 1e-5f);
+    bad |= ((f & 1u) != 0) != (p[0] >= 0) || ((f & 4u) != 0) != (p[1] >= 0) || ((f & 4u) && !(f & 2u)) || (f & ~7u);
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      if (p[k] < -1 || p[k] >= C) { bad = true; continue; }
+      if (p[k] >= 0 && e[k] >= 0 && e[k] < E) bad |= slot_token[((long long)e[k] * G + g) * C + p[k]] != s;
+    }
+  }
+  if (i < R) {
+    const int tok = slot_token[i];
+    const int c = (int)(i % C), g = (int)((i / C) % G), e = (int)(i / ((long long)C * G));
+    if (tok < -1 || tok >= S) {
+      bad = true;
+    } else if (tok >= 0) {
+      const long long t = (long long)g * S + tok;
+      const bool first = expert_idx[2 * t] == e && slot[2 * t] == c;
+      const bool second = expert_idx[2 * t + 1] == e && slot[2 * t + 1] == c;
+      bad |= !(first || second);
+    }
+  }
+  if (bad) set_device_status(status, GSHARD_ERR_INTERNAL);
+}
+
+void launch_routing_check(const Dims& d, const int32_t* expert_idx, const int32_t* slot, const float* weight,
+                          const uint8_t* flags, const int32_t* slot_token, int* status, cudaStream_t st) {
+  const long long n = d.N > d.R ? d.N : d.R;
+  routing_check_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(expert_idx, slot, weight, flags, slot_token, d.N, d.R,
+                                                                    d.G, d.S, d.E, d.C, status);
+  count_launch();
+}
+
 size_t capacity_smem_bytes(int E, int warps) { return (size_t)E * 4 + (size_t)warps * E * 2; }
 
 int capacity_warps_for(int E) {
@@ -208,6 +259,7 @@ int launch_capacity(const Dims& d, const int32_t* expert_idx, const float* gate1
                     const float* m, int32_t* slot, float* weight, uint8_t* flags, int32_t* first_count,
                     int32_t* total_count, int32_t* slot_token, float* l_aux_group, int32_t* stats_group,
                     float* l_aux, long long* stats, cudaStream_t st, int groups_in_mean) {
+  NvtxRange range("gshard.capacity");
   CapacityArgs a;
   a.S = d.S; a.E = d.E; a.C = d.C; a.G = d.G;
   a.warps_used = capacity_warps_for(d.E);

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
 
 #include "../../include/gshard_moe.h"
@@ -75,6 +76,14 @@ inline int grid_for_rows(long long rows) {
   return (int)(blocks < cap ? (blocks > 0 ? blocks : 1) : cap);
 }
 
+// NVTX range around a stage's launches (header-only NVTX 3: a no-op unless a profiler injects itself).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+  NvtxRange(const NvtxRange&) = delete;
+  NvtxRange& operator=(const NvtxRange&) = delete;
+};
+
 struct LaunchCounter {
   int n = 0;
 };
@@ -103,6 +112,7 @@ struct Dims {
   bool tf32_experts;    // fp32 dtype: expert FFN contractions on the tensor cores in TF32
   bool compact_slots;   // grouped-GEMM expert FFN over compacted rows (empty slots skipped)
   bool plain_stores;    // GEMM epilogues write with 16-byte stores instead of bulk tensor (TMA) stores
+  bool debug_checks;    // forward: verify the routing tensors on the device and record a violation in the status word
   bool bwd_paired;      // backward: read-heavy and write-heavy expert GEMMs side by side on half of the SMs each
 };
 
@@ -127,6 +137,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.add_residual = (s.flags & GSHARD_FLAG_ADD_RESIDUAL) != 0;
   d.bwd_paired = (s.flags & GSHARD_FLAG_BWD_PAIRED_GEMMS) != 0;
   d.plain_stores = (s.flags & GSHARD_FLAG_PLAIN_STORES) != 0;
+  d.debug_checks = (s.flags & GSHARD_FLAG_DEBUG_CHECKS) != 0;
   d.tf32_experts = !d.bf16 && (s.flags & GSHARD_FLAG_TF32_EXPERTS) != 0;
   // Compacted slots: on request, and by default where an expert has at least six 128-row tiles, so
   // that the usual 13-30 % of empty slots free at least one of them (measured at the MoE(128E) shape:

@@ -138,6 +138,7 @@ __global__ void __launch_bounds__(256) dispatch_compact_kernel(const uint4* __re
 
 void launch_dispatch_compact(const Dims& d, const void* x, const int32_t* crow_token, const int32_t* kept, void* buf,
                              cudaStream_t st) {
+  NvtxRange range("gshard.dispatch");
   const int row_vec = (int)((size_t)d.M * d.esize / 16);
   dispatch_compact_kernel<<<grid_for_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(x), crow_token, kept,
                                                               reinterpret_cast<uint4*>(buf), d.R, d.rows, d.N, row_vec);
@@ -145,6 +146,7 @@ void launch_dispatch_compact(const Dims& d, const void* x, const int32_t* crow_t
 }
 
 void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st) {
+  NvtxRange range("gshard.dispatch");
   const int row_vec = (int)((size_t)d.M * d.esize / 16);
   dispatch_kernel<<<grid_for_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(x), slot_token,
                                                       reinterpret_cast<uint4*>(buf), d.R, d.G, d.S, d.C, row_vec);
@@ -153,6 +155,7 @@ void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, vo
 
 void launch_combine(const Dims& d, const void* out, const int32_t* expert_idx, const int32_t* slot,
                     const float* weight, void* y, cudaStream_t st, const void* residual, const int32_t* slot_crow) {
+  NvtxRange range("gshard.combine");
   const int row_vec = (int)((size_t)d.M * d.esize / 16);
   if (d.bf16)
     combine_kernel<__nv_bfloat16><<<grid_for_rows(d.N), 256, 0, st>>>(

@@ -34,6 +34,10 @@ int launch_capacity(const Dims& d, const int32_t* expert_idx, const float* gate1
                     int32_t* slot_token, float* l_aux_group, int32_t* stats_group, float* l_aux, long long* stats,
                     cudaStream_t st, int groups_in_mean = 0);
 int capacity_warps_for(int E);
+// Debug check of the routing tensors (every invariant Algorithm 1 implies for them); a violation
+// records GSHARD_ERR_INTERNAL in *status, nothing traps.
+void launch_routing_check(const Dims& d, const int32_t* expert_idx, const int32_t* slot, const float* weight,
+                          const uint8_t* flags, const int32_t* slot_token, int* status, cudaStream_t st);
 
 // dispatch_combine.cu
 void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st);

@@ -97,3 +97,71 @@ def test_dispatch_and_combine_skip_out_of_range_indices(dtype):
                     continue
                 ref[g, s] += float(w[g, s, k]) * ob[ei[g, s, k], g, slot[g, s, k]]
     assert rel_fro(to_np(y), ref) < (1e-6 if dtype == "f32" else 4e-3)
+
+
+def test_debug_checks_pass_on_a_healthy_forward_and_catch_corrupted_routing():
+    """GSHARD_FLAG_DEBUG_CHECKS verifies the routing tensors inside the forward (status stays OK, results
+    are the same bits as without the flag); gshard_moe_check_routing, the same kernel on its own, must
+    record GSHARD_ERR_INTERNAL for each kind of corruption - and survive indices that point far outside
+    the tensors, because it bounds-checks before it dereferences."""
+    from paper_2006_16668_b200 import MoEConfig
+    cfg = MoEConfig("dbg", G=3, S=200, M=64, H=128, E=16, C=20, dtype="bf16", seed=12)
+    inp = make_inputs(cfg, "cuda")
+    outs = []
+    for flags in (0, B.GSHARD_FLAG_DEBUG_CHECKS):
+        shape = B.make_shape(cfg, flags=flags)
+        ws = B.alloc_workspace(shape)
+        rt, rs = B.alloc_routing(shape)
+        y = torch.empty_like(inp["x"])
+        l_aux = torch.zeros(1, device="cuda")
+        B.gshard_moe_top2_forward(shape, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l_aux, rs, None, ws)
+        assert B.gshard_moe_last_device_status(ws) == B.GSHARD_OK
+        outs.append((y, rt, B.gshard_moe_last_launch_count()))
+    assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16))
+    assert outs[1][2] == outs[0][2] + 1                      # one more kernel: the check
+    shape = B.make_shape(cfg)
+    ws = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    good = outs[0][1]
+
+    def status_of(**changed):
+        t = {k: v.clone() for k, v in good.items()}
+        for k, fn in changed.items():
+            fn(t[k])
+        B.gshard_moe_check_routing(shape, B.routing_struct(t), ws)
+        return B.gshard_moe_last_device_status(ws)
+
+    assert status_of() == B.GSHARD_OK
+    kept = (good["slot"][..., 0] >= 0).nonzero()[0].tolist()           # a token whose first choice was kept
+    g, s = kept
+
+    def bump_slot(t):
+        t[g, s, 0] = (t[g, s, 0] + 1) % cfg.C
+
+    def far_expert(t):
+        t[g, s, 1] = 1 << 24
+
+    def same_experts(t):
+        t[g, s, 1] = t[g, s, 0]
+
+    def huge_slot(t):
+        t[g, s, 0] = 1 << 20
+
+    def wrong_token(t):
+        e = int(good["expert_idx"][g, s, 0])
+        t[e, g, int(good["slot"][g, s, 0])] = (s + 1) % cfg.S
+
+    def far_token(t):
+        t[0, 0, 0] = 1 << 28
+
+    def bad_weight(t):
+        t[g, s, 0] = 0.9
+        t[g, s, 1] = 0.3
+
+    def bad_flag(t):
+        t[g, s] = t[g, s] ^ 1
+
+    for change in (dict(slot=bump_slot), dict(expert_idx=far_expert), dict(expert_idx=same_experts),
+                   dict(slot=huge_slot), dict(slot_token=wrong_token), dict(slot_token=far_token),
+                   dict(weight=bad_weight), dict(flags=bad_flag)):
+        assert status_of(**change) == B.GSHARD_ERR_INTERNAL, list(change)
+    assert status_of() == B.GSHARD_OK                        # the workspace's status word is reset per call
