@@ -147,6 +147,7 @@ class ClockSampler(threading.Thread):
         super().__init__(daemon=True)
         self.index = index
         self.samples = []
+        self.times = []          # host time at which each sample arrived
         self.proc = None
 
     def run(self):
@@ -157,6 +158,7 @@ class ClockSampler(threading.Thread):
                 parts = [p.strip() for p in line.strip().split(",")]
                 if len(parts) >= 6:
                     self.samples.append(parts)
+                    self.times.append(time.time())
         except Exception:
             pass
 
@@ -374,26 +376,46 @@ class Bench:
 
     def sustained(self, seconds: float, ms_per_step_hint: float) -> dict:
         """The same step back to back for at least `seconds`: what the layer does once the board has
-        settled under its power cap.  ms x MHz makes runs at different clocks comparable."""
+        settled under its power cap.  ms x MHz makes runs at different clocks comparable, and
+        `by_clock` gives the mean step time per band of the SM clock sampled while the step ran (the
+        run starts near the maximum clock and sinks), i.e. how the step time depends on the clock."""
         torch = self.torch
         steps = max(10, int(math.ceil(seconds * 1e3 / ms_per_step_hint * 1.1)))
         self.barrier()
         c0 = self.sampler.mark()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(self.stream)
-        for _ in range(steps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        t0 = time.time()
+        ev[0].record(self.stream)
+        for i in range(steps):
             self.step()
-        e1.record(self.stream)
+            ev[i + 1].record(self.stream)
         self.barrier()
-        total_ms = max_over_ranks(e0.elapsed_time(e1), self.world, self.dev)
+        total_ms = max_over_ranks(ev[0].elapsed_time(ev[-1]), self.world, self.dev)
         time.sleep(0.06)
         clocks = self.sampler.summary(c0)
         self.require_ok("the sustained run")
         ms = total_ms / steps
+        # step times against the clock sample nearest in time (the GPU runs the queued steps from t0 on)
+        samples = [(t, float(p[0])) for t, p in zip(self.sampler.times[c0:], self.sampler.samples[c0:])
+                   if p[0].replace(".", "").isdigit()]
+        bands = [(0, 1000), (1000, 1200), (1200, 1400), (1400, 1600), (1600, 1800), (1800, 10000)]
+        acc = {b: [] for b in bands}
+        done = 0.0
+        for i in range(steps):
+            step_ms = ev[i].elapsed_time(ev[i + 1])
+            mid = t0 + (done + 0.5 * step_ms) * 1e-3
+            done += step_ms
+            if samples:
+                mhz = min(samples, key=lambda s: abs(s[0] - mid))[1]
+                for b in bands:
+                    if b[0] <= mhz < b[1]:
+                        acc[b].append(step_ms)
+        by_clock = {f"{b[0]}-{b[1]} MHz" if b[1] < 10000 else f">={b[0]} MHz":
+                    {"steps": len(v), "ms_per_step": sum(v) / len(v)} for b, v in acc.items() if v}
         return {"steps": steps, "seconds": total_ms * 1e-3, "ms_per_step": ms,
                 "value": aggregate_throughput(self.cfg.N, self.world, ms), "sm_mhz": clocks["sm_mhz"],
                 "ms_x_mhz": ms * clocks["sm_mhz"] if clocks["sm_mhz"] else None, "reasons": clocks["reasons"],
-                "clock_samples": clocks["samples_under_load"]}
+                "clock_samples": clocks["samples_under_load"], "by_clock": by_clock}
 
     # ---- records ------------------------------------------------------------------------------------
     def rooflines(self, rec: dict):
