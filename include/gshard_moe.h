@@ -52,9 +52,10 @@ typedef enum {
 
 typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
 
-/* flags of gshard_moe_shape.  Bits 4..2048 choose between kernel forms of the bf16 tensor-core
- * path; the defaults are the forms that measured fastest on B200, results agree within the stated
- * tolerances whichever form runs. */
+/* flags of gshard_moe_shape.  Bits 1, 2, 1024 and 8192 change what is computed or kept (saved context,
+ * reading of the second loop, residual, TF32); the others choose between kernel forms of the bf16
+ * tensor-core path or add checks; the defaults are the forms that measured fastest on B200, results
+ * agree within the stated tolerances whichever form runs. */
 #define GSHARD_FLAG_SAVE_FOR_BACKWARD 1u      /* forward fills `context` for the backward call */
 #define GSHARD_FLAG_SECOND_SKIP_FREES_SLOT 2u /* other reading of Algorithm 1's second loop: a token
                                                  that fails 2*g2 > rnd does not advance the counter
