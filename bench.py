@@ -589,6 +589,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "ep"],
                     help="N > 1: independent replicas, or groups and experts sharded with two all-to-alls")
+    ap.add_argument("--ep-comm", default="nccl", choices=["nccl", "torch"],
+                    help="--parallelism ep: collectives as NCCL calls inside the library, or torch.distributed callbacks")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra-configs", action="store_true", help="measure only --config")

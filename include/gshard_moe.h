@@ -336,6 +336,15 @@ typedef struct {
   void* user;
 } gshard_ep_comm;
 
+/* The same collectives through NCCL itself, for callers that hold an ncclComm_t: all_to_all becomes
+ * one NCCL group of `world` sends and receives of equal slabs, all_reduce_sum_f32 an ncclAllReduce,
+ * both on the call's stream, with no callback into the caller's language.  nccl_comm: an initialised
+ * communicator of `world` ranks (an ncclComm_t passed as void*), owned by the caller and outliving
+ * `comm`; `state`: storage that `comm` points into, which must outlive it too.  NCCL is not linked:
+ * its functions are looked up in the process at run time (GSHARD_ERR_INTERNAL when there is none). */
+typedef struct { void* opaque[8]; } gshard_ep_nccl_state;
+int gshard_ep_comm_from_nccl(void* nccl_comm, int world, gshard_ep_nccl_state* state, gshard_ep_comm* comm);
+
 /* Host-only: validates the partitioning and fills `layout`.  GSHARD_ERR_UNSUPPORTED_SHAPE when G or
  * E is not a multiple of world (or SAVE_FOR_BACKWARD is set: the expert-parallel form is forward only). */
 int gshard_moe_ep_plan(const gshard_moe_shape* shape, int rank, int world, gshard_moe_ep_layout* layout);

@@ -68,6 +68,10 @@ class gshard_ep_comm(Structure):
     _fields_ = [("all_to_all", ALL_TO_ALL_FN), ("all_reduce_sum_f32", ALL_REDUCE_FN), ("user", c_void_p)]
 
 
+class gshard_ep_nccl_state(Structure):
+    _fields_ = [("opaque", c_void_p * 8)]
+
+
 EXPORTS = {
     # name: (restype, argtypes)
     "gshard_version": (c_int, []),
@@ -93,6 +97,7 @@ EXPORTS = {
     "gshard_moe_expert_ffn": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 5 + [c_size_t, c_void_p]),
     "gshard_moe_combine": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6),
     "gshard_moe_ep_plan": (c_int, [POINTER(gshard_moe_shape), c_int, c_int, POINTER(gshard_moe_ep_layout)]),
+    "gshard_ep_comm_from_nccl": (c_int, [c_void_p, c_int, POINTER(gshard_ep_nccl_state), POINTER(gshard_ep_comm)]),
     "gshard_moe_ep_regroup_host": (c_int, [POINTER(gshard_moe_ep_layout), c_void_p, c_void_p, c_size_t, c_int]),
     "gshard_moe_ep_workspace_bytes": (c_size_t, [POINTER(gshard_moe_shape), c_int]),
     "gshard_moe_top2_forward_ep": (c_int, [POINTER(gshard_moe_shape), c_int, c_int] + [c_void_p] * 7 +
@@ -302,6 +307,15 @@ def gshard_moe_ep_regroup_host(layout, src, dst, inverse=False):
     assert src.is_contiguous() and dst.is_contiguous() and src.numel() == dst.numel()
     _check(load().gshard_moe_ep_regroup_host(ctypes.byref(layout), src.data_ptr(), dst.data_ptr(), row_bytes,
                                              int(bool(inverse))), "gshard_moe_ep_regroup_host")
+
+
+def gshard_ep_comm_from_nccl(nccl_comm: int, world: int):
+    """(comm, state): a gshard_ep_comm whose collectives are NCCL calls on the given ncclComm_t handle;
+    keep both objects (and the communicator) alive while the comm is in use."""
+    state, comm = gshard_ep_nccl_state(), gshard_ep_comm()
+    _check(load().gshard_ep_comm_from_nccl(nccl_comm, int(world), ctypes.byref(state), ctypes.byref(comm)),
+           "gshard_ep_comm_from_nccl")
+    return comm, state
 
 
 def gshard_moe_ep_workspace_bytes(shape, world) -> int:

@@ -8,6 +8,7 @@ shares of l_aux) and slices each rank's share out of global tensors.
 """
 from __future__ import annotations
 
+import ctypes
 import traceback
 
 import torch
@@ -59,6 +60,62 @@ class TorchDistComm:
             return 1
 
 
+class NcclComm:
+    """The collectives as direct NCCL calls from inside the library (no Python in the data path).
+
+    Creates its own ncclComm_t with the NCCL library torch has loaded: rank 0 draws the unique id, the
+    process group (any backend) carries it to the other ranks, every rank joins with
+    ncclCommInitRank.  One GPU per process, the current device.
+    """
+
+    class _UniqueId(ctypes.Structure):
+        _fields_ = [("internal", ctypes.c_byte * 128)]
+
+    def __init__(self, rank: int, world: int, group=None):
+        self.lib = self._load_nccl()
+        self.rank, self.world = rank, world
+        uid = self._UniqueId()
+        if rank == 0:
+            self._ok(self.lib.ncclGetUniqueId(ctypes.byref(uid)), "ncclGetUniqueId")
+        if world > 1:
+            payload = [bytes(uid.internal) if rank == 0 else None]
+            dist.broadcast_object_list(payload, src=0, group=group)
+            ctypes.memmove(ctypes.byref(uid), payload[0], 128)
+        self.handle = ctypes.c_void_p()
+        self.lib.ncclCommInitRank.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, self._UniqueId, ctypes.c_int]
+        self._ok(self.lib.ncclCommInitRank(ctypes.byref(self.handle), world, uid, rank), "ncclCommInitRank")
+        self.struct, self._state = B.gshard_ep_comm_from_nccl(self.handle.value, world)
+
+    @staticmethod
+    def _load_nccl():
+        import glob
+        import os
+        cands = []
+        try:
+            import nvidia.nccl
+            for d in list(getattr(nvidia.nccl, "__path__", [])):       # a namespace package has no __file__
+                cands += sorted(glob.glob(os.path.join(d, "lib", "libnccl.so*")))
+        except ImportError:
+            pass
+        for path in cands + ["libnccl.so.2"]:
+            try:
+                return ctypes.CDLL(path, mode=ctypes.RTLD_GLOBAL)
+            except OSError:
+                continue
+        raise ImportError("no NCCL library found")
+
+    @staticmethod
+    def _ok(code, what):
+        if code != 0:
+            raise RuntimeError(f"{what} failed with NCCL result {code}")
+
+    def close(self):
+        if self.handle:
+            self.lib.ncclCommDestroy.argtypes = [ctypes.c_void_p]
+            self.lib.ncclCommDestroy(self.handle)
+            self.handle = ctypes.c_void_p()
+
+
 def local_slices(layout: B.gshard_moe_ep_layout):
     """(group slice, expert slice) of this rank in the global tensors."""
     g0, e0 = layout.group_begin, layout.expert_begin
@@ -66,10 +123,14 @@ def local_slices(layout: B.gshard_moe_ep_layout):
 
 
 def forward(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux, routing_out=None,
-            workspace=None, group=None):
+            workspace=None, group=None, comm=None):
     """One expert-parallel forward on this rank (global `shape`); the process group must be
-    initialised when world > 1.  Enqueues on torch's current stream."""
-    comm = None
+    initialised when world > 1.  Enqueues on torch's current stream.  comm: a NcclComm to reuse, else
+    the collectives go through torch.distributed."""
+    if comm is not None:
+        B.gshard_moe_top2_forward_ep(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux,
+                                     routing_out, comm.struct, workspace)
+        return
     if world > 1:
         comm = TorchDistComm(workspace, l_aux, group)
     try:

@@ -31,8 +31,11 @@ def run(args, cfg, dev, world, rank, metric, unit, sampler):
     ws = torch.empty(B.gshard_moe_ep_workspace_bytes(shape, world), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
+    # collectives: NCCL called from inside the library (default), or torch.distributed through callbacks
+    comm = ep.NcclComm(rank, world) if (world > 1 and getattr(args, "ep_comm", "nccl") == "nccl") else None
+
     def step():
-        ep.forward(shape, rank, world, x, wg, wi, wo, u, y, l_aux, None, ws)
+        ep.forward(shape, rank, world, x, wg, wi, wo, u, y, l_aux, None, ws, comm=comm)
 
     def barrier():
         if world > 1:

@@ -202,3 +202,36 @@ def test_bad_arguments():
     # world > 1 needs the collectives
     assert lib.gshard_moe_top2_forward_ep(ctypes.byref(shape), 0, 2, *args, fake, None, None, fake, 1 << 40, None) == B.GSHARD_ERR_INVALID_ARG
     assert lib.gshard_moe_top2_forward_ep(ctypes.byref(shape), 0, 1, *args, fake, None, None, fake, 16, None) == B.GSHARD_ERR_WORKSPACE_TOO_SMALL
+
+
+def test_nccl_comm_single_rank():
+    """The NCCL-backed collectives at world 1 (all that one GPU can run): the all-to-all is a group of
+    one send and one receive to the rank itself, the all-reduce an identity; both are called through the
+    function pointers the library fills in, then the expert-parallel forward runs with that comm."""
+    import ctypes
+    comm = ep.NcclComm(0, 1)
+    try:
+        stream = torch.cuda.current_stream().cuda_stream
+        send = torch.randint(0, 255, (4096,), dtype=torch.uint8, device="cuda")
+        recv = torch.zeros_like(send)
+        assert comm.struct.all_to_all(comm.struct.user, send.data_ptr(), recv.data_ptr(), send.numel(), stream) == 0
+        v = torch.tensor([1.5, -2.0], device="cuda")
+        assert comm.struct.all_reduce_sum_f32(comm.struct.user, v.data_ptr(), 2, stream) == 0
+        torch.cuda.synchronize()
+        assert torch.equal(recv, send) and v.tolist() == [1.5, -2.0]
+        cfg = MoEConfig("nccl1", G=4, S=128, M=64, H=128, E=16, C=16, dtype="bf16", seed=3)
+        inp = make_inputs(cfg, "cuda")
+        y_ref, l_ref, _ = _single(cfg, inp)
+        shape = B.make_shape(cfg)
+        ws = torch.empty(B.gshard_moe_ep_workspace_bytes(shape, 1), dtype=torch.uint8, device="cuda")
+        y = torch.empty_like(inp["x"])
+        l_aux = torch.zeros(1, device="cuda")
+        ep.forward(shape, 0, 1, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l_aux, None, ws, comm=comm)
+        assert B.gshard_moe_last_device_status(ws) == B.GSHARD_OK
+        assert torch.equal(y.view(torch.int16), y_ref.view(torch.int16)) and torch.equal(l_aux, l_ref)
+    finally:
+        comm.close()
+    # without a communicator the constructor refuses
+    lib = B.load()
+    state, c = B.gshard_ep_nccl_state(), B.gshard_ep_comm()
+    assert lib.gshard_ep_comm_from_nccl(None, 1, ctypes.byref(state), ctypes.byref(c)) == B.GSHARD_ERR_INVALID_ARG
