@@ -589,8 +589,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "ep"],
                     help="N > 1: independent replicas, or groups and experts sharded with two all-to-alls")
-    ap.add_argument("--ep-comm", default="nccl", choices=["nccl", "torch"],
-                    help="--parallelism ep: collectives as NCCL calls inside the library, or torch.distributed callbacks")
+    ap.add_argument("--ep-comm", default="nccl", choices=["nccl", "torch", "p2p"],
+                    help="--parallelism ep: collectives as NCCL calls inside the library, torch.distributed callbacks, "
+                         "or no collective: peer stores/loads inside the dispatch and combine kernels")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extra-configs", action="store_true", help="measure only --config")
@@ -625,14 +626,18 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the layer has no CPU path")
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl")
+    p2p_single = world == 1 and args.parallelism == "ep" and args.ep_comm == "p2p"
+    if p2p_single:                        # symmetric memory wants a process group even for one rank
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29517")
+    if world > 1 or p2p_single:
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=torch.device("cuda", local_rank))
     dev = torch.device("cuda", local_rank)
     args.warmup = max(args.warmup, 3)
     if args.parallelism == "ep":
         from paper_2006_16668_b200 import ep_bench
         ep_bench.run(args, cfg, dev, world, rank, METRIC, UNIT, ClockSampler(local_rank))
-        if world > 1:
+        if dist.is_initialized():
             dist.destroy_process_group()
         return
 

@@ -374,6 +374,37 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
                                const gshard_moe_routing* routing_out, const gshard_ep_comm* comm,
                                void* workspace, size_t workspace_bytes, void* cuda_stream);
 
+/* The expert-parallel forward with the exchange FUSED into the dispatch and combine kernels (same
+ * partitioning and results as gshard_moe_top2_forward_ep).  The dispatch kernel stores each token row
+ * directly into the expert owner's input buffer over NVLink, already in the layout the expert FFN
+ * reads; the combine kernel loads a token's expert output rows directly from the owners' output
+ * buffers.  No AllToAll and no regrouping copy remain; the expert FFN reads and writes only this GPU's
+ * own memory; nothing is multicast.
+ *   peer_buffers[w]: rank w's exchange buffer (gshard_moe_ep_p2p_buffer_bytes each, 256-byte aligned)
+ *   as a device pointer valid in THIS process (peer access enabled / an IPC or symmetric-memory
+ *   mapping); entry [rank] is this rank's own buffer.  First half: the FFN input of the rank's experts
+ *   [E/world][G*C][M], written by every rank; second half: their output, read by every rank.
+ *   rendezvous(user, phase, stream): orders the ranks - it must make this rank's stream publish that
+ *   its work enqueued so far has completed AND wait for the same from every other rank (for instance
+ *   one interprocess event per rank: record mine, wait on the others').  Called with phase 0 (the
+ *   previous use of the buffers is over), 1 (all rows have arrived) and 2 (all expert outputs are
+ *   complete); returns 0 on success.  No kernel of this library waits for another rank's kernel.
+ *   comm: optional, only its all_reduce_sum_f32 is used (for l_aux; without it l_aux holds this rank's
+ *   share, sum of its group losses / G).  workspace: gshard_moe_top2_workspace_bytes of the LOCAL shape
+ *   (layout.local) suffices. */
+typedef struct {
+  int (*rendezvous)(void* user, int phase, void* cuda_stream);
+  void* user;
+  void* const* peer_buffers;   /* [world] */
+} gshard_ep_p2p;
+size_t gshard_moe_ep_p2p_buffer_bytes(const gshard_moe_shape* shape, int world);
+int gshard_moe_top2_forward_ep_p2p(const gshard_moe_shape* shape, int rank, int world, const void* x_local,
+                                   const void* wg, const void* wi_local, const void* wo_local,
+                                   const float* u_local, void* y_local, float* l_aux,
+                                   const gshard_moe_routing* routing_out, const gshard_ep_p2p* p2p,
+                                   const gshard_ep_comm* comm, void* workspace, size_t workspace_bytes,
+                                   void* cuda_stream);
+
 /* The position-wise feed-forward sub-layer of the ordinary Transformer layers that alternate with
  * the MoE layers (section 2.1: every other feed-forward layer is replaced by a MoE layer; the
  * performance section times "MoE layer + adjacent Transformer layer"): y = relu(x . wi) . wo over

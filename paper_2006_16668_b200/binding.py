@@ -68,6 +68,13 @@ class gshard_ep_comm(Structure):
     _fields_ = [("all_to_all", ALL_TO_ALL_FN), ("all_reduce_sum_f32", ALL_REDUCE_FN), ("user", c_void_p)]
 
 
+RENDEZVOUS_FN = ctypes.CFUNCTYPE(c_int, c_void_p, c_int, c_void_p)
+
+
+class gshard_ep_p2p(Structure):
+    _fields_ = [("rendezvous", RENDEZVOUS_FN), ("user", c_void_p), ("peer_buffers", POINTER(c_void_p))]
+
+
 class gshard_ep_nccl_state(Structure):
     _fields_ = [("opaque", c_void_p * 8)]
 
@@ -97,6 +104,10 @@ EXPORTS = {
     "gshard_moe_expert_ffn": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 5 + [c_size_t, c_void_p]),
     "gshard_moe_combine": (c_int, [POINTER(gshard_moe_shape)] + [c_void_p] * 6),
     "gshard_moe_ep_plan": (c_int, [POINTER(gshard_moe_shape), c_int, c_int, POINTER(gshard_moe_ep_layout)]),
+    "gshard_moe_ep_p2p_buffer_bytes": (c_size_t, [POINTER(gshard_moe_shape), c_int]),
+    "gshard_moe_top2_forward_ep_p2p": (c_int, [POINTER(gshard_moe_shape), c_int, c_int] + [c_void_p] * 7 +
+                                       [POINTER(gshard_moe_routing), POINTER(gshard_ep_p2p), POINTER(gshard_ep_comm),
+                                        c_void_p, c_size_t, c_void_p]),
     "gshard_ep_comm_from_nccl": (c_int, [c_void_p, c_int, POINTER(gshard_ep_nccl_state), POINTER(gshard_ep_comm)]),
     "gshard_moe_ep_regroup_host": (c_int, [POINTER(gshard_moe_ep_layout), c_void_p, c_void_p, c_size_t, c_int]),
     "gshard_moe_ep_workspace_bytes": (c_size_t, [POINTER(gshard_moe_shape), c_int]),
@@ -307,6 +318,20 @@ def gshard_moe_ep_regroup_host(layout, src, dst, inverse=False):
     assert src.is_contiguous() and dst.is_contiguous() and src.numel() == dst.numel()
     _check(load().gshard_moe_ep_regroup_host(ctypes.byref(layout), src.data_ptr(), dst.data_ptr(), row_bytes,
                                              int(bool(inverse))), "gshard_moe_ep_regroup_host")
+
+
+def gshard_moe_ep_p2p_buffer_bytes(shape, world) -> int:
+    return int(load().gshard_moe_ep_p2p_buffer_bytes(ctypes.byref(shape), int(world)))
+
+
+def gshard_moe_top2_forward_ep_p2p(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux,
+                                   routing_out, p2p, comm, workspace, stream=None):
+    rp = ctypes.byref(routing_out) if routing_out is not None else None
+    cp = ctypes.byref(comm) if comm is not None else None
+    _check(load().gshard_moe_top2_forward_ep_p2p(ctypes.byref(shape), int(rank), int(world), _p(x_local), _p(wg),
+                                                 _p(wi_local), _p(wo_local), _p(u_local), _p(y_local), _p(l_aux), rp,
+                                                 ctypes.byref(p2p), cp, _p(workspace), workspace.numel(), _stream(stream)),
+           "gshard_moe_top2_forward_ep_p2p")
 
 
 def gshard_ep_comm_from_nccl(nccl_comm: int, world: int):

@@ -196,3 +196,203 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Expert-parallel forward with the exchange fused into the dispatch and combine kernels.
+//
+// Instead of dispatching into a local buffer and handing it to an AllToAll, the dispatch kernel
+// writes every token row straight into the expert owner's input buffer over NVLink (peer stores),
+// already in the layout the expert FFN reads ([El][G*C][M], rows in global group order), and the
+// combine kernel gathers a token's (at most two) expert output rows straight out of the owners'
+// output buffers (peer loads).  Each row crosses NVLink once, inside the kernel that produces or
+// consumes it; the two AllToAll passes and the two regrouping copies of the collective form
+// disappear.  The expert FFN itself only ever reads and writes this GPU's own memory (its TMA
+// tensor maps never cover a peer's memory), and nothing is multicast.
+// Ordering between ranks is the caller's, through one callback: rendezvous(phase) must make this
+// rank's stream (a) publish "my work enqueued so far is done" and (b) wait for the same from every
+// other rank - e.g. an interprocess event per rank, recorded and waited on; no kernel waits for
+// another rank's kernel.
+namespace gshard {
+namespace {
+
+constexpr int kMaxPeers = 64;
+struct PeerPtrs { unsigned char* p[kMaxPeers]; };
+
+// in_of(d) = peer d's exchange buffer; its first half is the FFN input [El][G*C][M], its second half
+// the FFN output.  Row of (local expert el, global group g, position c): (el*G + g)*C + c.
+template <typename V>
+__global__ void __launch_bounds__(256) dispatch_p2p_kernel(const V* __restrict__ x, const int32_t* __restrict__ slot_token,
+                                                           PeerPtrs peers, long long rows_all, int G, int Gl, int S, int C,
+                                                           int El, int rank, int row_vec) {
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long r = warp; r < rows_all; r += nwarps) {       // r = (e*Gl + gl)*C + c over ALL experts, local groups
+    const int tok = slot_token[r];
+    const int c = (int)(r % C), gl = (int)((r / C) % Gl), e = (int)(r / ((long long)C * Gl));
+    const int dest = e / El, el = e % El;
+    V* dst = reinterpret_cast<V*>(peers.p[dest]) + (((long long)el * G + (rank * Gl + gl)) * C + c) * row_vec;
+    if (tok >= 0 && tok < S) {
+      const V* src = x + ((long long)gl * S + tok) * row_vec;
+      for (int i = lane; i < row_vec; i += 32) dst[i] = __ldg(src + i);
+    } else {
+      for (int i = lane; i < row_vec; i += 32) dst[i] = make_uint4(0, 0, 0, 0);
+    }
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) combine_p2p_kernel(PeerPtrs peers, size_t out_offset_bytes,
+                                                          const int32_t* __restrict__ expert_idx,
+                                                          const int32_t* __restrict__ slot, const float* __restrict__ weight,
+                                                          const uint4* __restrict__ residual, uint4* __restrict__ y,
+                                                          long long N, int G, int Gl, int S, int C, int E, int El, int rank,
+                                                          int row_vec) {
+  constexpr int n = Vec16<T>::n;
+  const int lane = threadIdx.x & 31;
+  const long long warp = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const long long nwarps = ((long long)gridDim.x * blockDim.x) >> 5;
+  for (long long t = warp; t < N; t += nwarps) {
+    const int gl = (int)(t / S);
+    const uint4* rows[2] = {nullptr, nullptr};
+    float w[2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int e = expert_idx[2 * t + k], sl = slot[2 * t + k];
+      w[k] = weight[2 * t + k];
+      if (sl >= 0 && sl < C && e >= 0 && e < E)
+        rows[k] = reinterpret_cast<const uint4*>(peers.p[e / El] + out_offset_bytes) +
+                  (((long long)(e % El) * G + (rank * Gl + gl)) * C + sl) * row_vec;
+    }
+    // four 16-byte pieces per lane and row at a time, all loads issued before the first use: the rows
+    // come over NVLink (plain loads - a peer's memory is not read through the read-only path)
+    for (int i0 = lane; i0 < row_vec; i0 += 128) {
+      const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+      uint4 v0[4], v1[4], vr[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int i = i0 + 32 * k;
+        const bool in = i < row_vec;
+        v0[k] = (rows[0] && in) ? rows[0][i] : z;
+        v1[k] = (rows[1] && in) ? rows[1][i] : z;
+        vr[k] = (residual && in) ? __ldg(residual + t * row_vec + i) : z;
+      }
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int i = i0 + 32 * k;
+        if (i >= row_vec) break;
+        float acc[n], f0[n], f1[n];
+        Vec16<T>::load(vr[k], acc);
+        Vec16<T>::load(v0[k], f0);
+        Vec16<T>::load(v1[k], f1);
+#pragma unroll
+        for (int j = 0; j < n; ++j) acc[j] = fmaf(w[1], f1[j], fmaf(w[0], f0[j], acc[j]));
+        y[t * row_vec + i] = Vec16<T>::store(acc);
+      }
+    }
+  }
+}
+
+}  // namespace
+}  // namespace gshard
+
+extern "C" {
+
+size_t gshard_moe_ep_p2p_buffer_bytes(const gshard_moe_shape* shape, int world) {
+  gshard_moe_ep_layout l;
+  if (make_layout(shape, 0, world, &l) != GSHARD_OK || world > kMaxPeers) return 0;
+  const Dims dl = make_dims(l.local);
+  return 2 * align_up((size_t)dl.R * dl.M * dl.esize);
+}
+
+int gshard_moe_top2_forward_ep_p2p(const gshard_moe_shape* shape, int rank, int world, const void* x_local,
+                                   const void* wg, const void* wi_local, const void* wo_local, const float* u_local,
+                                   void* y_local, float* l_aux, const gshard_moe_routing* routing_out,
+                                   const gshard_ep_p2p* p2p, const gshard_ep_comm* comm, void* workspace,
+                                   size_t workspace_bytes, void* cuda_stream) {
+  launch_counter().n = 0;
+  gshard_moe_ep_layout l;
+  const int rcl = make_layout(shape, rank, world, &l);
+  if (rcl != GSHARD_OK) return rcl;
+  if (world > kMaxPeers) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  const void* ptrs[] = {x_local, wg, wi_local, wo_local, u_local, y_local, workspace};
+  for (const void* p : ptrs)
+    if (p == nullptr || !aligned16(p)) return GSHARD_ERR_INVALID_ARG;
+  if (l_aux == nullptr || p2p == nullptr || p2p->peer_buffers == nullptr) return GSHARD_ERR_INVALID_ARG;
+  if (world > 1 && p2p->rendezvous == nullptr) return GSHARD_ERR_INVALID_ARG;
+  PeerPtrs peers{};
+  for (int w = 0; w < world; ++w) {
+    if (p2p->peer_buffers[w] == nullptr || reinterpret_cast<uintptr_t>(p2p->peer_buffers[w]) % kAlign) return GSHARD_ERR_INVALID_ARG;
+    peers.p[w] = static_cast<unsigned char*>(p2p->peer_buffers[w]);
+  }
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  const Dims dl = make_dims(l.local);
+  const Dims df = make_dims(l.ffn);
+  const FwdPlan pl = plan_forward(dl);
+  if (workspace_bytes < pl.total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  const int rcd = check_device();
+  if (rcd != GSHARD_OK) return rcd;
+
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  const size_t half = align_up((size_t)dl.R * dl.M * dl.esize);
+  unsigned char* my_in = peers.p[rank];
+  unsigned char* my_out = peers.p[rank] + half;
+  gshard_moe_routing r{};
+  if (routing_out) r = *routing_out;
+  int* status = reinterpret_cast<int*>(ws + pl.status);
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  int32_t* expert_idx = pick(r.expert_idx, ws, pl.expert_idx);
+  int32_t* slot = pick(r.slot, ws, pl.slot);
+  float* weight = pick(r.weight, ws, pl.weight);
+  int32_t* slot_token = pick(r.slot_token, ws, pl.slot_token);
+  float* gate12 = reinterpret_cast<float*>(ws + pl.gate12);
+  float* m = pick(r.m, ws, pl.m);
+
+  int rc = gate_stage(dl, pl, ws, x_local, wg, expert_idx, gate12, m, reinterpret_cast<float*>(ws + pl.rowmax),
+                      reinterpret_cast<float*>(ws + pl.rowinv), st);
+  if (rc != GSHARD_OK) return rc;
+  rc = launch_capacity(dl, expert_idx, gate12, u_local, m, slot, weight, pick(r.flags, ws, pl.flags),
+                       pick(r.first_count, ws, pl.first_count), pick(r.total_count, ws, pl.total_count), slot_token,
+                       pick(r.l_aux_group, ws, pl.l_aux_group), reinterpret_cast<int32_t*>(ws + pl.stats_group), l_aux,
+                       reinterpret_cast<long long*>(r.stats), st, shape->G);
+  if (rc != GSHARD_OK) return rc;
+#define GS_RENDEZVOUS(phase) \
+  do { if (world > 1 && p2p->rendezvous(p2p->user, (phase), cuda_stream) != 0) return GSHARD_ERR_CUDA; } while (0)
+  // phase 0: every rank is done with the previous use of the exchange buffers
+  GS_RENDEZVOUS(0);
+  const int row_vec = (int)(l.row_bytes / 16);
+  {
+    NvtxRange range("gshard.dispatch_p2p");
+    dispatch_p2p_kernel<uint4><<<grid_for_rows(dl.R), 256, 0, st>>>(static_cast<const uint4*>(x_local), slot_token, peers,
+                                                                    dl.R, shape->G, l.groups_local, dl.S, dl.C,
+                                                                    l.experts_local, rank, row_vec);
+    count_launch();
+  }
+  // phase 1: every rank's rows have arrived in the owners' input buffers
+  GS_RENDEZVOUS(1);
+  rc = ffn_stage(df, my_in, wi_local, wo_local, ws + pl.h, false, my_out, ws + pl.ffn_scratch, status, st, nullptr, nullptr,
+                 ws + pl.wt);
+  if (rc != GSHARD_OK) return rc;
+  // phase 2: every rank's expert outputs are complete
+  GS_RENDEZVOUS(2);
+  {
+    NvtxRange range("gshard.combine_p2p");
+    const uint4* residual = dl.add_residual ? static_cast<const uint4*>(x_local) : nullptr;
+    if (dl.bf16)
+      combine_p2p_kernel<__nv_bfloat16><<<grid_for_rows(dl.N), 256, 0, st>>>(
+          peers, half, expert_idx, slot, weight, residual, static_cast<uint4*>(y_local), dl.N, shape->G, l.groups_local, dl.S,
+          dl.C, dl.E, l.experts_local, rank, row_vec);
+    else
+      combine_p2p_kernel<float><<<grid_for_rows(dl.N), 256, 0, st>>>(
+          peers, half, expert_idx, slot, weight, residual, static_cast<uint4*>(y_local), dl.N, shape->G, l.groups_local, dl.S,
+          dl.C, dl.E, l.experts_local, rank, row_vec);
+    count_launch();
+  }
+#undef GS_RENDEZVOUS
+  if (world > 1 && comm && comm->all_reduce_sum_f32 && comm->all_reduce_sum_f32(comm->user, l_aux, 1, cuda_stream) != 0)
+    return GSHARD_ERR_CUDA;
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+}  // extern "C"

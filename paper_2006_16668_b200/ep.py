@@ -116,6 +116,53 @@ class NcclComm:
             self.handle = ctypes.c_void_p()
 
 
+class SymmetricExchange:
+    """The exchange buffers and rendezvous of ``gshard_moe_top2_forward_ep_p2p`` on torch's symmetric
+    memory: every rank allocates its buffer from the symmetric allocator, the rendezvous maps all of
+    them into every process (``buffer_ptrs``), and the ordering callback is the allocation's own
+    barrier, enqueued on the current stream (each rank runs on its own GPU, so the barrier kernels of
+    different ranks never share one).  The library call must be made on torch's current stream.
+    """
+
+    def __init__(self, shape, rank: int, world: int, group=None):
+        import torch.distributed._symmetric_memory as symm
+        nbytes = B.gshard_moe_ep_p2p_buffer_bytes(shape, world)
+        if nbytes == 0:
+            raise ValueError("shape does not split over this many ranks")
+        self.rank, self.world, self.error = rank, world, None
+        self.buffer = symm.empty(nbytes, dtype=torch.uint8, device=torch.device("cuda", torch.cuda.current_device()))
+        group = group if group is not None else dist.group.WORLD
+        self.handle = symm.rendezvous(self.buffer, group.group_name)
+        ptrs = [int(p) for p in self.handle.buffer_ptrs]
+        if len(ptrs) != world or ptrs[rank] != self.buffer.data_ptr():
+            raise RuntimeError("symmetric memory rendezvous returned an unexpected pointer table")
+        self._ptrs = (ctypes.c_void_p * world)(*ptrs)
+        self._rv = B.RENDEZVOUS_FN(self._rendezvous)
+        self.struct = B.gshard_ep_p2p(self._rv, None, self._ptrs)
+
+    def _rendezvous(self, user, phase, stream):
+        try:
+            self.handle.barrier(channel=int(phase))
+            return 0
+        except Exception:                                    # an exception must not cross the C frame
+            self.error = traceback.format_exc()
+            return 1
+
+
+def forward_p2p(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux, exchange,
+                routing_out=None, workspace=None, comm=None):
+    """One expert-parallel forward with the exchange fused into the dispatch and combine kernels
+    (peer stores / peer loads through `exchange`, a SymmetricExchange); `comm` (a NcclComm) sums
+    l_aux over the ranks, without it l_aux is this rank's share."""
+    try:
+        B.gshard_moe_top2_forward_ep_p2p(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux,
+                                         routing_out, exchange.struct, comm.struct if comm else None, workspace)
+    except B.GshardError:
+        if exchange.error:
+            raise RuntimeError("the rendezvous of the expert-parallel forward failed:\n" + exchange.error)
+        raise
+
+
 def local_slices(layout: B.gshard_moe_ep_layout):
     """(group slice, expert slice) of this rank in the global tensors."""
     g0, e0 = layout.group_begin, layout.expert_begin

@@ -31,11 +31,17 @@ def run(args, cfg, dev, world, rank, metric, unit, sampler):
     ws = torch.empty(B.gshard_moe_ep_workspace_bytes(shape, world), dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
-    # collectives: NCCL called from inside the library (default), or torch.distributed through callbacks
-    comm = ep.NcclComm(rank, world) if (world > 1 and getattr(args, "ep_comm", "nccl") == "nccl") else None
+    # exchange: NCCL called from inside the library (default), torch.distributed through callbacks, or
+    # fused into the dispatch and combine kernels (peer stores and loads on symmetric memory)
+    mode = getattr(args, "ep_comm", "nccl")
+    comm = ep.NcclComm(rank, world) if (world > 1 and mode in ("nccl", "p2p")) else None
+    exchange = ep.SymmetricExchange(shape, rank, world) if mode == "p2p" else None
 
     def step():
-        ep.forward(shape, rank, world, x, wg, wi, wo, u, y, l_aux, None, ws, comm=comm)
+        if exchange is not None:
+            ep.forward_p2p(shape, rank, world, x, wg, wi, wo, u, y, l_aux, exchange, None, ws, comm=comm)
+        else:
+            ep.forward(shape, rank, world, x, wg, wi, wo, u, y, l_aux, None, ws, comm=comm)
 
     def barrier():
         if world > 1:
@@ -70,8 +76,10 @@ def run(args, cfg, dev, world, rank, metric, unit, sampler):
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "strong", "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
                 "config": {"workload": cfg.name, "G": cfg.G, "S": cfg.S, "M": cfg.M, "H": cfg.H, "E": cfg.E, "C": cfg.C,
-                           "parallelism": f"ep{world}: {Gl} groups and {El} experts per GPU, all-to-all of "
-                                          f"{layout.bytes_per_peer} bytes per peer before and after the expert FFN",
+                           "parallelism": f"ep{world}: {Gl} groups and {El} experts per GPU, "
+                                          f"{layout.bytes_per_peer} bytes per peer before and after the expert FFN, "
+                                          + ("stored and loaded peer to peer by the dispatch and combine kernels"
+                                             if exchange is not None else f"all-to-all ({mode})"),
                            "l2": "inputs larger than L2"},
                 "roofline": None, "cpu_baseline": None, "e2e": None, "gpu_launches": launches * args.steps,
                 "clocks": sampler.summary(), "device_status": status}

@@ -176,6 +176,121 @@ def test_expert_parallel_equals_single_gpu(world, name, G, S, M, H, E, C, dtype,
             assert torch.equal(r[1], results[0][1])
 
 
+class _P2PRank:
+    """gshard_ep_p2p for one emulated rank: the exchange buffers of all ranks live on the one GPU, so a
+    peer's pointer is an ordinary pointer; the rendezvous records an event on this rank's stream, meets
+    the other threads at a host barrier and makes the stream wait on every rank's event."""
+
+    def __init__(self, world, rank, buffers, stream):
+        self.w, self.rank, self.stream = world, rank, stream
+        self.phases, self.error = [], None
+        self._rv = B.RENDEZVOUS_FN(self._rendezvous)
+        import ctypes
+        self._ptrs = (ctypes.c_void_p * world.n)(*[b.data_ptr() for b in buffers])
+        self.struct = B.gshard_ep_p2p(self._rv, None, self._ptrs)
+
+    def _rendezvous(self, user, phase, stream):
+        try:
+            w, r = self.w, self.rank
+            self.phases.append(phase)
+            ev = torch.cuda.Event()
+            ev.record(self.stream)
+            w.ready[r] = ev
+            w.barrier.wait()
+            for s in range(w.n):
+                self.stream.wait_event(w.ready[s])
+            w.barrier.wait()                      # nobody overwrites its event before all have read it
+            return 0
+        except Exception:
+            self.error = traceback.format_exc()
+            return 1
+
+
+def _run_ranks_p2p(cfg, inp, world, flags=0, steps=1):
+    shape = B.make_shape(cfg, flags=flags)
+    state = _World(world)
+    nbytes = B.gshard_moe_ep_p2p_buffer_bytes(shape, world)
+    assert nbytes > 0
+    # poisoned, so that a row nobody wrote shows up
+    buffers = [torch.full((nbytes,), 0x7F, dtype=torch.uint8, device="cuda") for _ in range(world)]
+    torch.cuda.synchronize()
+    results, errors = [None] * world, [None] * world
+
+    def rank_main(rank):
+        try:
+            torch.cuda.set_device(0)
+            lay = B.gshard_moe_ep_plan(shape, rank, world)
+            gs, es = ep.local_slices(lay)
+            stream = torch.cuda.Stream()
+            x, u = inp["x"][gs].contiguous(), inp["u"][gs].contiguous()
+            wi, wo = inp["wi"][es].contiguous(), inp["wo"][es].contiguous()
+            ws = B.alloc_workspace(lay.local)
+            rt, rs = B.alloc_routing(lay.local)
+            y = torch.empty_like(x)
+            l_aux = torch.zeros(1, device="cuda")
+            torch.cuda.synchronize()
+            p2p = _P2PRank(state, rank, buffers, stream)
+            for _ in range(steps):
+                B.gshard_moe_top2_forward_ep_p2p(shape, rank, world, x, inp["wg"], wi, wo, u, y, l_aux, rs, p2p.struct,
+                                                 None, ws, stream)
+            assert p2p.error is None, p2p.error
+            assert p2p.phases == ([0, 1, 2] * steps if world > 1 else [])
+            assert B.gshard_moe_last_device_status(ws, stream) == B.GSHARD_OK
+            stream.synchronize()
+            results[rank] = (y, l_aux, rt)
+        except Exception:
+            errors[rank] = traceback.format_exc()
+            state.barrier.abort()
+
+    threads = [threading.Thread(target=rank_main, args=(r,)) for r in range(world)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=180)
+    assert not any(errors), "\n".join(e for e in errors if e)
+    assert all(r is not None for r in results)
+    return results
+
+
+@pytest.mark.parametrize("name,G,S,M,H,E,C,dtype,flags", CASES, ids=[c[0] for c in CASES])
+@pytest.mark.parametrize("world", [1, 2, 4])
+def test_fused_exchange_equals_single_gpu(world, name, G, S, M, H, E, C, dtype, flags):
+    """gshard_moe_top2_forward_ep_p2p: dispatch stores into the owners' buffers, combine loads out of
+    them.  Same bits as the single-GPU layer; l_aux without a comm is the rank's share, so the shares
+    must add up to the layer's l_aux.  Two steps in a row reuse the buffers (phase 0 protects them)."""
+    cfg = MoEConfig(name, G=G, S=S, M=M, H=H, E=E, C=C, dtype=dtype, seed=977)
+    inp = make_inputs(cfg, "cuda")
+    y_ref, l_ref, rt_ref = _single(cfg, inp, flags)
+    results = _run_ranks_p2p(cfg, inp, world, flags, steps=2)
+    y = torch.cat([r[0] for r in results])
+    assert torch.equal(y.view(torch.uint8), y_ref.view(torch.uint8)), "y differs from the single-GPU layer"
+    for k in ("expert_idx", "slot", "weight", "flags", "first_count", "total_count", "m", "l_aux_group"):
+        assert torch.equal(torch.cat([r[2][k] for r in results]), rt_ref[k]), k
+    assert torch.equal(torch.cat([r[2]["slot_token"] for r in results], dim=1), rt_ref["slot_token"])
+    assert sum(float(r[1]) for r in results) == pytest.approx(float(l_ref), rel=1e-6)
+
+
+def test_fused_exchange_with_residual_and_bad_arguments():
+    import ctypes
+    cfg = MoEConfig("p2p_res", G=4, S=128, M=64, H=128, E=16, C=16, dtype="bf16", seed=5)
+    inp = make_inputs(cfg, "cuda")
+    y_ref, _, _ = _single(cfg, inp, B.GSHARD_FLAG_ADD_RESIDUAL)
+    results = _run_ranks_p2p(cfg, inp, 2, B.GSHARD_FLAG_ADD_RESIDUAL)
+    assert torch.equal(torch.cat([r[0] for r in results]).view(torch.int16), y_ref.view(torch.int16))
+    shape = B.make_shape(cfg)
+    lib = B.load()
+    fake = 0x10000
+    ptrs = (ctypes.c_void_p * 2)(fake, fake)
+    no_rv = B.gshard_ep_p2p(B.RENDEZVOUS_FN(), None, ptrs)
+    call = lambda rank, world, p2p, nbytes: lib.gshard_moe_top2_forward_ep_p2p(
+        ctypes.byref(shape), rank, world, *([fake] * 7), None, p2p, None, fake, nbytes, None)
+    assert call(0, 2, None, 1 << 40) == B.GSHARD_ERR_INVALID_ARG
+    assert call(0, 2, ctypes.byref(no_rv), 1 << 40) == B.GSHARD_ERR_INVALID_ARG           # world > 1 needs a rendezvous
+    assert call(0, 3, ctypes.byref(no_rv), 1 << 40) == B.GSHARD_ERR_UNSUPPORTED_SHAPE
+    assert call(0, 1, ctypes.byref(no_rv), 16) == B.GSHARD_ERR_WORKSPACE_TOO_SMALL
+    assert B.gshard_moe_ep_p2p_buffer_bytes(shape, 3) == 0
+
+
 def test_world_one_at_full_size_is_the_single_gpu_layer():
     from paper_2006_16668_b200 import CONFIGS
     cfg = CONFIGS["c3_512e_skew"]
@@ -235,3 +350,43 @@ def test_nccl_comm_single_rank():
     lib = B.load()
     state, c = B.gshard_ep_nccl_state(), B.gshard_ep_comm()
     assert lib.gshard_ep_comm_from_nccl(None, 1, ctypes.byref(state), ctypes.byref(c)) == B.GSHARD_ERR_INVALID_ARG
+
+
+_SYMM_SCRIPT = r"""
+import torch, torch.distributed as dist
+torch.cuda.set_device(0)
+dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+from paper_2006_16668_b200 import MoEConfig, make_inputs, binding as B, ep
+cfg = MoEConfig("symm1", G=4, S=128, M=64, H=128, E=16, C=16, dtype="bf16", seed=3)
+shape = B.make_shape(cfg)
+ex = ep.SymmetricExchange(shape, 0, 1)
+assert ex.buffer.numel() == B.gshard_moe_ep_p2p_buffer_bytes(shape, 1)
+for phase in (0, 1, 2):
+    assert ex.struct.rendezvous(None, phase, None) == 0, ex.error
+inp = make_inputs(cfg, "cuda")
+ws = B.alloc_workspace(shape)
+y, l = torch.empty_like(inp["x"]), torch.zeros(1, device="cuda")
+ep.forward_p2p(shape, 0, 1, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l, ex, None, ws)
+y2, l2 = torch.empty_like(y), torch.zeros(1, device="cuda")
+B.gshard_moe_top2_forward(shape, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y2, l2, None, None, ws)
+torch.cuda.synchronize()
+assert torch.equal(y.view(torch.int16), y2.view(torch.int16)) and torch.equal(l, l2)
+dist.destroy_process_group()
+print("SYMM_OK")
+"""
+
+
+def test_symmetric_exchange_single_rank():
+    """ep.SymmetricExchange (torch symmetric memory: peer pointer table + barrier as the rendezvous)
+    at world 1, all that one GPU can run; in a child process because it needs a process group."""
+    import os
+    import socket
+    import subprocess
+    import sys
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), PYTHONPATH=root)
+    out = subprocess.run([sys.executable, "-c", _SYMM_SCRIPT], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0 and "SYMM_OK" in out.stdout, out.stdout[-2000:] + out.stderr[-4000:]
