@@ -328,8 +328,9 @@ typedef struct {
  * cuda_stream (or order themselves after and before it) and return 0 on success.
  *   all_to_all: equal splits; bytes [i*bytes_per_peer, (i+1)*bytes_per_peer) of send go to rank i,
  *     the same range of recv receives from rank i.  send and recv are device buffers inside the
- *     workspace of the call and never alias.
- *   all_reduce_sum_f32: in-place sum over the ranks of `count` floats in device memory. */
+ *     workspace (or, with SAVE_FOR_BACKWARD, the context) of the call and never alias.
+ *   all_reduce_sum_f32: in-place sum over the ranks of `count` floats in device memory (the l_aux
+ *     scalar in the forward, dwg in the backward). */
 typedef struct {
   int (*all_to_all)(void* user, const void* send, void* recv, size_t bytes_per_peer, void* cuda_stream);
   int (*all_reduce_sum_f32)(void* user, float* buf, size_t count, void* cuda_stream);
@@ -346,7 +347,7 @@ typedef struct { void* opaque[8]; } gshard_ep_nccl_state;
 int gshard_ep_comm_from_nccl(void* nccl_comm, int world, gshard_ep_nccl_state* state, gshard_ep_comm* comm);
 
 /* Host-only: validates the partitioning and fills `layout`.  GSHARD_ERR_UNSUPPORTED_SHAPE when G or
- * E is not a multiple of world (or SAVE_FOR_BACKWARD is set: the expert-parallel form is forward only). */
+ * E is not a multiple of world. */
 int gshard_moe_ep_plan(const gshard_moe_shape* shape, int rank, int world, gshard_moe_ep_layout* layout);
 
 /* Host-only: the permutation between the layout an AllToAll delivers, [world (source rank)]
@@ -358,7 +359,9 @@ int gshard_moe_ep_plan(const gshard_moe_shape* shape, int rank, int world, gshar
 int gshard_moe_ep_regroup_host(const gshard_moe_ep_layout* layout, const void* src, void* dst, size_t row_bytes,
                                int inverse);
 
-size_t gshard_moe_ep_workspace_bytes(const gshard_moe_shape* shape, int world);
+size_t gshard_moe_ep_workspace_bytes(const gshard_moe_shape* shape, int world);          /* forward */
+size_t gshard_moe_ep_context_bytes(const gshard_moe_shape* shape, int world);
+size_t gshard_moe_ep_backward_workspace_bytes(const gshard_moe_shape* shape, int world);
 
 /* Forward of the layer on rank `rank` of `world` (shape is the GLOBAL shape).
  *   x_local, y_local [G/world, S, M], u_local [G/world, S]: this rank's groups; wg [M, E] replicated;
@@ -366,13 +369,32 @@ size_t gshard_moe_ep_workspace_bytes(const gshard_moe_shape* shape, int world);
  *   l_aux: the layer's loss (mean over ALL groups), identical on every rank after the call.
  *   routing_out: optional outputs for the LOCAL groups (shapes as in gshard_moe_routing with
  *   G = G/world; stats are this rank's).  comm: the collectives; may be NULL when world == 1.
+ *   context: with GSHARD_FLAG_SAVE_FOR_BACKWARD, gshard_moe_ep_context_bytes(shape, world) bytes
+ *   that receive what gshard_moe_top2_backward_ep needs (routing and softmax statistics of the local
+ *   groups; inputs, hidden activations and ReLU mask of the local experts); else NULL.
  * With world == 1 the call runs exactly the kernels of gshard_moe_top2_forward and gives the same
- * bits.  Every received slab lies in this GPU's own workspace before a kernel reads it. */
+ * bits.  Every received slab lies in this GPU's own memory before a kernel reads it. */
 int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int world, const void* x_local,
                                const void* wg, const void* wi_local, const void* wo_local,
                                const float* u_local, void* y_local, float* l_aux,
-                               const gshard_moe_routing* routing_out, const gshard_ep_comm* comm,
-                               void* workspace, size_t workspace_bytes, void* cuda_stream);
+                               const gshard_moe_routing* routing_out, void* context,
+                               const gshard_ep_comm* comm, void* workspace, size_t workspace_bytes,
+                               void* cuda_stream);
+
+/* Backward of the expert-parallel layer (same loss and conventions as gshard_moe_top2_backward): the
+ * gradients of the expert outputs go to the experts' owners through an AllToAll, the expert FFN
+ * backward runs over the local experts, the gradients of the expert inputs come back through a second
+ * AllToAll, and the gating backward runs over the local groups.
+ *   dy_local, dx_local [G/world, S, M]; dwi_local [E/world, M, H], dwo_local [E/world, H, M]: this
+ *   rank's share; dwg [M, E] float: wg is replicated, so every rank ends with the SUM over the ranks
+ *   (all_reduce_sum_f32).  context: filled by gshard_moe_top2_forward_ep on this rank.
+ *   workspace: gshard_moe_ep_backward_workspace_bytes(shape, world). */
+int gshard_moe_top2_backward_ep(const gshard_moe_shape* shape, int rank, int world, const void* x_local,
+                                const void* wg, const void* wi_local, const void* wo_local,
+                                const void* context, const void* dy_local, float l_aux_weight,
+                                void* dx_local, float* dwg, void* dwi_local, void* dwo_local,
+                                const gshard_ep_comm* comm, void* workspace, size_t workspace_bytes,
+                                void* cuda_stream);
 
 /* The expert-parallel forward with the exchange FUSED into the dispatch and combine kernels (same
  * partitioning and results as gshard_moe_top2_forward_ep).  The dispatch kernel stores each token row
@@ -391,7 +413,7 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
  *   complete); returns 0 on success.  No kernel of this library waits for another rank's kernel.
  *   comm: optional, only its all_reduce_sum_f32 is used (for l_aux; without it l_aux holds this rank's
  *   share, sum of its group losses / G).  workspace: gshard_moe_top2_workspace_bytes of the LOCAL shape
- *   (layout.local) suffices. */
+ *   (layout.local) suffices.  Forward only: SAVE_FOR_BACKWARD shapes are refused. */
 typedef struct {
   int (*rendezvous)(void* user, int phase, void* cuda_stream);
   void* user;

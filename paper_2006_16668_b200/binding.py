@@ -111,9 +111,13 @@ EXPORTS = {
     "gshard_ep_comm_from_nccl": (c_int, [c_void_p, c_int, POINTER(gshard_ep_nccl_state), POINTER(gshard_ep_comm)]),
     "gshard_moe_ep_regroup_host": (c_int, [POINTER(gshard_moe_ep_layout), c_void_p, c_void_p, c_size_t, c_int]),
     "gshard_moe_ep_workspace_bytes": (c_size_t, [POINTER(gshard_moe_shape), c_int]),
+    "gshard_moe_ep_context_bytes": (c_size_t, [POINTER(gshard_moe_shape), c_int]),
+    "gshard_moe_ep_backward_workspace_bytes": (c_size_t, [POINTER(gshard_moe_shape), c_int]),
     "gshard_moe_top2_forward_ep": (c_int, [POINTER(gshard_moe_shape), c_int, c_int] + [c_void_p] * 7 +
-                                   [POINTER(gshard_moe_routing), POINTER(gshard_ep_comm), c_void_p, c_size_t,
+                                   [POINTER(gshard_moe_routing), c_void_p, POINTER(gshard_ep_comm), c_void_p, c_size_t,
                                     c_void_p]),
+    "gshard_moe_top2_backward_ep": (c_int, [POINTER(gshard_moe_shape), c_int, c_int] + [c_void_p] * 6 + [c_float] +
+                                    [c_void_p] * 4 + [POINTER(gshard_ep_comm), c_void_p, c_size_t, c_void_p]),
     "gshard_dense_ffn_workspace_bytes": (c_size_t, [ctypes.c_int64, c_int32, c_int32, c_int32]),
     "gshard_dense_ffn_forward": (c_int, [ctypes.c_int64, c_int32, c_int32, c_int32, c_uint32] + [c_void_p] * 5 +
                                  [c_size_t, c_void_p]),
@@ -347,14 +351,32 @@ def gshard_moe_ep_workspace_bytes(shape, world) -> int:
     return int(load().gshard_moe_ep_workspace_bytes(ctypes.byref(shape), int(world)))
 
 
+def gshard_moe_ep_context_bytes(shape, world) -> int:
+    return int(load().gshard_moe_ep_context_bytes(ctypes.byref(shape), int(world)))
+
+
+def gshard_moe_ep_backward_workspace_bytes(shape, world) -> int:
+    return int(load().gshard_moe_ep_backward_workspace_bytes(ctypes.byref(shape), int(world)))
+
+
 def gshard_moe_top2_forward_ep(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux,
-                               routing_out=None, comm=None, workspace=None, stream=None):
+                               routing_out=None, comm=None, workspace=None, stream=None, context=None):
     rp = ctypes.byref(routing_out) if routing_out is not None else None
     cp = ctypes.byref(comm) if comm is not None else None
     _check(load().gshard_moe_top2_forward_ep(ctypes.byref(shape), int(rank), int(world), _p(x_local), _p(wg),
-                                             _p(wi_local), _p(wo_local), _p(u_local), _p(y_local), _p(l_aux), rp, cp,
-                                             _p(workspace), workspace.numel(), _stream(stream)),
+                                             _p(wi_local), _p(wo_local), _p(u_local), _p(y_local), _p(l_aux), rp,
+                                             _p(context), cp, _p(workspace), workspace.numel(), _stream(stream)),
            "gshard_moe_top2_forward_ep")
+
+
+def gshard_moe_top2_backward_ep(shape, rank, world, x_local, wg, wi_local, wo_local, context, dy_local, l_aux_weight,
+                                dx_local, dwg, dwi_local, dwo_local, comm=None, workspace=None, stream=None):
+    cp = ctypes.byref(comm) if comm is not None else None
+    _check(load().gshard_moe_top2_backward_ep(ctypes.byref(shape), int(rank), int(world), _p(x_local), _p(wg),
+                                              _p(wi_local), _p(wo_local), _p(context), _p(dy_local),
+                                              float(l_aux_weight), _p(dx_local), _p(dwg), _p(dwi_local), _p(dwo_local),
+                                              cp, _p(workspace), workspace.numel(), _stream(stream)),
+           "gshard_moe_top2_backward_ep")
 
 
 def _dtype_code(t) -> int:

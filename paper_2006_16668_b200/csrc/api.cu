@@ -250,7 +250,7 @@ using namespace gshard;
 
 extern "C" {
 
-int gshard_version(void) { return 200; }
+int gshard_version(void) { return 210; }
 
 const char* gshard_status_string(int s) {
   switch (s) {

@@ -237,84 +237,50 @@ int run_gemm_pair(const Dims& d, UmmaGemm a, UmmaGemm b, int share_a, int* statu
   return GSHARD_OK;
 }
 
+// Combine backward over the groups of `d`: dw (per token and choice) and dout (per slot) into the
+// backward workspace laid out by plan_backward(d).
 template <typename T>
-int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, const void* wo, const unsigned char* ctx,
-               const void* dy, float k_aux, void* dx, float* dwg, void* dwi, void* dwo, unsigned char* ws,
-               cudaStream_t st) {
-  NvtxRange range("gshard.backward");
+int combine_bwd_t(const Dims& d, const unsigned char* ctx, const void* dy, unsigned char* ws, cudaStream_t st) {
+  NvtxRange range("gshard.backward.combine");
+  const BwdPlan bp = plan_backward(d);
+  const CtxPlan cp = plan_context(d);
+  const int32_t* expert_idx = reinterpret_cast<const int32_t*>(ctx + cp.expert_idx);
+  const int32_t* slot = reinterpret_cast<const int32_t*>(ctx + cp.slot);
+  const int row_vec = (int)((size_t)d.M * d.esize / 16);
+  combine_bwd_kernel<T><<<grid_for_rows(d.N), 256, 0, st>>>(
+      reinterpret_cast<const uint4*>(dy), reinterpret_cast<const uint4*>(ctx + cp.out), expert_idx, slot,
+      reinterpret_cast<float*>(ws + bp.dw), d.N, d.G, d.S, d.C, row_vec);
+  dout_kernel<T><<<grid_for_rows(d.R), 256, 0, st>>>(
+      reinterpret_cast<const uint4*>(dy), reinterpret_cast<const int32_t*>(ctx + cp.slot_token), expert_idx, slot,
+      reinterpret_cast<const float*>(ctx + cp.weight), reinterpret_cast<uint4*>(ws + bp.dout), d.R, d.G, d.S, d.C, row_vec);
+  count_launch(2);
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+// Gating backward and dx over the groups of `d`.  groups_in_mean: the group count l_aux averages
+// over (the global one when `d` is one rank's share of the groups).  dbuf: [E, G*C, M] of `d`.
+template <typename T>
+int gate_bwd_t(const Dims& d, const void* x, const void* wg, const unsigned char* ctx, const void* dy, float k_aux,
+               int groups_in_mean, const void* dbuf, void* dx, float* dwg, unsigned char* ws, cudaStream_t st) {
+  NvtxRange gate_range("gshard.backward.gate");
   const BwdPlan bp = plan_backward(d);
   const CtxPlan cp = plan_context(d);
   int* status = reinterpret_cast<int*>(ws + bp.status);
-  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
   const int32_t* expert_idx = reinterpret_cast<const int32_t*>(ctx + cp.expert_idx);
   const int32_t* slot = reinterpret_cast<const int32_t*>(ctx + cp.slot);
-  const float* weight = reinterpret_cast<const float*>(ctx + cp.weight);
   const int32_t* first_count = reinterpret_cast<const int32_t*>(ctx + cp.first_count);
-  const int32_t* slot_token = reinterpret_cast<const int32_t*>(ctx + cp.slot_token);
   const float* gate12 = reinterpret_cast<const float*>(ctx + cp.gate12);
   const float* rowmax = reinterpret_cast<const float*>(ctx + cp.rowmax);
   const float* rowinv = reinterpret_cast<const float*>(ctx + cp.rowinv);
-  const void* h = ctx + cp.h;
-  const uint32_t* hbits = d.simt ? nullptr : reinterpret_cast<const uint32_t*>(ctx + cp.hbits);
-  const void* out = ctx + cp.out;
   float* logits = reinterpret_cast<float*>(ws + bp.logits);
   T* dlogits = reinterpret_cast<T*>(ws + bp.dlogits);
-  float* dw = reinterpret_cast<float*>(ws + bp.dw);
-  const void* buf = ctx + cp.buf;              // dispatched inputs, as the forward wrote them
-  void* dout = ws + bp.dout;
-  void* dh = ws + bp.dh;
-  void* dbuf = ws + bp.dbuf;
+  const float* dw = reinterpret_cast<const float*>(ws + bp.dw);
   float* dxg = reinterpret_cast<float*>(ws + bp.dxg);
   const int row_vec = (int)((size_t)d.M * d.esize / 16);
-  const long long rows = d.rows;
-
-  // combine backward
-  nvtxRangePushA("gshard.backward.combine");
-  combine_bwd_kernel<T><<<grid_for_rows(d.N), 256, 0, st>>>(reinterpret_cast<const uint4*>(dy),
-                                                        reinterpret_cast<const uint4*>(out), expert_idx, slot, dw, d.N,
-                                                        d.G, d.S, d.C, row_vec);
-  dout_kernel<T><<<grid_for_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(dy), slot_token, expert_idx, slot,
-                                                 weight, reinterpret_cast<uint4*>(dout), d.R, d.G, d.S, d.C, row_vec);
-  count_launch(2);
-
-  nvtxRangePop();
-  nvtxRangePushA("gshard.backward.expert_ffn");
-  // expert FFN backward.  dh and dbuf stream the weights (read-heavy), dwo and dwi write a gradient the
-  // size of the weights from short contractions (write-heavy): one of each runs side by side.
-  UmmaGemm g_dh{}, g_dwo{}, g_dwi{}, g_dbuf{};
-  // dh = (dout . wo^T) masked by h > 0
-  g_dh.A = dout; g_dh.B = wo; g_dh.C = dh; g_dh.mask = h; g_dh.mask_bits = hbits; g_dh.rows = d.rows; g_dh.cols = d.H; g_dh.K = d.M; g_dh.batch = d.E;
-  g_dh.a_kmajor = true; g_dh.b_kmajor = true;
-  g_dh.a_ld = d.M; g_dh.a_bs = rows * d.M; g_dh.b_ld = d.M; g_dh.b_bs = (long long)d.H * d.M; g_dh.c_ld = d.H; g_dh.c_bs = rows * d.H;
-  g_dh.b_stream = 1; g_dh.prefer_two_sm = 1;
-  // dwo[e] = h[e]^T . dout[e]   [H x M]
-  g_dwo.A = h; g_dwo.B = dout; g_dwo.C = dwo; g_dwo.rows = d.H; g_dwo.cols = d.M; g_dwo.K = d.rows; g_dwo.batch = d.E;
-  g_dwo.a_kmajor = false; g_dwo.b_kmajor = false;
-  g_dwo.a_ld = d.H; g_dwo.a_bs = rows * d.H; g_dwo.b_ld = d.M; g_dwo.b_bs = rows * d.M; g_dwo.c_ld = d.M; g_dwo.c_bs = (long long)d.H * d.M;
-  // dwi[e] = buf[e]^T . dh[e]   [M x H]
-  g_dwi.A = buf; g_dwi.B = dh; g_dwi.C = dwi; g_dwi.rows = d.M; g_dwi.cols = d.H; g_dwi.K = d.rows; g_dwi.batch = d.E;
-  g_dwi.a_kmajor = false; g_dwi.b_kmajor = false;
-  g_dwi.a_ld = d.M; g_dwi.a_bs = rows * d.M; g_dwi.b_ld = d.H; g_dwi.b_bs = rows * d.H; g_dwi.c_ld = d.H; g_dwi.c_bs = (long long)d.M * d.H;
-  // dbuf = dh . wi^T   [rows x M]
-  g_dbuf.A = dh; g_dbuf.B = wi; g_dbuf.C = dbuf; g_dbuf.rows = d.rows; g_dbuf.cols = d.M; g_dbuf.K = d.H; g_dbuf.batch = d.E;
-  g_dbuf.a_kmajor = true; g_dbuf.b_kmajor = true;
-  g_dbuf.a_ld = d.H; g_dbuf.a_bs = rows * d.H; g_dbuf.b_ld = d.H; g_dbuf.b_bs = (long long)d.M * d.H; g_dbuf.c_ld = d.M; g_dbuf.c_bs = rows * d.M;
-  g_dbuf.b_stream = 1; g_dbuf.prefer_two_sm = 1;
-  // On request each read-heavy GEMM shares the GPU with a write-heavy one (half of the multiprocessors
-  // each, two streams).  Measured at the MoE(512E) training shape this is slower than running the four
-  // one after another on all multiprocessors, so it is not the default.
-  const int share = d.bwd_paired ? (device_sms() / 2) & ~1 : 0;
-  int rc = run_gemm_pair(d, g_dh, g_dwo, share, status, st);
+  // recompute the logits, softmax backward, two GEMMs
+  int rc = gate_logits(d, x, wg, logits, status, st);
   if (rc) return rc;
-  rc = run_gemm_pair(d, g_dbuf, g_dwi, share, status, st);
-  if (rc) return rc;
-
-  nvtxRangePop();
-  NvtxRange gate_range("gshard.backward.gate");
-  // gating backward: recompute the logits, softmax backward, two GEMMs
-  rc = gate_logits(d, x, wg, logits, status, st);
-  if (rc) return rc;
-  const float aux_coef = k_aux / ((float)d.G * (float)d.E * (float)d.S * (float)d.S);
+  const float aux_coef = k_aux / ((float)groups_in_mean * (float)d.E * (float)d.S * (float)d.S);
   gate_bwd_kernel<T><<<grid_for_rows(d.N), 256, 0, st>>>(logits, rowmax, rowinv, expert_idx, gate12, dw, first_count,
                                                      aux_coef, dlogits, d.N, d.S, d.E);
   count_launch();
@@ -363,15 +329,74 @@ int backward_t(const Dims& d, const void* x, const void* wg, const void* wi, con
 
 }  // namespace
 
+int backward_combine_stage(const Dims& d, const void* context, const void* dy, void* workspace, cudaStream_t st) {
+  const unsigned char* ctx = static_cast<const unsigned char*>(context);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  return d.bf16 ? combine_bwd_t<__nv_bfloat16>(d, ctx, dy, ws, st) : combine_bwd_t<float>(d, ctx, dy, ws, st);
+}
+
+// Expert FFN backward over the problems of `d` (E experts with d.rows rows each).  dh and dbuf stream
+// the weights (read-heavy), dwo and dwi write a gradient the size of the weights from short
+// contractions (write-heavy).
+int backward_expert_stage(const Dims& d, const void* dout, const void* h, const uint32_t* hbits, const void* buf,
+                          const void* wi, const void* wo, void* dh, void* dbuf, void* dwi, void* dwo, int* status,
+                          cudaStream_t st) {
+  NvtxRange range("gshard.backward.expert_ffn");
+  const long long rows = d.rows;
+  UmmaGemm g_dh{}, g_dwo{}, g_dwi{}, g_dbuf{};
+  // dh = (dout . wo^T) masked by h > 0
+  g_dh.A = dout; g_dh.B = wo; g_dh.C = dh; g_dh.mask = h; g_dh.mask_bits = hbits; g_dh.rows = d.rows; g_dh.cols = d.H; g_dh.K = d.M; g_dh.batch = d.E;
+  g_dh.a_kmajor = true; g_dh.b_kmajor = true;
+  g_dh.a_ld = d.M; g_dh.a_bs = rows * d.M; g_dh.b_ld = d.M; g_dh.b_bs = (long long)d.H * d.M; g_dh.c_ld = d.H; g_dh.c_bs = rows * d.H;
+  g_dh.b_stream = 1; g_dh.prefer_two_sm = 1;
+  // dwo[e] = h[e]^T . dout[e]   [H x M]
+  g_dwo.A = h; g_dwo.B = dout; g_dwo.C = dwo; g_dwo.rows = d.H; g_dwo.cols = d.M; g_dwo.K = d.rows; g_dwo.batch = d.E;
+  g_dwo.a_kmajor = false; g_dwo.b_kmajor = false;
+  g_dwo.a_ld = d.H; g_dwo.a_bs = rows * d.H; g_dwo.b_ld = d.M; g_dwo.b_bs = rows * d.M; g_dwo.c_ld = d.M; g_dwo.c_bs = (long long)d.H * d.M;
+  // dwi[e] = buf[e]^T . dh[e]   [M x H]
+  g_dwi.A = buf; g_dwi.B = dh; g_dwi.C = dwi; g_dwi.rows = d.M; g_dwi.cols = d.H; g_dwi.K = d.rows; g_dwi.batch = d.E;
+  g_dwi.a_kmajor = false; g_dwi.b_kmajor = false;
+  g_dwi.a_ld = d.M; g_dwi.a_bs = rows * d.M; g_dwi.b_ld = d.H; g_dwi.b_bs = rows * d.H; g_dwi.c_ld = d.H; g_dwi.c_bs = (long long)d.M * d.H;
+  // dbuf = dh . wi^T   [rows x M]
+  g_dbuf.A = dh; g_dbuf.B = wi; g_dbuf.C = dbuf; g_dbuf.rows = d.rows; g_dbuf.cols = d.M; g_dbuf.K = d.H; g_dbuf.batch = d.E;
+  g_dbuf.a_kmajor = true; g_dbuf.b_kmajor = true;
+  g_dbuf.a_ld = d.H; g_dbuf.a_bs = rows * d.H; g_dbuf.b_ld = d.H; g_dbuf.b_bs = (long long)d.M * d.H; g_dbuf.c_ld = d.M; g_dbuf.c_bs = rows * d.M;
+  g_dbuf.b_stream = 1; g_dbuf.prefer_two_sm = 1;
+  // On request each read-heavy GEMM shares the GPU with a write-heavy one (half of the multiprocessors
+  // each, two streams).  Measured at the MoE(512E) training shape this is slower than running the four
+  // one after another on all multiprocessors, so it is not the default.
+  const int share = d.bwd_paired ? (device_sms() / 2) & ~1 : 0;
+  int rc = run_gemm_pair(d, g_dh, g_dwo, share, status, st);
+  if (rc) return rc;
+  return run_gemm_pair(d, g_dbuf, g_dwi, share, status, st);
+}
+
+int backward_gate_stage(const Dims& d, const void* x, const void* wg, const void* context, const void* dy, float k_aux,
+                        int groups_in_mean, const void* dbuf, void* dx, float* dwg, void* workspace, cudaStream_t st) {
+  const unsigned char* ctx = static_cast<const unsigned char*>(context);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  return d.bf16 ? gate_bwd_t<__nv_bfloat16>(d, x, wg, ctx, dy, k_aux, groups_in_mean, dbuf, dx, dwg, ws, st)
+                : gate_bwd_t<float>(d, x, wg, ctx, dy, k_aux, groups_in_mean, dbuf, dx, dwg, ws, st);
+}
+
 int backward_device(const gshard_moe_shape* shape, const void* x, const void* wg, const void* wi, const void* wo,
                     const void* context, const void* dy, float k_aux, void* dx, float* dwg, void* dwi, void* dwo,
                     void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  NvtxRange range("gshard.backward");
   const Dims d = make_dims(*shape);
-  if (workspace_bytes < plan_backward(d).total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  const BwdPlan bp = plan_backward(d);
+  const CtxPlan cp = plan_context(d);
+  if (workspace_bytes < bp.total) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
   const unsigned char* ctx = static_cast<const unsigned char*>(context);
   unsigned char* ws = static_cast<unsigned char*>(workspace);
-  if (d.bf16) return backward_t<__nv_bfloat16>(d, x, wg, wi, wo, ctx, dy, k_aux, dx, dwg, dwi, dwo, ws, st);
-  return backward_t<float>(d, x, wg, wi, wo, ctx, dy, k_aux, dx, dwg, dwi, dwo, ws, st);
+  int* status = reinterpret_cast<int*>(ws + bp.status);
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  int rc = backward_combine_stage(d, ctx, dy, ws, st);
+  if (rc) return rc;
+  rc = backward_expert_stage(d, ws + bp.dout, ctx + cp.h, d.simt ? nullptr : reinterpret_cast<const uint32_t*>(ctx + cp.hbits),
+                             ctx + cp.buf, wi, wo, ws + bp.dh, ws + bp.dbuf, dwi, dwo, status, st);
+  if (rc) return rc;
+  return backward_gate_stage(d, x, wg, ctx, dy, k_aux, d.G, ws + bp.dbuf, dx, dwg, ws, st);
 }
 
 }  // namespace gshard

@@ -66,7 +66,6 @@ int make_layout(const gshard_moe_shape* shape, int rank, int world, gshard_moe_e
   if (rc != GSHARD_OK) return rc;
   if (world < 1 || rank < 0 || rank >= world) return GSHARD_ERR_INVALID_ARG;
   if (shape->G % world || shape->E % world) return GSHARD_ERR_UNSUPPORTED_SHAPE;
-  if (shape->flags & GSHARD_FLAG_SAVE_FOR_BACKWARD) return GSHARD_ERR_UNSUPPORTED_SHAPE;
   gshard_moe_ep_layout l;
   l.rank = rank; l.world = world;
   l.groups_local = shape->G / world; l.experts_local = shape->E / world;
@@ -122,9 +121,22 @@ size_t gshard_moe_ep_workspace_bytes(const gshard_moe_shape* shape, int world) {
   return plan_forward(dl).total + 2 * align_up((size_t)dl.R * dl.M * dl.esize);
 }
 
+size_t gshard_moe_ep_context_bytes(const gshard_moe_shape* shape, int world) {
+  gshard_moe_ep_layout l;
+  if (make_layout(shape, 0, world, &l) != GSHARD_OK) return 0;
+  return plan_context(make_dims(l.local)).total;
+}
+
+size_t gshard_moe_ep_backward_workspace_bytes(const gshard_moe_shape* shape, int world) {
+  gshard_moe_ep_layout l;
+  if (make_layout(shape, 0, world, &l) != GSHARD_OK) return 0;
+  const Dims dl = make_dims(l.local);
+  return plan_backward(dl).total + 2 * align_up((size_t)dl.R * dl.M * dl.esize);
+}
+
 int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int world, const void* x_local,
                                const void* wg, const void* wi_local, const void* wo_local, const float* u_local,
-                               void* y_local, float* l_aux, const gshard_moe_routing* routing_out,
+                               void* y_local, float* l_aux, const gshard_moe_routing* routing_out, void* context,
                                const gshard_ep_comm* comm, void* workspace, size_t workspace_bytes,
                                void* cuda_stream) {
   launch_counter().n = 0;
@@ -137,6 +149,8 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
   if (l_aux == nullptr) return GSHARD_ERR_INVALID_ARG;
   if (world > 1 && (!comm || !comm->all_to_all || !comm->all_reduce_sum_f32)) return GSHARD_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSHARD_ERR_INVALID_ARG;
+  const bool save = (shape->flags & GSHARD_FLAG_SAVE_FOR_BACKWARD) != 0;
+  if (save && (!context || reinterpret_cast<uintptr_t>(context) % kAlign)) return GSHARD_ERR_INVALID_ARG;
   if (workspace_bytes < gshard_moe_ep_workspace_bytes(shape, world)) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
   const int rcd = check_device();
   if (rcd != GSHARD_OK) return rcd;
@@ -145,7 +159,9 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
   const Dims dl = make_dims(l.local);          // G = Gl, E global
   const Dims df = make_dims(l.ffn);            // G global, E = El: rows per expert = G*C
   const FwdPlan pl = plan_forward(dl);
+  const CtxPlan cp = plan_context(dl);
   unsigned char* ws = static_cast<unsigned char*>(workspace);
+  unsigned char* ctx = static_cast<unsigned char*>(context);
   const size_t slab_bytes = align_up((size_t)dl.R * dl.M * dl.esize);
   void* xa = ws + pl.total;                    // exchange buffers
   void* xb = ws + pl.total + slab_bytes;
@@ -153,25 +169,33 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
   if (routing_out) r = *routing_out;
   int* status = reinterpret_cast<int*>(ws + pl.status);
   if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
-  int32_t* expert_idx = pick(r.expert_idx, ws, pl.expert_idx);
-  int32_t* slot = pick(r.slot, ws, pl.slot);
-  float* weight = pick(r.weight, ws, pl.weight);
-  int32_t* slot_token = pick(r.slot_token, ws, pl.slot_token);
-  float* gate12 = reinterpret_cast<float*>(ws + pl.gate12);
+  // with SAVE_FOR_BACKWARD the routing tensors and the activations the backward needs live in the
+  // context: routing, softmax statistics and `out` in the LOCAL layout (this rank's groups), the
+  // expert inputs, h and its ReLU mask in the FFN layout (this rank's experts, all groups)
+  int32_t* expert_idx = save ? reinterpret_cast<int32_t*>(ctx + cp.expert_idx) : pick(r.expert_idx, ws, pl.expert_idx);
+  int32_t* slot = save ? reinterpret_cast<int32_t*>(ctx + cp.slot) : pick(r.slot, ws, pl.slot);
+  float* weight = save ? reinterpret_cast<float*>(ctx + cp.weight) : pick(r.weight, ws, pl.weight);
+  int32_t* first_count = save ? reinterpret_cast<int32_t*>(ctx + cp.first_count) : pick(r.first_count, ws, pl.first_count);
+  int32_t* slot_token = save ? reinterpret_cast<int32_t*>(ctx + cp.slot_token) : pick(r.slot_token, ws, pl.slot_token);
+  float* gate12 = save ? reinterpret_cast<float*>(ctx + cp.gate12) : reinterpret_cast<float*>(ws + pl.gate12);
+  float* rowmax = save ? reinterpret_cast<float*>(ctx + cp.rowmax) : reinterpret_cast<float*>(ws + pl.rowmax);
+  float* rowinv = save ? reinterpret_cast<float*>(ctx + cp.rowinv) : reinterpret_cast<float*>(ws + pl.rowinv);
   float* m = pick(r.m, ws, pl.m);
   void* buf = ws + pl.buf;
-  void* h = ws + pl.h;
-  void* out = ws + pl.out;
+  void* h = save ? static_cast<void*>(ctx + cp.h) : static_cast<void*>(ws + pl.h);
+  void* out = save ? static_cast<void*>(ctx + cp.out) : static_cast<void*>(ws + pl.out);
+  void* ffn_in_saved = save ? static_cast<void*>(ctx + cp.buf) : nullptr;
 
-  int rc = gate_stage(dl, pl, ws, x_local, wg, expert_idx, gate12, m, reinterpret_cast<float*>(ws + pl.rowmax),
-                      reinterpret_cast<float*>(ws + pl.rowinv), st);
+  int rc = gate_stage(dl, pl, ws, x_local, wg, expert_idx, gate12, m, rowmax, rowinv, st);
   if (rc != GSHARD_OK) return rc;
   // l_aux: this rank's group losses over the GLOBAL group count; the all-reduce below adds the shares
-  rc = launch_capacity(dl, expert_idx, gate12, u_local, m, slot, weight, pick(r.flags, ws, pl.flags),
-                       pick(r.first_count, ws, pl.first_count), pick(r.total_count, ws, pl.total_count), slot_token,
-                       pick(r.l_aux_group, ws, pl.l_aux_group), reinterpret_cast<int32_t*>(ws + pl.stats_group), l_aux,
-                       reinterpret_cast<long long*>(r.stats), st, shape->G);
+  rc = launch_capacity(dl, expert_idx, gate12, u_local, m, slot, weight, pick(r.flags, ws, pl.flags), first_count,
+                       pick(r.total_count, ws, pl.total_count), slot_token, pick(r.l_aux_group, ws, pl.l_aux_group),
+                       reinterpret_cast<int32_t*>(ws + pl.stats_group), l_aux, reinterpret_cast<long long*>(r.stats), st,
+                       shape->G);
   if (rc != GSHARD_OK) return rc;
+  // one rank: the dispatch buffer is the FFN input, so it goes straight to where the backward finds it
+  if (world == 1 && save) buf = ffn_in_saved;
   launch_dispatch(dl, x_local, slot_token, buf, st);
 
   const int row_vec = (int)(l.row_bytes / 16);
@@ -179,12 +203,13 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
   void* ffn_out = out;
   if (world > 1) {
     if (comm->all_to_all(comm->user, buf, xa, l.bytes_per_peer, cuda_stream) != 0) return GSHARD_ERR_CUDA;
-    launch_ep_regroup(xa, xb, world, l.experts_local, l.rows_local, row_vec, 0, st);
-    ffn_in = xb;
+    void* regrouped = save ? ffn_in_saved : xb;
+    launch_ep_regroup(xa, regrouped, world, l.experts_local, l.rows_local, row_vec, 0, st);
+    ffn_in = regrouped;
     ffn_out = xa;
   }
-  rc = ffn_stage(df, ffn_in, wi_local, wo_local, h, false, ffn_out, ws + pl.ffn_scratch, status, st, nullptr, nullptr,
-                 ws + pl.wt);
+  rc = ffn_stage(df, ffn_in, wi_local, wo_local, h, save, ffn_out, ws + pl.ffn_scratch, status, st, nullptr, nullptr,
+                 ws + pl.wt, nullptr, (save && !df.simt) ? reinterpret_cast<uint32_t*>(ctx + cp.hbits) : nullptr);
   if (rc != GSHARD_OK) return rc;
   if (world > 1) {
     launch_ep_regroup(xa, xb, world, l.experts_local, l.rows_local, row_vec, 1, st);
@@ -192,6 +217,76 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
     if (comm->all_reduce_sum_f32(comm->user, l_aux, 1, cuda_stream) != 0) return GSHARD_ERR_CUDA;
   }
   launch_combine(dl, out, expert_idx, slot, weight, y_local, st, dl.add_residual ? x_local : nullptr);
+  if (save) {   // hand the caller the routing tensors it asked for
+    struct { void* dst; const void* src; size_t n; } cps[] = {
+        {r.expert_idx, expert_idx, (size_t)dl.N * 2 * 4}, {r.slot, slot, (size_t)dl.N * 2 * 4},
+        {r.weight, weight, (size_t)dl.N * 2 * 4},         {r.first_count, first_count, (size_t)dl.G * dl.E * 4},
+        {r.slot_token, slot_token, (size_t)dl.R * 4}};
+    for (auto& c : cps)
+      if (c.dst && cudaMemcpyAsync(c.dst, c.src, c.n, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  }
+  return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
+}
+
+int gshard_moe_top2_backward_ep(const gshard_moe_shape* shape, int rank, int world, const void* x_local, const void* wg,
+                                const void* wi_local, const void* wo_local, const void* context, const void* dy_local,
+                                float l_aux_weight, void* dx_local, float* dwg, void* dwi_local, void* dwo_local,
+                                const gshard_ep_comm* comm, void* workspace, size_t workspace_bytes, void* cuda_stream) {
+  launch_counter().n = 0;
+  gshard_moe_ep_layout l;
+  const int rcl = make_layout(shape, rank, world, &l);
+  if (rcl != GSHARD_OK) return rcl;
+  if (!(shape->flags & GSHARD_FLAG_SAVE_FOR_BACKWARD)) return GSHARD_ERR_INVALID_ARG;
+  const void* ptrs[] = {x_local, wg, wi_local, wo_local, context, dy_local, dx_local, dwg, dwi_local, dwo_local, workspace};
+  for (const void* p : ptrs)
+    if (p == nullptr || !aligned16(p)) return GSHARD_ERR_INVALID_ARG;
+  if (world > 1 && (!comm || !comm->all_to_all || !comm->all_reduce_sum_f32)) return GSHARD_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign || reinterpret_cast<uintptr_t>(context) % kAlign)
+    return GSHARD_ERR_INVALID_ARG;
+  if (workspace_bytes < gshard_moe_ep_backward_workspace_bytes(shape, world)) return GSHARD_ERR_WORKSPACE_TOO_SMALL;
+  const int rcd = check_device();
+  if (rcd != GSHARD_OK) return rcd;
+
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const Dims dl = make_dims(l.local);
+  const Dims df = make_dims(l.ffn);
+  const BwdPlan bp = plan_backward(dl);
+  const CtxPlan cp = plan_context(dl);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  const unsigned char* ctx = static_cast<const unsigned char*>(context);
+  const size_t slab_bytes = align_up((size_t)dl.R * dl.M * dl.esize);
+  void* xa = ws + bp.total;
+  void* xb = ws + bp.total + slab_bytes;
+  int* status = reinterpret_cast<int*>(ws + bp.status);
+  if (cudaMemsetAsync(status, 0, sizeof(int), st) != cudaSuccess) return GSHARD_ERR_CUDA;
+  const int row_vec = (int)(l.row_bytes / 16);
+
+  // 1. combine backward over the local groups: dw per choice, dout [E, Gl*C, M]
+  int rc = backward_combine_stage(dl, ctx, dy_local, ws, st);
+  if (rc != GSHARD_OK) return rc;
+  // 2. the gradients of the expert outputs travel to the experts' owners, as the inputs did
+  const void* dout_ffn = ws + bp.dout;
+  void* dbuf_ffn = ws + bp.dbuf;
+  if (world > 1) {
+    if (comm->all_to_all(comm->user, ws + bp.dout, xa, l.bytes_per_peer, cuda_stream) != 0) return GSHARD_ERR_CUDA;
+    launch_ep_regroup(xa, xb, world, l.experts_local, l.rows_local, row_vec, 0, st);
+    dout_ffn = xb;
+    dbuf_ffn = ws + bp.dout;                  // the local dout has been sent: its region takes dbuf in FFN order
+  }
+  // 3. expert FFN backward over the local experts and all groups' rows
+  rc = backward_expert_stage(df, dout_ffn, ctx + cp.h, df.simt ? nullptr : reinterpret_cast<const uint32_t*>(ctx + cp.hbits),
+                             ctx + cp.buf, wi_local, wo_local, ws + bp.dh, dbuf_ffn, dwi_local, dwo_local, status, st);
+  if (rc != GSHARD_OK) return rc;
+  // 4. the gradients of the expert inputs travel back to the groups' owners
+  if (world > 1) {
+    launch_ep_regroup(dbuf_ffn, xa, world, l.experts_local, l.rows_local, row_vec, 1, st);
+    if (comm->all_to_all(comm->user, xa, ws + bp.dbuf, l.bytes_per_peer, cuda_stream) != 0) return GSHARD_ERR_CUDA;
+  }
+  // 5. gating backward and dx over the local groups; wg is replicated, so its gradient is the sum of
+  //    the ranks' contributions
+  rc = backward_gate_stage(dl, x_local, wg, ctx, dy_local, l_aux_weight, shape->G, ws + bp.dbuf, dx_local, dwg, ws, st);
+  if (rc != GSHARD_OK) return rc;
+  if (world > 1 && comm->all_reduce_sum_f32(comm->user, dwg, (size_t)dl.M * dl.E, cuda_stream) != 0) return GSHARD_ERR_CUDA;
   return cudaGetLastError() == cudaSuccess ? GSHARD_OK : GSHARD_ERR_CUDA;
 }
 
@@ -314,7 +409,7 @@ int gshard_moe_top2_forward_ep_p2p(const gshard_moe_shape* shape, int rank, int 
   gshard_moe_ep_layout l;
   const int rcl = make_layout(shape, rank, world, &l);
   if (rcl != GSHARD_OK) return rcl;
-  if (world > kMaxPeers) return GSHARD_ERR_UNSUPPORTED_SHAPE;
+  if (world > kMaxPeers || (shape->flags & GSHARD_FLAG_SAVE_FOR_BACKWARD)) return GSHARD_ERR_UNSUPPORTED_SHAPE;
   const void* ptrs[] = {x_local, wg, wi_local, wo_local, u_local, y_local, workspace};
   for (const void* p : ptrs)
     if (p == nullptr || !aligned16(p)) return GSHARD_ERR_INVALID_ARG;

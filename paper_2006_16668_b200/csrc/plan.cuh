@@ -128,4 +128,13 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
               void* wt = nullptr, const int* tile_base = nullptr, uint32_t* relu_bits_out = nullptr);
 int check_device();
 
+// The three parts of the backward pass (backward.cu); workspace laid out by plan_backward(d),
+// context by plan_context(d).
+int backward_combine_stage(const Dims& d, const void* context, const void* dy, void* workspace, cudaStream_t st);
+int backward_expert_stage(const Dims& d, const void* dout, const void* h, const uint32_t* hbits, const void* buf,
+                          const void* wi, const void* wo, void* dh, void* dbuf, void* dwi, void* dwo, int* status,
+                          cudaStream_t st);
+int backward_gate_stage(const Dims& d, const void* x, const void* wg, const void* context, const void* dy, float k_aux,
+                        int groups_in_mean, const void* dbuf, void* dx, float* dwg, void* workspace, cudaStream_t st);
+
 }  // namespace gshard

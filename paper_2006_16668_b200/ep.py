@@ -20,14 +20,16 @@ from . import binding as B
 class TorchDistComm:
     """A ``gshard_ep_comm`` whose all-to-all and all-reduce are torch.distributed collectives.
 
-    The library passes raw device pointers; they always point into the workspace of the call (or at
-    the l_aux scalar), so they are turned back into views of those tensors.  torch's NCCL collectives
-    order themselves after the current stream and make it wait for their completion, which is the
-    contract of the callbacks as long as the library call is made on torch's current stream.
+    The library passes raw device pointers; they always point into a tensor of the call (workspace,
+    context, the l_aux scalar, dwg), so they are turned back into views of the tensors registered
+    here.  torch's NCCL collectives order themselves after the current stream and make it wait for
+    their completion, which is the contract of the callbacks as long as the library call is made on
+    torch's current stream.
     """
 
-    def __init__(self, workspace: torch.Tensor, l_aux: torch.Tensor, group=None):
-        self.workspace, self.l_aux, self.group = workspace, l_aux, group
+    def __init__(self, tensors, group=None):
+        self.tensors = [t for t in tensors if t is not None]
+        self.group = group
         self.world = dist.get_world_size(group) if dist.is_initialized() else 1
         self.error = None
         self._a2a = B.ALL_TO_ALL_FN(self._all_to_all)        # keep the thunks alive
@@ -35,10 +37,11 @@ class TorchDistComm:
         self.struct = B.gshard_ep_comm(self._a2a, self._ar, None)
 
     def _view(self, ptr: int, nbytes: int) -> torch.Tensor:
-        off = ptr - self.workspace.data_ptr()
-        if off < 0 or off + nbytes > self.workspace.numel():
-            raise ValueError("collective buffer outside the workspace")
-        return self.workspace[off:off + nbytes]
+        for t in self.tensors:
+            off = ptr - t.data_ptr()
+            if 0 <= off and off + nbytes <= t.numel() * t.element_size():
+                return t.view(-1).view(torch.uint8)[off:off + nbytes]
+        raise ValueError("collective buffer outside the tensors of the call")
 
     def _all_to_all(self, user, send, recv, bytes_per_peer, stream):
         try:
@@ -51,9 +54,7 @@ class TorchDistComm:
 
     def _all_reduce(self, user, buf, count, stream):
         try:
-            if buf != self.l_aux.data_ptr() or count > self.l_aux.numel():
-                raise ValueError("all-reduce buffer is not the l_aux tensor")
-            dist.all_reduce(self.l_aux[:count], op=dist.ReduceOp.SUM, group=self.group)
+            dist.all_reduce(self._view(buf, 4 * count).view(torch.float32), op=dist.ReduceOp.SUM, group=self.group)
             return 0
         except Exception:
             self.error = traceback.format_exc()
@@ -169,21 +170,32 @@ def local_slices(layout: B.gshard_moe_ep_layout):
     return slice(g0, g0 + layout.groups_local), slice(e0, e0 + layout.experts_local)
 
 
+def _call(fn, comm, what):
+    try:
+        fn(comm.struct if comm is not None else None)
+    except B.GshardError:
+        if comm is not None and getattr(comm, "error", None):
+            raise RuntimeError(f"a collective of the expert-parallel {what} failed:\n" + comm.error)
+        raise
+
+
 def forward(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux, routing_out=None,
-            workspace=None, group=None, comm=None):
+            workspace=None, group=None, comm=None, context=None):
     """One expert-parallel forward on this rank (global `shape`); the process group must be
     initialised when world > 1.  Enqueues on torch's current stream.  comm: a NcclComm to reuse, else
-    the collectives go through torch.distributed."""
-    if comm is not None:
-        B.gshard_moe_top2_forward_ep(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux,
-                                     routing_out, comm.struct, workspace)
-        return
-    if world > 1:
-        comm = TorchDistComm(workspace, l_aux, group)
-    try:
-        B.gshard_moe_top2_forward_ep(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local, l_aux,
-                                     routing_out, comm.struct if comm else None, workspace)
-    except B.GshardError:
-        if comm is not None and comm.error:
-            raise RuntimeError("a collective of the expert-parallel forward failed:\n" + comm.error)
-        raise
+    the collectives go through torch.distributed.  context: with SAVE_FOR_BACKWARD, a uint8 tensor of
+    gshard_moe_ep_context_bytes(shape, world) for `backward`."""
+    if comm is None and world > 1:
+        comm = TorchDistComm([workspace, context, l_aux], group)
+    _call(lambda c: B.gshard_moe_top2_forward_ep(shape, rank, world, x_local, wg, wi_local, wo_local, u_local, y_local,
+                                                 l_aux, routing_out, c, workspace, context=context), comm, "forward")
+
+
+def backward(shape, rank, world, x_local, wg, wi_local, wo_local, context, dy_local, l_aux_weight, dx_local, dwg,
+             dwi_local, dwo_local, workspace=None, group=None, comm=None):
+    """The backward of `forward` on this rank; dwg ends as the sum over the ranks."""
+    if comm is None and world > 1:
+        comm = TorchDistComm([workspace, dwg], group)
+    _call(lambda c: B.gshard_moe_top2_backward_ep(shape, rank, world, x_local, wg, wi_local, wo_local, context, dy_local,
+                                                  l_aux_weight, dx_local, dwg, dwi_local, dwo_local, c, workspace),
+          comm, "backward")

@@ -16,7 +16,8 @@ from .inputs import _normal
 
 
 def run(args, cfg, dev, world, rank, metric, unit, sampler):
-    shape = B.make_shape(cfg, flags=args.flags)
+    train = bool(getattr(cfg, "backward", False))            # a training-step configuration: forward + backward
+    shape = B.make_shape(cfg, flags=args.flags | (B.GSHARD_FLAG_SAVE_FOR_BACKWARD if train else 0))
     layout = B.gshard_moe_ep_plan(shape, rank, world)
     Gl, El, dt = layout.groups_local, layout.experts_local, cfg.torch_dtype
     gen = torch.Generator(device=dev).manual_seed(cfg.seed)              # wg is replicated: same draw everywhere
@@ -34,12 +35,23 @@ def run(args, cfg, dev, world, rank, metric, unit, sampler):
     # exchange: NCCL called from inside the library (default), torch.distributed through callbacks, or
     # fused into the dispatch and combine kernels (peer stores and loads on symmetric memory)
     mode = getattr(args, "ep_comm", "nccl")
+    if train and mode == "p2p":
+        raise SystemExit("--ep-comm p2p is the forward only; use nccl or torch for a training-step configuration")
     comm = ep.NcclComm(rank, world) if (world > 1 and mode in ("nccl", "p2p")) else None
     exchange = ep.SymmetricExchange(shape, rank, world) if mode == "p2p" else None
+    if train:
+        ctx = torch.empty(B.gshard_moe_ep_context_bytes(shape, world), dtype=torch.uint8, device=dev)
+        wsb = torch.empty(B.gshard_moe_ep_backward_workspace_bytes(shape, world), dtype=torch.uint8, device=dev)
+        dy = _normal((Gl, cfg.S, cfg.M), 1.0, gen, dev, dt)
+        dx, dwi, dwo = torch.empty_like(x), torch.empty_like(wi), torch.empty_like(wo)
+        dwg = torch.empty(cfg.M, cfg.E, dtype=torch.float32, device=dev)
 
     def step():
         if exchange is not None:
             ep.forward_p2p(shape, rank, world, x, wg, wi, wo, u, y, l_aux, exchange, None, ws, comm=comm)
+        elif train:
+            ep.forward(shape, rank, world, x, wg, wi, wo, u, y, l_aux, None, ws, comm=comm, context=ctx)
+            ep.backward(shape, rank, world, x, wg, wi, wo, ctx, dy, cfg.k_aux, dx, dwg, dwi, dwo, wsb, comm=comm)
         else:
             ep.forward(shape, rank, world, x, wg, wi, wo, u, y, l_aux, None, ws, comm=comm)
 
@@ -54,6 +66,10 @@ def run(args, cfg, dev, world, rank, metric, unit, sampler):
     if B.gshard_moe_last_device_status(ws) != B.GSHARD_OK:
         raise SystemExit("device status is not OK after warm-up")
     launches = B.gshard_moe_last_launch_count()
+    if train:                                                 # the counter restarts in every call: add the forward's
+        ep.forward(shape, rank, world, x, wg, wi, wo, u, y, l_aux, None, ws, comm=comm, context=ctx)
+        launches += B.gshard_moe_last_launch_count()
+        barrier()
     sampler.start()
     sampler.wait_first_sample()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -80,7 +96,7 @@ def run(args, cfg, dev, world, rank, metric, unit, sampler):
                                           f"{layout.bytes_per_peer} bytes per peer before and after the expert FFN, "
                                           + ("stored and loaded peer to peer by the dispatch and combine kernels"
                                              if exchange is not None else f"all-to-all ({mode})"),
-                           "l2": "inputs larger than L2"},
+                           "step": "forward + backward" if train else "forward", "l2": "inputs larger than L2"},
                 "roofline": None, "cpu_baseline": None, "e2e": None, "gpu_launches": launches * args.steps,
                 "clocks": sampler.summary(), "device_status": status}
         print(json.dumps(line))

@@ -46,17 +46,20 @@ class _World:
 class _ThreadComm:
     """gshard_ep_comm for one emulated rank (a host thread with its own stream)."""
 
-    def __init__(self, world, rank, workspace, l_aux, stream):
-        self.w, self.rank, self.ws, self.l_aux, self.stream = world, rank, workspace, l_aux, stream
+    def __init__(self, world, rank, tensors, stream):
+        self.w, self.rank, self.tensors, self.stream = world, rank, [t for t in tensors if t is not None], stream
         self.error = None
         self._a2a = B.ALL_TO_ALL_FN(self._all_to_all)
         self._ar = B.ALL_REDUCE_FN(self._all_reduce)
         self.struct = B.gshard_ep_comm(self._a2a, self._ar, None)
 
     def _view(self, ptr, n):
-        off = ptr - self.ws.data_ptr()
-        assert 0 <= off and off + n <= self.ws.numel()
-        return self.ws[off:off + n]
+        """The n bytes at ptr as a view of the tensor of this call that contains them."""
+        for t in self.tensors:
+            off = ptr - t.data_ptr()
+            if 0 <= off and off + n <= t.numel() * t.element_size():
+                return t.view(-1).view(torch.uint8)[off:off + n]
+        raise AssertionError("collective buffer outside the tensors of the call")
 
     def _exchange(self, mine, consume):
         """Publish `mine`, wait until every rank has published, run consume(all buffers) on this
@@ -95,10 +98,10 @@ class _ThreadComm:
 
     def _all_reduce(self, user, buf, count, stream):
         try:
-            assert buf == self.l_aux.data_ptr() and count == 1
-            total = self._exchange(self.l_aux, lambda bufs: torch.stack([b.clone() for b in bufs]).sum(0))
+            mine = self._view(buf, 4 * count).view(torch.float32)
+            total = self._exchange(mine, lambda bufs: torch.stack([b.clone() for b in bufs]).sum(0))
             with torch.cuda.stream(self.stream):
-                self.l_aux.copy_(total)
+                mine.copy_(total)
             return 0
         except Exception:
             self.error = traceback.format_exc()
@@ -123,13 +126,28 @@ def _run_ranks(cfg, inp, world, flags=0):
             y = torch.empty_like(x)
             l_aux = torch.zeros(1, device="cuda")
             torch.cuda.synchronize()
-            comm = _ThreadComm(state, rank, ws, l_aux, stream)
+            save = bool(flags & B.GSHARD_FLAG_SAVE_FOR_BACKWARD)
+            ctx = torch.empty(B.gshard_moe_ep_context_bytes(shape, world), dtype=torch.uint8, device="cuda") if save else None
+            comm = _ThreadComm(state, rank, [ws, ctx, l_aux], stream)
             B.gshard_moe_top2_forward_ep(shape, rank, world, x, inp["wg"], wi, wo, u, y, l_aux, rs, comm.struct, ws,
-                                         stream)
+                                         stream, context=ctx)
             assert comm.error is None, comm.error
             assert B.gshard_moe_last_device_status(ws, stream) == B.GSHARD_OK
+            grads = None
+            if save:
+                dy = inp["dy"][gs].contiguous()
+                wsb = torch.empty(B.gshard_moe_ep_backward_workspace_bytes(shape, world), dtype=torch.uint8, device="cuda")
+                dx, dwi, dwo = torch.empty_like(x), torch.empty_like(wi), torch.empty_like(wo)
+                dwg = torch.empty(cfg.M, cfg.E, dtype=torch.float32, device="cuda")
+                torch.cuda.synchronize()
+                comm_b = _ThreadComm(state, rank, [wsb, dwg], stream)
+                B.gshard_moe_top2_backward_ep(shape, rank, world, x, inp["wg"], wi, wo, ctx, dy, cfg.k_aux, dx, dwg, dwi,
+                                              dwo, comm_b.struct, wsb, stream)
+                assert comm_b.error is None, comm_b.error
+                assert B.gshard_moe_last_device_status(wsb, stream) == B.GSHARD_OK
+                grads = (dx, dwg, dwi, dwo)
             stream.synchronize()
-            results[rank] = (y, l_aux, rt)
+            results[rank] = (y, l_aux, rt, grads)
         except Exception:
             errors[rank] = traceback.format_exc()
             state.barrier.abort()
@@ -174,6 +192,59 @@ def test_expert_parallel_equals_single_gpu(world, name, G, S, M, H, E, C, dtype,
         else:
             assert float(r[1]) == pytest.approx(float(l_ref), rel=1e-6)
             assert torch.equal(r[1], results[0][1])
+
+
+BWD_CASES = [
+    ("f32", 4, 64, 32, 64, 8, 12, "f32"),
+    ("bf16_pairs", 4, 256, 256, 512, 16, 40, "bf16"),          # 160 rows per expert on one GPU, per rank the same
+    ("bf16_resident_wgrad", 4, 512, 512, 512, 16, 64, "bf16"),  # 256 rows per expert: the weight-gradient kernel
+]
+
+
+@pytest.mark.parametrize("name,G,S,M,H,E,C,dtype", BWD_CASES, ids=[c[0] for c in BWD_CASES])
+@pytest.mark.parametrize("world", [1, 2, 4])
+def test_expert_parallel_backward_equals_single_gpu(world, name, G, S, M, H, E, C, dtype):
+    """gshard_moe_top2_backward_ep after gshard_moe_top2_forward_ep with SAVE_FOR_BACKWARD.  The expert
+    FFN sees the same rows in the same order as on one GPU and the token-wise kernels are row-wise, so
+    dx, dwi, dwo must have the single-GPU bits (whose parity with the oracle test_gpu_backward.py
+    establishes); dwg is a sum over tokens split differently (per-rank partial sums, then the
+    all-reduce), compared to 1e-5 relative, and must be identical on all ranks."""
+    from test_gpu_backward import run_fwd_bwd
+    cfg = MoEConfig(name, G=G, S=S, M=M, H=H, E=E, C=C, dtype=dtype, seed=2468, backward=True, k_aux=0.01)
+    inp = make_inputs(cfg, "cuda")
+    y_ref, l_ref, rt_ref, dx_ref, dwg_ref, dwi_ref, dwo_ref = run_fwd_bwd(cfg, inp)
+    results = _run_ranks(cfg, inp, world, B.GSHARD_FLAG_SAVE_FOR_BACKWARD)
+    bits = lambda t: t.contiguous().view(torch.uint8)
+    assert torch.equal(bits(torch.cat([r[0] for r in results])), bits(y_ref))
+    assert torch.equal(bits(torch.cat([r[3][0] for r in results])), bits(dx_ref)), "dx"
+    assert torch.equal(bits(torch.cat([r[3][2] for r in results])), bits(dwi_ref)), "dwi"
+    assert torch.equal(bits(torch.cat([r[3][3] for r in results])), bits(dwo_ref)), "dwo"
+    scale = float(dwg_ref.abs().max())
+    for r in results:
+        assert float((r[3][1] - dwg_ref).abs().max()) <= 1e-5 * scale + 1e-9, "dwg"
+        assert torch.equal(r[3][1], results[0][3][1])
+    for k in ("expert_idx", "slot", "weight", "first_count"):          # the routing the caller asked for
+        assert torch.equal(torch.cat([r[2][k] for r in results]), rt_ref[k]), k
+
+
+def test_expert_parallel_backward_against_the_oracle():
+    """World 2 straight against the oracle's gradients (not through the single-GPU layer)."""
+    import numpy as np
+    from test_gpu_backward import GRAD_TOL, oracle_with_gpu_routing
+    from oracle import gshard_oracle as orc
+    from parity_util import rel_fro, to_np
+    cfg = MoEConfig("ep_bwd_oracle", G=4, S=128, M=64, H=128, E=16, C=12, dtype="bf16", seed=99, backward=True, k_aux=0.01)
+    inp = make_inputs(cfg, "cuda")
+    results = _run_ranks(cfg, inp, 2, B.GSHARD_FLAG_SAVE_FOR_BACKWARD)
+    rt = {k: torch.cat([r[2][k] for r in results]) for k in ("expert_idx", "slot", "first_count")}
+    f = oracle_with_gpu_routing(cfg, inp, rt)
+    rdx, rdwg, rdwi, rdwo = orc.backward(to_np(inp["x"]), to_np(inp["wg"]), to_np(inp["wi"]), to_np(inp["wo"]), f,
+                                         to_np(inp["dy"]), cfg.k_aux)
+    errs = {"dx": rel_fro(to_np(torch.cat([r[3][0] for r in results])), rdx),
+            "dwg": rel_fro(to_np(results[1][3][1]), rdwg),
+            "dwi": rel_fro(to_np(torch.cat([r[3][2] for r in results])), rdwi),
+            "dwo": rel_fro(to_np(torch.cat([r[3][3] for r in results])), rdwo)}
+    assert all(v <= GRAD_TOL for v in errs.values()), errs
 
 
 class _P2PRank:
@@ -312,11 +383,19 @@ def test_bad_arguments():
     fake = 0x10000
     import ctypes
     args = [fake] * 6
-    assert lib.gshard_moe_top2_forward_ep(ctypes.byref(shape), 0, 3, *args, fake, None, None, fake, 1 << 40, None) == B.GSHARD_ERR_UNSUPPORTED_SHAPE
-    assert lib.gshard_moe_top2_forward_ep(ctypes.byref(shape), 2, 2, *args, fake, None, None, fake, 1 << 40, None) == B.GSHARD_ERR_INVALID_ARG
-    # world > 1 needs the collectives
-    assert lib.gshard_moe_top2_forward_ep(ctypes.byref(shape), 0, 2, *args, fake, None, None, fake, 1 << 40, None) == B.GSHARD_ERR_INVALID_ARG
-    assert lib.gshard_moe_top2_forward_ep(ctypes.byref(shape), 0, 1, *args, fake, None, None, fake, 16, None) == B.GSHARD_ERR_WORKSPACE_TOO_SMALL
+    fwd = lambda rank, world, ctx, nbytes, sh=shape: lib.gshard_moe_top2_forward_ep(
+        ctypes.byref(sh), rank, world, *args, fake, None, ctx, None, fake, nbytes, None)
+    assert fwd(0, 3, None, 1 << 40) == B.GSHARD_ERR_UNSUPPORTED_SHAPE
+    assert fwd(2, 2, None, 1 << 40) == B.GSHARD_ERR_INVALID_ARG
+    assert fwd(0, 2, None, 1 << 40) == B.GSHARD_ERR_INVALID_ARG                 # world > 1 needs the collectives
+    assert fwd(0, 1, None, 16) == B.GSHARD_ERR_WORKSPACE_TOO_SMALL
+    saving = B.make_shape(cfg, flags=B.GSHARD_FLAG_SAVE_FOR_BACKWARD)
+    assert fwd(0, 1, None, 1 << 40, saving) == B.GSHARD_ERR_INVALID_ARG         # SAVE_FOR_BACKWARD needs a context
+    bwd = lambda sh, nbytes: lib.gshard_moe_top2_backward_ep(ctypes.byref(sh), 0, 1, *([fake] * 6), 0.01, *([fake] * 4),
+                                                            None, fake, nbytes, None)
+    assert bwd(shape, 1 << 40) == B.GSHARD_ERR_INVALID_ARG                      # forward did not save
+    assert bwd(saving, 16) == B.GSHARD_ERR_WORKSPACE_TOO_SMALL
+    assert B.gshard_moe_ep_context_bytes(saving, 1) == B.gshard_moe_top2_context_bytes(saving)
 
 
 def test_nccl_comm_single_rank():
