@@ -142,7 +142,11 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
                                                  the inverse slot list; every access bounds-checked) and
                                                  records GSHARD_ERR_INTERNAL in the status word on a
                                                  violation - nothing traps */
-#define GSHARD_FLAG_ALL 65535u
+#define GSHARD_FLAG_BULK_DISPATCH 65536u      /* dispatch: token rows move through the TMA unit (bulk
+                                                 global->shared->global copies, empty slots as bulk
+                                                 stores of a zero row) instead of 16-byte loads and
+                                                 stores; same bytes */
+#define GSHARD_FLAG_ALL 131071u
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
  * (Algorithm 1 "Data"; the paper sets C = 2N/(G*E) = 2S/E).  Limits: M % 8 == 0, H % 8 == 0,

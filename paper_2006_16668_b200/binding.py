@@ -41,6 +41,7 @@ GSHARD_FLAG_BWD_PAIRED_GEMMS = 4096
 GSHARD_FLAG_TF32_EXPERTS = 8192
 GSHARD_FLAG_COMPACT_SLOTS = 16384
 GSHARD_FLAG_DEBUG_CHECKS = 32768
+GSHARD_FLAG_BULK_DISPATCH = 65536
 
 
 class gshard_moe_shape(Structure):

@@ -109,7 +109,7 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   if (!tile_base && ffn_runs_fused(d, keep_h)) {
     const int rc = launch_ffn_fused(d, buf, wi, wo, fused_scratch, out, status, st, x, slot_token);
     if (rc != GSHARD_ERR_UNSUPPORTED_SHAPE) return rc;
-    if (x) launch_dispatch(d, x, slot_token, const_cast<void*>(buf), st);   // rows were to be gathered in the launch
+    if (x) launch_dispatch(d, x, slot_token, const_cast<void*>(buf), st, status);   // rows were to be gathered in the launch
   }
   UmmaGemm g{};
   g.A = buf; g.B = wi; g.C = h; g.rows = d.rows; g.cols = d.H; g.K = d.M; g.batch = d.E;
@@ -216,7 +216,7 @@ int forward_device(const gshard_moe_shape* shape, const void* x, const void* wg,
     launch_compact(d, slot_token, crow_token, slot_crow, kept, tile_base, st);
     launch_dispatch_compact(d, x, crow_token, kept, buf, st);
   } else if (!gather) {
-    launch_dispatch(d, x, slot_token, buf, st);
+    launch_dispatch(d, x, slot_token, buf, st, status);
   }
   // optional event pair around the expert FFN, armed for one call by gshard_moe_time_expert_ffn
   FfnTiming& ft = ffn_timing();

@@ -111,6 +111,7 @@ struct Dims {
   bool gather_dispatch; // single-launch FFN gathers its rows from x instead of reading a dispatch buffer
   bool tf32_experts;    // fp32 dtype: expert FFN contractions on the tensor cores in TF32
   bool compact_slots;   // grouped-GEMM expert FFN over compacted rows (empty slots skipped)
+  bool bulk_dispatch;   // dispatch rows move through the TMA unit (cp.async.bulk) instead of 16-byte loads and stores
   bool plain_stores;    // GEMM epilogues write with 16-byte stores instead of bulk tensor (TMA) stores
   bool debug_checks;    // forward: verify the routing tensors on the device and record a violation in the status word
   bool bwd_paired;      // backward: read-heavy and write-heavy expert GEMMs side by side on half of the SMs each
@@ -137,6 +138,7 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.add_residual = (s.flags & GSHARD_FLAG_ADD_RESIDUAL) != 0;
   d.bwd_paired = (s.flags & GSHARD_FLAG_BWD_PAIRED_GEMMS) != 0;
   d.plain_stores = (s.flags & GSHARD_FLAG_PLAIN_STORES) != 0;
+  d.bulk_dispatch = (s.flags & GSHARD_FLAG_BULK_DISPATCH) != 0;
   d.debug_checks = (s.flags & GSHARD_FLAG_DEBUG_CHECKS) != 0;
   d.tf32_experts = !d.bf16 && (s.flags & GSHARD_FLAG_TF32_EXPERTS) != 0;
   // Compacted slots: on request, and by default where an expert has at least six 128-row tiles, so

@@ -3,6 +3,7 @@
 // gather form with s_indices[E,G,C] in its section on mixing manual and automatic sharding).
 // Both are HBM-bound: one warp moves one row with 16-byte accesses.
 #include "kernels.cuh"
+#include "sm100_ptx.cuh"
 
 namespace gshard {
 
@@ -27,6 +28,92 @@ __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__
       const uint4 z = make_uint4(0, 0, 0, 0);
       for (int i = lane; i < row_vec; i += 32) dst[i] = z;
     }
+  }
+}
+
+// The same copy through the TMA unit (GSHARD_FLAG_BULK_DISPATCH).  Every warp owns a ring of kStages row
+// buffers in shared memory; its lane 0 keeps kStages - 2 bulk loads (global -> shared, completion
+// counted on an mbarrier per stage) and two bulk stores (shared -> global) in flight; an empty slot is
+// a bulk store from a row of zeros.  No thread touches the data; the warp's other lanes only fetch the
+// slot indices 32 rows ahead.  Row i of a warp's run uses stage i mod kStages; at
+// step i the row i - (kStages - 2) is completed (wait for its bytes, issue its store), then at most two
+// stores may still be reading shared memory - the one that last used stage i mod kStages was issued two
+// steps earlier - and the load of row i is issued.
+template <int kBulkWarps, int kBulkStages>
+__global__ void __launch_bounds__(kBulkWarps * 32) dispatch_bulk_kernel(const unsigned char* __restrict__ x,
+                                                                        const int32_t* __restrict__ slot_token,
+                                                                        unsigned char* __restrict__ buf, long long R,
+                                                                        int G, int S, int C, uint32_t row_bytes,
+                                                                        int* status) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ __align__(8) uint64_t bars[kBulkWarps][kBulkStages];
+  __shared__ int no_abort;
+  unsigned char* zero_row = smem;
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  unsigned char* ring = smem + (size_t)row_bytes * (1 + w * kBulkStages);
+  for (uint32_t i = threadIdx.x * 16; i < row_bytes; i += blockDim.x * 16)
+    *reinterpret_cast<uint4*>(zero_row + i) = make_uint4(0, 0, 0, 0);
+  if (threadIdx.x == 0) no_abort = 0;
+  if (lane == 0) {
+#pragma unroll
+    for (int s = 0; s < kBulkStages; ++s) ptx::mbar_init(&bars[w][s], 1);
+    ptx::fence_mbar_init();
+  }
+  ptx::fence_proxy_async();                     // the zero row, written by threads, is read by bulk stores
+  __syncthreads();
+
+  volatile int* abort_flag = status ? status : &no_abort;
+  // a warp owns a contiguous run of rows: coalesced index loads, one long run of destination bytes
+  const long long nwarps = (long long)gridDim.x * kBulkWarps;
+  const long long per_warp = (R + nwarps - 1) / nwarps;
+  const long long row0 = ((long long)blockIdx.x * kBulkWarps + w) * per_warp;
+  const long long n_rows = row0 < R ? (R - row0 < per_warp ? R - row0 : per_warp) : 0;
+  constexpr int kLag = kBulkStages - 2;
+  uint32_t parity = 0;                          // bit s: parity of the next completion on stage s
+  uint32_t loaded = 0;                          // bit s: the row in stage s has a load in flight (not an empty slot)
+  bool ok = true;
+  // the whole warp fetches the indices of the next 32 rows; lane 0 alone drives the copies
+  for (long long base = 0; base < n_rows + kLag; base += 32) {
+    const long long mine = base + lane;
+    const int tok_lane = mine < n_rows ? slot_token[row0 + mine] : -1;
+#pragma unroll 1
+    for (int k = 0; k < 32; ++k) {
+      const long long i = base + k;
+      if (i >= n_rows + kLag) break;            // uniform over the warp
+      const int tok = __shfl_sync(0xffffffffu, tok_lane, k);
+      if (lane != 0 || !ok) continue;
+      const long long j = i - kLag;             // the row to complete
+      if (j >= 0) {
+        const int s = (int)(j % kBulkStages);
+        unsigned char* dst = buf + (row0 + j) * (long long)row_bytes;
+        if ((loaded >> s) & 1u) {
+          ok = ptx::mbar_wait(&bars[w][s], (parity >> s) & 1u, abort_flag);
+          parity ^= 1u << s;
+          if (ok) ptx::bulk_store(dst, ring + (size_t)s * row_bytes, row_bytes);
+        } else {
+          ptx::bulk_store(dst, zero_row, row_bytes);
+        }
+        ptx::tma_store_commit();
+      }
+      if (i < n_rows && ok) {
+        ptx::bulk_wait_read<2>();
+        const int s = (int)(i % kBulkStages);
+        if (tok >= 0 && tok < S) {
+          const long long r = row0 + i;         // r = (e*G + g)*C + c
+          const int g = (int)((r / C) % G);
+          ptx::mbar_arrive_expect_tx(&bars[w][s], row_bytes);
+          ptx::bulk_load(ring + (size_t)s * row_bytes, x + ((long long)g * S + tok) * (long long)row_bytes, row_bytes,
+                         &bars[w][s]);
+          loaded |= 1u << s;
+        } else {
+          loaded &= ~(1u << s);
+        }
+      }
+    }
+  }
+  if (lane == 0) {
+    if (!ok && status) set_device_status(status, GSHARD_ERR_TIMEOUT);
+    ptx::tma_store_wait_all();                  // shared memory must outlive the stores that read it
   }
 }
 
@@ -145,9 +232,29 @@ void launch_dispatch_compact(const Dims& d, const void* x, const int32_t* crow_t
   count_launch();
 }
 
-void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st) {
+void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st, int* status) {
   NvtxRange range("gshard.dispatch");
   const int row_vec = (int)((size_t)d.M * d.esize / 16);
+  const size_t row_bytes = (size_t)d.M * d.esize;
+  constexpr int kWarps = 16, kStages = 4;       // of the ring shapes tried (4-32 warps, 3-8 stages) the fastest
+  const size_t bulk_smem = row_bytes * (1 + (size_t)kWarps * kStages);
+  if (d.bulk_dispatch && bulk_smem <= 200 * 1024) {
+    static thread_local int attr_device = -1;   // the attribute is per function and device
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (attr_device != dev) {
+      cudaFuncSetAttribute(dispatch_bulk_kernel<kWarps, kStages>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+      attr_device = dev;
+    }
+    long long blocks = (d.R + kWarps - 1) / kWarps;
+    const long long cap = device_sms();         // one CTA per multiprocessor: the rings fill its shared memory
+    if (blocks > cap) blocks = cap;
+    dispatch_bulk_kernel<kWarps, kStages><<<(int)blocks, kWarps * 32, bulk_smem, st>>>(
+        static_cast<const unsigned char*>(x), slot_token, static_cast<unsigned char*>(buf), d.R, d.G, d.S, d.C,
+        (uint32_t)row_bytes, status);
+    count_launch();
+    return;
+  }
   dispatch_kernel<<<grid_for_rows(d.R), 256, 0, st>>>(reinterpret_cast<const uint4*>(x), slot_token,
                                                       reinterpret_cast<uint4*>(buf), d.R, d.G, d.S, d.C, row_vec);
   count_launch();

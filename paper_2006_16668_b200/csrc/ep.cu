@@ -196,7 +196,7 @@ int gshard_moe_top2_forward_ep(const gshard_moe_shape* shape, int rank, int worl
   if (rc != GSHARD_OK) return rc;
   // one rank: the dispatch buffer is the FFN input, so it goes straight to where the backward finds it
   if (world == 1 && save) buf = ffn_in_saved;
-  launch_dispatch(dl, x_local, slot_token, buf, st);
+  launch_dispatch(dl, x_local, slot_token, buf, st, status);
 
   const int row_vec = (int)(l.row_bytes / 16);
   const void* ffn_in = buf;

@@ -40,7 +40,8 @@ void launch_routing_check(const Dims& d, const int32_t* expert_idx, const int32_
                           const uint8_t* flags, const int32_t* slot_token, int* status, cudaStream_t st);
 
 // dispatch_combine.cu
-void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st);
+void launch_dispatch(const Dims& d, const void* x, const int32_t* slot_token, void* buf, cudaStream_t st,
+                     int* status = nullptr);
 // slot_crow (optional): the expert outputs are stored by compacted row; slot_crow[e, g*C+c] is the row.
 void launch_combine(const Dims& d, const void* out, const int32_t* expert_idx, const int32_t* slot,
                     const float* weight, void* y, cudaStream_t st, const void* residual = nullptr,

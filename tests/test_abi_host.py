@@ -68,7 +68,7 @@ def test_workspace_sizes_for_the_paper_configs():
     (dict(C=0), B.GSHARD_ERR_INVALID_ARG), (dict(M=20), B.GSHARD_ERR_UNSUPPORTED_SHAPE),
     (dict(S=40000), B.GSHARD_ERR_UNSUPPORTED_SHAPE), (dict(E=20000), B.GSHARD_ERR_UNSUPPORTED_SHAPE),
     (dict(dtype="bf16", M=72), B.GSHARD_ERR_UNSUPPORTED_SHAPE),
-    (dict(flags=65536), B.GSHARD_ERR_INVALID_ARG),
+    (dict(flags=131072), B.GSHARD_ERR_INVALID_ARG),
     # more (group, 128-token tile) pairs, or 64-row tiles of the CUDA-core GEMM, than a grid's y extent
     (dict(G=70000, S=1), B.GSHARD_ERR_UNSUPPORTED_SHAPE), (dict(G=600, S=16384), B.GSHARD_ERR_UNSUPPORTED_SHAPE),
     (dict(flags=B.GSHARD_FLAG_FUSED_FFN | B.GSHARD_FLAG_UNFUSED_FFN), B.GSHARD_ERR_INVALID_ARG),

@@ -69,12 +69,13 @@ def test_capacity_kernel_bit_exact(G, S, E, C, variant_a, conc):
     assert float(l_aux) == pytest.approx(float(np.mean(l_groups)), rel=1e-5)
 
 
+@pytest.mark.parametrize("bulk", [0, B.GSHARD_FLAG_BULK_DISPATCH], ids=["vector_loads", "tma_bulk"])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_dispatch_and_combine(dtype):
+def test_dispatch_and_combine(dtype, bulk):
     G, S, M, H, E, C = 3, 50, 72, 8, 6, 5
     rng = np.random.default_rng(5)
     tdt = torch.float32 if dtype == "f32" else torch.bfloat16
-    shape = _shape(G, S, M, H, E, C, dtype, B.GSHARD_FLAG_SIMT_CONTRACTIONS if dtype == "bf16" else 0)
+    shape = _shape(G, S, M, H, E, C, dtype, (B.GSHARD_FLAG_SIMT_CONTRACTIONS if dtype == "bf16" else 0) | bulk)
     x = torch.randn(G, S, M, device="cuda").to(tdt)
     # a valid routing from the oracle
     p = rng.dirichlet(np.ones(E), size=(G, S))
@@ -217,3 +218,42 @@ def test_gate_stage_against_oracle(G, S, M, E, flags):
     B.gshard_moe_gate(shape, x, wg, ei2, g122, m2, ws)
     torch.cuda.synchronize()
     assert torch.equal(ei, ei2) and torch.equal(g12, g122) and torch.equal(m, m2)
+
+
+@pytest.mark.parametrize("G,S,M,E,C,dtype", [(8, 300, 1024, 64, 40, "bf16"),     # 2 KB rows, 20480 rows: 17-18 per warp, the ring turns twice
+                                             (4, 64, 4096, 16, 8, "f32"),        # 16 KB rows: ring too large, falls back
+                                             (1, 16, 64, 16, 2, "bf16")])        # 128-byte rows, fewer rows than warps
+def test_bulk_dispatch_is_the_same_copy(G, S, M, E, C, dtype):
+    """GSHARD_FLAG_BULK_DISPATCH (rows through the TMA unit) against the definition: buf[e, g, c] is the
+    token's row or zeros, bit for bit; invalid token indices count as empty slots."""
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    gen = torch.Generator(device="cuda").manual_seed(11)
+    x = torch.randn(G, S, M, device="cuda", generator=gen).to(tdt)
+    st = torch.randint(-1, S, (E, G, C), device="cuda", generator=gen, dtype=torch.int32)
+    st[0, 0, 0], st[-1, -1, -1] = S, -5                                          # out of range: treated as empty
+    shape = _shape(G, S, M, 64, E, C, dtype, B.GSHARD_FLAG_BULK_DISPATCH)
+    buf = torch.full((E, G * C, M), 3.0, device="cuda").to(tdt)
+    B.gshard_moe_dispatch(shape, x, st, buf)
+    valid = (st >= 0) & (st < S)
+    g_idx = torch.arange(G, device="cuda").view(1, G, 1).expand(E, G, C)
+    expect = torch.where(valid.unsqueeze(-1), x[g_idx, st.clamp(0, S - 1).long()], torch.zeros((), device="cuda", dtype=tdt))
+    assert torch.equal(buf.view(E, G, C, M), expect)
+
+
+@pytest.mark.parametrize("G,S,M,H,E,C,extra", [(4, 512, 1024, 256, 64, 4, 0),                      # single-launch FFN, 2 KB rows
+                                               (2, 256, 256, 512, 16, 40, 0),                      # CTA pairs
+                                               (2, 256, 256, 512, 16, 40, B.GSHARD_FLAG_SAVE_FOR_BACKWARD)])
+def test_forward_with_bulk_dispatch_has_the_same_bits(G, S, M, H, E, C, extra):
+    from paper_2006_16668_b200 import MoEConfig, make_inputs
+    cfg = MoEConfig("bulk", G=G, S=S, M=M, H=H, E=E, C=C, dtype="bf16", seed=31)
+    inp = make_inputs(cfg, "cuda")
+    ys = []
+    for flags in (extra, extra | B.GSHARD_FLAG_BULK_DISPATCH):
+        shape = B.make_shape(cfg, flags=flags)
+        ws = B.alloc_workspace(shape)
+        ctx = torch.empty(max(B.gshard_moe_top2_context_bytes(shape), 256), dtype=torch.uint8, device="cuda") if extra else None
+        y, l_aux = torch.empty_like(inp["x"]), torch.zeros(1, device="cuda")
+        B.gshard_moe_top2_forward(shape, inp["x"], inp["wg"], inp["wi"], inp["wo"], inp["u"], y, l_aux, None, ctx, ws)
+        assert B.gshard_moe_last_device_status(ws) == B.GSHARD_OK
+        ys.append((y, l_aux))
+    assert torch.equal(ys[0][0].view(torch.int16), ys[1][0].view(torch.int16)) and torch.equal(ys[0][1], ys[1][1])
