@@ -425,18 +425,26 @@ class Bench:
         ffn_bytes, ffn_flops = ffn_work(cfg.M, cfg.H, cfg.E, rows, es)
         fused = (cfg.dtype == "bf16" and not self.train and
                  (args.fused_ffn or (not args.unfused_ffn and rows <= 128)))
-        compact = (args.flags & 16384) or (rows >= 768 and not (args.one_sm_mma or args.two_sm_mma or args.fused_ffn
-                                                            or self.train))
-        pairs = rows > 128 and not args.one_sm_mma and not compact
+        other_form = bool(args.one_sm_mma or args.two_sm_mma or args.fused_ffn or (args.flags & (512 | 32 | 8)))
+        compact = (not self.train and cfg.dtype == "bf16" and not fused and
+                   bool((args.flags & 16384) or (rows > 128 and not other_form)))
+        one_sm = bool(args.one_sm_mma or (args.flags & 512))
+        pairs = rows > 128 and not one_sm
         if fused:
             kernel, label, n_launch = "ffn_group4_kernel", "expert FFN, both GEMMs in 1 launch", 1
         else:
             kernel = "umma2_gemm_kernel" if pairs else "umma_gemm_kernel"
             label, n_launch = "expert FFN, 2 grouped-GEMM launches (sum of both)", 2
-            if compact:
+            if compact and pairs:
+                kernel = "umma2_gemm_kernel + umma_gemm_kernel"
+                label = ("expert FFN over compacted slots, 2 grouped GEMMs of 2 launches each (sum of the four): kept "
+                         "rows in 256-row tiles on CTA pairs, the remaining 128-row tile on single CTAs")
+                n_launch = 4
+            elif compact:
                 label += ", compacted slots: only row tiles that hold kept rows"
         roof = kernel_roofline(ffn_bytes, ffn_flops, rec["ffn_ms"], peaks)
-        roof.update({"kernel": f"{kernel} ({label})", "launches_per_step": n_launch, "launch_ms": rec["ffn_ms"] / n_launch,
+        roof.update({"kernel": f"{kernel} ({label})", "launches_per_step": n_launch,
+                     "launch_ms": rec["ffn_ms"] / min(n_launch, 2),     # per GEMM where a GEMM takes two launches
                      "algorithmic_bytes": ffn_bytes, "algorithmic_flops": ffn_flops,
                      "ffn_tflops": ffn_flops / (rec["ffn_ms"] * 1e-3) / 1e12,
                      "ffn_gbs": ffn_bytes / (rec["ffn_ms"] * 1e-3) / 1e9,

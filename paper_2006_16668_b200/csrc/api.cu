@@ -122,11 +122,30 @@ int ffn_stage(const Dims& d, const void* buf, const void* wi, const void* wo, vo
   g2.a_kmajor = true; g2.b_kmajor = false;
   g2.a_ld = d.H; g2.a_bs = rows * d.H; g2.b_ld = d.M; g2.b_bs = (long long)d.H * d.M; g2.c_ld = d.M; g2.c_bs = rows * d.M;
   g2.b_stream = 1; g2.prefer_two_sm = 1;
-  if (tile_base) {
-    // compacted rows: each expert's row-tile count comes from the device-side prefix; 128-row tiles on
-    // single CTAs (a 256-row pair tile would round the kept rows up further)
-    g.tile_base = tile_base; g.prefer_two_sm = 0;
-    g2.tile_base = tile_base; g2.prefer_two_sm = 0;
+  // Compacted rows: each expert's row-tile count comes from the device-side prefixes.  Either 128-row
+  // tiles on single CTAs throughout, or (hybrid) the kept rows in 256-row tiles on CTA pairs and the one
+  // 128-row tile that may remain behind them on a single CTA, in a second launch of each GEMM.
+  const bool hybrid = tile_base && !d.one_sm_mma && d.rows > 128 && !(d.tf32_experts && wt);
+  const int* pair_base = tile_base ? tile_base + (d.E + 1) : nullptr;
+  const int* single_base = tile_base ? tile_base + 2 * (d.E + 1) : nullptr;
+  const int* owners = tile_base ? tile_base + 3 * (d.E + 1) : nullptr;      // three lists of compact_max_tiles(d)
+  const int max_tiles = compact_max_tiles(d);
+  if (tile_base && !hybrid) {
+    g.tile_base = tile_base; g.tile_problem = owners; g.prefer_two_sm = 0;
+    g2.tile_base = tile_base; g2.tile_problem = owners; g2.prefer_two_sm = 0;
+  }
+  if (hybrid) {
+    for (const UmmaGemm& whole : {g, g2}) {
+      UmmaGemm on_pairs = whole, rest = whole;
+      on_pairs.tile_base = pair_base; on_pairs.tile_problem = owners + max_tiles; on_pairs.ragged_on_pairs = 1;
+      rest.tile_base = single_base; rest.tile_problem = owners + 2 * max_tiles; rest.pair_base = pair_base;
+      rest.prefer_two_sm = 0;
+      if (run_gemm(d, on_pairs, status, st) != GSHARD_OK) {   // a refused cluster launch ran nothing
+        rest.tile_base = tile_base; rest.tile_problem = owners; rest.pair_base = nullptr;   // all tiles on single CTAs
+      }
+      GS_TRY(run_gemm(d, rest, status, st));
+    }
+    return GSHARD_OK;
   }
   if (d.tf32_experts && wt) {
     // The tensor core reads 32-bit operands K-major only, and the weights are contiguous along the

@@ -141,14 +141,15 @@ inline Dims make_dims(const gshard_moe_shape& s) {
   d.bulk_dispatch = (s.flags & GSHARD_FLAG_BULK_DISPATCH) != 0;
   d.debug_checks = (s.flags & GSHARD_FLAG_DEBUG_CHECKS) != 0;
   d.tf32_experts = !d.bf16 && (s.flags & GSHARD_FLAG_TF32_EXPERTS) != 0;
-  // Compacted slots: on request, and by default where an expert has at least six 128-row tiles, so
-  // that the usual 13-30 % of empty slots free at least one of them (measured at the MoE(128E) shape:
-  // 3.68 against 3.74 ms for a burst of steps, 4.08 against 4.62 ms sustained under the power cap; at
-  // 256 rows per expert nothing is saved and the CTA-pair GEMM is faster).  A flag that names
-  // another GEMM form switches the default off.
+  // Compacted slots: on request, and by default wherever the expert FFN runs as two grouped GEMMs (more
+  // than one 128-row tile per expert), so that the usual 13-30 % of empty slots free row tiles: the
+  // kept rows run in 256-row tiles on CTA pairs and the 128-row tile that may remain on a single CTA.
+  // Measured: MoE(128E) shape 3.44 against 3.79 ms per step for a burst, 3.88 against 4.11 ms sustained
+  // under the power cap; MoE(512E) shape (256 slots per expert, mostly still one pair tile) 3.92 against
+  // 4.00 ms and 4.26 against 4.36 ms.  A flag that names another GEMM form switches the default off.
   const bool other_form = (s.flags & (GSHARD_FLAG_ONE_SM_MMA | GSHARD_FLAG_TWO_SM_MMA | GSHARD_FLAG_FUSED_FFN)) != 0;
   d.compact_slots = d.bf16 && !d.simt && !(s.flags & GSHARD_FLAG_SAVE_FOR_BACKWARD) &&
-                    ((s.flags & GSHARD_FLAG_COMPACT_SLOTS) != 0 || (d.rows >= 768 && !other_form));
+                    ((s.flags & GSHARD_FLAG_COMPACT_SLOTS) != 0 || (d.rows > 128 && !other_form));
   return d;
 }
 

@@ -48,37 +48,58 @@ __global__ void __launch_bounds__(kCompactThreads) compact_kernel(const int32_t*
   if (threadIdx.x == 0) kept[e] = running;
 }
 
-// tile_base[e] = sum over e' < e of ceil(kept[e'] / 128), tile_base[E] = total (one CTA, in order).
-__global__ void __launch_bounds__(1024) tile_prefix_kernel(const int32_t* __restrict__ kept, int E,
+// Three exclusive prefixes over the experts (one CTA, in order), each with E + 1 entries, stored one
+// after the other in tile_base: [0] of t = ceil(kept / 128), the 128-row tiles of the single-CTA GEMM;
+// [1] of t / 2, the 256-row tiles a launch on CTA pairs covers; [2] of t mod 2, the one 128-row tile
+// that remains behind them.  Behind the prefixes, for each of the three lists, the expert that owns
+// every row tile (max_tiles entries per list).
+__global__ void __launch_bounds__(1024) tile_prefix_kernel(const int32_t* __restrict__ kept, int E, int max_tiles,
                                                            int32_t* __restrict__ tile_base) {
-  __shared__ int warp_sum[32];
-  __shared__ int running;
+  __shared__ int warp_sum[3][32];
+  __shared__ int running[3];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  if (threadIdx.x == 0) running = 0;
+  if (threadIdx.x < 3) running[threadIdx.x] = 0;
   __syncthreads();
   for (int e0 = 0; e0 < E; e0 += 1024) {
     const int e = e0 + threadIdx.x;
     const int tiles = e < E ? (kept[e] + 127) / 128 : 0;
-    int incl = tiles;
+    const int v[3] = {tiles, tiles / 2, tiles % 2};
+    int incl[3];
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const int v = __shfl_up_sync(0xffffffffu, incl, off);
-      if (lane >= off) incl += v;
+    for (int k = 0; k < 3; ++k) {
+      incl[k] = v[k];
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, incl[k], off);
+        if (lane >= off) incl[k] += u;
+      }
+      if (lane == 31) warp_sum[k][w] = incl[k];
     }
-    if (lane == 31) warp_sum[w] = incl;
     __syncthreads();
-    int before = running;
-    for (int i = 0; i < w; ++i) before += warp_sum[i];
-    if (e < E) tile_base[e] = before + incl - tiles;
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+      int before = running[k];
+      for (int i = 0; i < w; ++i) before += warp_sum[k][i];
+      if (e < E) tile_base[(size_t)k * (E + 1) + e] = before + incl[k] - v[k];
+    }
     __syncthreads();
-    if (threadIdx.x == 0) {
+    if (threadIdx.x < 3) {
       int add = 0;
-      for (int i = 0; i < 32; ++i) add += warp_sum[i];
-      running += add;
+      for (int i = 0; i < 32; ++i) add += warp_sum[threadIdx.x][i];
+      running[threadIdx.x] += add;
     }
     __syncthreads();
   }
-  if (threadIdx.x == 0) tile_base[E] = running;
+  if (threadIdx.x < 3) tile_base[(size_t)threadIdx.x * (E + 1) + E] = running[threadIdx.x];
+  // tile_problem lists behind the prefixes, max_tiles entries each: the expert that owns every row tile
+  __syncthreads();
+  int32_t* tile_problem = tile_base + 3 * (size_t)(E + 1);
+  for (int e = threadIdx.x; e < E; e += 1024)
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+      const int32_t* base = tile_base + (size_t)k * (E + 1);
+      for (int j = base[e]; j < base[e + 1]; ++j) tile_problem[(size_t)k * max_tiles + j] = e;
+    }
 }
 
 }  // namespace
@@ -86,7 +107,7 @@ __global__ void __launch_bounds__(1024) tile_prefix_kernel(const int32_t* __rest
 void launch_compact(const Dims& d, const int32_t* slot_token, int32_t* crow_token, int32_t* slot_crow, int32_t* kept,
                     int32_t* tile_base, cudaStream_t st) {
   compact_kernel<<<d.E, kCompactThreads, 0, st>>>(slot_token, d.rows, d.S, d.C, crow_token, slot_crow, kept);
-  tile_prefix_kernel<<<1, 1024, 0, st>>>(kept, d.E, tile_base);
+  tile_prefix_kernel<<<1, 1024, 0, st>>>(kept, d.E, compact_max_tiles(d), tile_base);
   count_launch(2);
 }
 

@@ -17,6 +17,7 @@ inline int run_gemm(const Dims& d, const UmmaGemm& g_in, int* status, cudaStream
     // forward expert GEMMs); the flags force either form everywhere.  A single row tile would leave
     // the second CTA of a pair without rows.
     if (g.tf32) return GSHARD_ERR_INTERNAL;   // bf16 operands cannot be read as TF32
+    if (g.tile_base && g.ragged_on_pairs) return launch_umma2_gemm(g, status, st);   // a ragged list of 256-row tiles
     if (g.rows > 128 && !g.tile_base && !d.one_sm_mma && (d.two_sm_mma || g.prefer_two_sm)) {
       const int rc = launch_umma2_gemm(g, status, st);
       if (rc == GSHARD_OK) return rc;       // a refused cluster launch ran nothing: single CTAs take over

@@ -50,7 +50,11 @@ void launch_combine(const Dims& d, const void* out, const int32_t* expert_idx, c
 // compact.cu: per expert, the filled slots in (group, position) order become rows 0 .. kept-1.
 //   crow_token [E, G*C]  global token index (g*S + s) of compacted row j, j < kept[e]
 //   slot_crow  [E, G*C]  compacted row of slot (g, c), or -1 for an empty slot
-//   kept [E], tile_base [E+1]: exclusive prefix of ceil(kept / 128)
+//   kept [E]; tile_base: three exclusive prefixes with E + 1 entries each (128-row tiles; 256-row
+//   tiles for CTA pairs; the 128-row tile left behind those), then for each list the expert that owns
+//   every row tile, compact_max_tiles(d) entries per list
+inline int compact_max_tiles(const Dims& d) { return d.E * ((d.rows + 127) / 128); }
+inline size_t compact_tile_ints(const Dims& d) { return 3 * ((size_t)d.E + 1) + 3 * (size_t)compact_max_tiles(d); }
 void launch_compact(const Dims& d, const int32_t* slot_token, int32_t* crow_token, int32_t* slot_crow, int32_t* kept,
                     int32_t* tile_base, cudaStream_t st);
 // buf[e, j, :] = x[crow_token[e, j], :] for j < kept[e]; other rows are left untouched
@@ -79,7 +83,13 @@ struct UmmaGemm {
   int tf32;                  // A and B hold float: contraction on the tensor cores in TF32 (both operands
                              // K-major, float output)
   const int* tile_base;      // ragged batch (device pointer, batch + 1 ints): problem b has
-                             // tile_base[b+1] - tile_base[b] row tiles of 128 rows; single-CTA kernel only
+                             // tile_base[b+1] - tile_base[b] row tiles (128 rows on single CTAs, 256 rows on
+                             // pairs)
+  const int* tile_problem;   // with tile_base: the problem that owns each row tile (tile_base[batch] ints)
+  const int* pair_base;      // single-CTA kernel with tile_base: problem b's row tiles start behind
+                             // 2 * (pair_base[b+1] - pair_base[b]) tiles of 128 rows, which a launch on CTA
+                             // pairs covers (same kind of prefix array)
+  int ragged_on_pairs;       // tile_base counts 256-row tiles: run on CTA pairs
   int plain_stores;          // epilogue writes C with 16-byte stores instead of bulk tensor (TMA) stores
   int max_ctas;              // > 0: use at most this many CTAs (persistent grid), leaving the other
                              // multiprocessors to a kernel running beside this one on another stream

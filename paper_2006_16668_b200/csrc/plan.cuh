@@ -49,7 +49,7 @@ inline FwdPlan plan_forward(const Dims& d) {
   p.crow_token = c.take(d.compact_slots ? R * 4 : 0);
   p.slot_crow = c.take(d.compact_slots ? R * 4 : 0);
   p.kept = c.take(d.compact_slots ? (size_t)d.E * 4 : 0);
-  p.tile_base = c.take(d.compact_slots ? ((size_t)d.E + 1) * 4 : 0);
+  p.tile_base = c.take(d.compact_slots ? compact_tile_ints(d) * 4 : 0);   // prefixes and tile owners (compact.cu)
   p.total = c.off;
   return p;
 }

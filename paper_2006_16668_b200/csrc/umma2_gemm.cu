@@ -55,16 +55,24 @@ struct Params2 {
   int n_fastest;
   int* status;
   int tma_store;   // epilogue rows leave by bulk tensor stores through map_c
+  // Ragged batches (compacted expert rows): problem b owns the 256-row tiles [tile_base[b], tile_base[b+1])
+  // of a device-side prefix array with batch + 1 entries; nullptr = every problem has m_tiles row tiles.
+  const int* tile_base;
+  const int* tile_problem;     // with tile_base: the problem that owns each row tile
 };
 
+// Tile index -> (row tile, column tile, problem).
+__device__ __forceinline__ int total_tiles_of(const Params2& p) {
+  return p.tile_base ? __ldg(p.tile_base + p.batch) * p.n_tiles : p.total_tiles;
+}
 __device__ __forceinline__ TileCoord decode(const Params2& p, int tile) {
+  if (p.tile_base) return decode_ragged(p, tile);
   TileCoord t;
   t.mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
   t.nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
   t.b = tile / (p.m_tiles * p.n_tiles);
   return t;
 }
-
 
 template <bool A_K, bool B_K, bool MASK>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -109,8 +117,11 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       const uint64_t pol_a = p.a_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
       const uint64_t pol_b = p.b_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
       int stage = 0; uint32_t phase = 0;
-      for (int tile = pair; tile < p.total_tiles && ok; tile += n_pairs) {
-        const TileCoord t = decode(p, tile);
+      const int total_tiles = total_tiles_of(p);
+      TileCoord tn = pair < total_tiles ? decode(p, pair) : TileCoord{};
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+        const TileCoord t = tn;
+        if (tile + n_pairs < total_tiles) tn = decode(p, tile + n_pairs);   // the next tile's coordinates load meanwhile
         const int row0 = t.mt * 2 * BM + (int)rank * BM;      // this CTA's 128 rows of the 256-row tile
         const int col0 = t.nt * BN + (int)rank * BNH;         // this CTA's half of the B columns
         for (int kb = 0; kb < p.k_blocks; ++kb) {
@@ -143,7 +154,8 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
       constexpr uint32_t idesc = ptx::make_idesc_bf16(2 * BM, BN, !A_K, !B_K);
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
-      for (int tile = pair; tile < p.total_tiles && ok; tile += n_pairs) {
+      const int total_tiles = total_tiles_of(p);
+      for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
         if (!ptx::mbar_wait(acc_empty + acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
@@ -175,8 +187,11 @@ umma2_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const int half = ew >> 2;
     unsigned char* stg = smem + kStgOff + ew * kStgWarpBytes;
     int acc = 0; uint32_t acc_phase = 0;
-    for (int tile = pair; tile < p.total_tiles && ok; tile += n_pairs) {
-      const TileCoord t = decode(p, tile);
+    const int total_tiles = total_tiles_of(p);
+    TileCoord tn = pair < total_tiles ? decode(p, pair) : TileCoord{};
+    for (int tile = pair; tile < total_tiles && ok; tile += n_pairs) {
+      const TileCoord t = tn;
+      if (tile + n_pairs < total_tiles) tn = decode(p, tile + n_pairs);
       const int tile_row0 = t.mt * 2 * BM + (int)rank * BM;     // this CTA's 128 rows of the 256-row tile
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
@@ -256,10 +271,14 @@ int launch_umma2_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   p.out_f32 = g.out_f32; p.relu = g.relu; p.a_stream = g.a_stream; p.b_stream = g.b_stream;
   p.n_fastest = (g.rows > g.cols) ? 1 : 0;
   p.status = status;
+  p.tile_base = g.ragged_on_pairs ? g.tile_base : nullptr;
+  p.tile_problem = g.tile_problem;
+  if (p.tile_base && !p.tile_problem) return GSHARD_ERR_INTERNAL;
+  if (p.tile_base) p.n_fastest = 0;            // ragged lists are walked with the row tiles fastest
   const int sms = device_sms();
   int pairs = sms / 2;
   if (g.max_ctas > 0 && pairs > g.max_ctas / 2) pairs = g.max_ctas / 2 > 0 ? g.max_ctas / 2 : 1;
-  if (pairs > p.total_tiles) pairs = p.total_tiles;
+  if (pairs > p.total_tiles && !p.tile_base) pairs = p.total_tiles;   // ragged: count known on the device only
 #define GSHARD_DISPATCH2(AK, BKM) \
   (p.mask_bits ? launch2_t<AK, BKM, true>(ma, mb, mc, p, pairs, st) : launch2_t<AK, BKM, false>(ma, mb, mc, p, pairs, st))
   if (g.a_kmajor && g.b_kmajor) return GSHARD_DISPATCH2(true, true);

@@ -14,6 +14,22 @@ constexpr int kStgWarpBytes = 32 * kStgRowBytes;
 
 struct TileCoord { int mt, nt, b; };
 
+// Ragged batches (compacted expert rows).  Problem b owns the row tiles [tile_base[b], tile_base[b+1]) of
+// a device-side prefix array with batch + 1 entries, and tile_problem[r] names the problem that owns
+// row tile r, so a tile index is decoded with three loads and no search; the callers decode the NEXT
+// tile before they work on the current one, which hides those loads.  Within a problem the row tiles
+// run fastest: they share the B tile.
+template <typename P>
+__device__ __forceinline__ TileCoord decode_ragged(const P& p, int tile) {
+  TileCoord t;
+  t.b = __ldg(p.tile_problem + tile / p.n_tiles);
+  const int first = __ldg(p.tile_base + t.b);
+  const int m_b = __ldg(p.tile_base + t.b + 1) - first;
+  const int i = tile - first * p.n_tiles;
+  t.mt = i % m_b; t.nt = i / m_b;
+  return t;
+}
+
 // Writes a warp's staged 32 rows x 128 bytes to C: lane l handles 16-byte piece (l & 7) of rows
 // 4*i + (l >> 3); pieces beyond the matrix edge are skipped (cols is a multiple of the piece width).
 // Whether the output rows should be kept in L2 (they are re-read soon by the same launch).  A kernel

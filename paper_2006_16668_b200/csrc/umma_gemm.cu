@@ -59,33 +59,29 @@ struct Params {
   // Ragged batches (compacted expert rows): problem b owns the row tiles [tile_base[b], tile_base[b+1])
   // of a device-side prefix array with batch + 1 entries; nullptr = every problem has m_tiles row tiles.
   const int* tile_base;
+  const int* tile_problem;     // with tile_base: the problem that owns each row tile
+  // with tile_base: problem b's tiles start behind the 2 * (pair_base[b+1] - pair_base[b]) row tiles that
+  // a launch on CTA pairs covers; nullptr = they start at row 0
+  const int* pair_base;
   int tma_store;   // epilogue rows leave by bulk tensor stores through map_c
 };
 
-// Tile index -> (row tile, column tile, problem).  A thread walks its tiles in increasing order, so
-// for ragged batches it keeps the problem index of its last tile and moves forward from there
-// instead of searching the prefix array.
-struct TileWalk {
-  int b = 0;
-  __device__ __forceinline__ int total(const Params& p) const {
-    return p.tile_base ? __ldg(p.tile_base + p.batch) * p.n_tiles : p.total_tiles;
-  }
-  __device__ __forceinline__ TileCoord decode(const Params& p, int tile) {
-    TileCoord t;
-    if (p.tile_base) {
-      while (b + 1 < p.batch && __ldg(p.tile_base + b + 1) * p.n_tiles <= tile) ++b;
-      const int first = __ldg(p.tile_base + b);
-      const int m_b = __ldg(p.tile_base + b + 1) - first;           // row tiles of this problem (>= 1 here)
-      const int i = tile - first * p.n_tiles;
-      t.mt = i % m_b; t.nt = i / m_b; t.b = b;                      // row tiles fastest: they share the B tile
-      return t;
-    }
-    t.mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
-    t.nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
-    t.b = tile / (p.m_tiles * p.n_tiles);
+// Tile index -> (row tile, column tile, problem).
+__device__ __forceinline__ int total_tiles_of(const Params& p) {
+  return p.tile_base ? __ldg(p.tile_base + p.batch) * p.n_tiles : p.total_tiles;
+}
+__device__ __forceinline__ TileCoord decode(const Params& p, int tile) {
+  if (p.tile_base) {
+    TileCoord t = decode_ragged(p, tile);
+    if (p.pair_base) t.mt += 2 * (__ldg(p.pair_base + t.b + 1) - __ldg(p.pair_base + t.b));
     return t;
   }
-};
+  TileCoord t;
+  t.mt = p.n_fastest ? (tile / p.n_tiles) % p.m_tiles : tile % p.m_tiles;
+  t.nt = p.n_fastest ? tile % p.n_tiles : (tile / p.m_tiles) % p.n_tiles;
+  t.b = tile / (p.m_tiles * p.n_tiles);
+  return t;
+}
 
 // TF32: A and B hold fp32 values that the tensor core reads as TF32 (K-major operands only: with a
 // 32-bit MN-major operand the instruction returns zeros).  A shared-memory row is still 128 bytes,
@@ -136,28 +132,29 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       const uint64_t pol_a = p.a_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
       const uint64_t pol_b = p.b_stream ? ptx::policy_evict_first() : ptx::policy_evict_last();
       int stage = 0; uint32_t phase = 0;
-      TileWalk walk;
-      const int total_tiles = walk.total(p);
+      const int total_tiles = total_tiles_of(p);
+      TileCoord t = (int)blockIdx.x < total_tiles ? decode(p, blockIdx.x) : TileCoord{};
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-        const TileCoord t = walk.decode(p, tile);
+        const TileCoord cur = t;
+        if (tile + (int)gridDim.x < total_tiles) t = decode(p, tile + gridDim.x);   // the next tile's coordinates load meanwhile
         for (int kb = 0; kb < p.k_blocks; ++kb) {
           if (!ptx::mbar_wait(empty + stage, phase ^ 1u, abort_flag)) { ok = false; break; }
           unsigned char* sa = smem + stage * C_::stage_bytes;
           unsigned char* sb = sa + kABytes;
           ptx::mbar_arrive_expect_tx(full + stage, (uint32_t)C_::stage_bytes);
           if (A_K) {
-            ptx::tma_load_3d(sa, &map_a, full + stage, kb * BKE, t.mt * BM, t.b, pol_a);
+            ptx::tma_load_3d(sa, &map_a, full + stage, kb * BKE, cur.mt * BM, cur.b, pol_a);
           } else {
 #pragma unroll
             for (int j = 0; j < BM / kBoxMN; ++j)
-              ptx::tma_load_3d(sa + j * kBoxB, &map_a, full + stage, t.mt * BM + j * kBoxMN, kb * BKE, t.b, pol_a);
+              ptx::tma_load_3d(sa + j * kBoxB, &map_a, full + stage, cur.mt * BM + j * kBoxMN, kb * BKE, cur.b, pol_a);
           }
           if (B_K) {
-            ptx::tma_load_3d(sb, &map_b, full + stage, kb * BKE, t.nt * BN, t.b, pol_b);
+            ptx::tma_load_3d(sb, &map_b, full + stage, kb * BKE, cur.nt * BN, cur.b, pol_b);
           } else {
 #pragma unroll
             for (int j = 0; j < BN / kBoxMN; ++j)
-              ptx::tma_load_3d(sb + j * kBoxB, &map_b, full + stage, t.nt * BN + j * kBoxMN, kb * BKE, t.b, pol_b);
+              ptx::tma_load_3d(sb + j * kBoxB, &map_b, full + stage, cur.nt * BN + j * kBoxMN, kb * BKE, cur.b, pol_b);
           }
           if (++stage == C_::stages) { stage = 0; phase ^= 1u; }
         }
@@ -169,7 +166,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
       constexpr uint32_t idesc = TF32 ? ptx::make_idesc_tf32(BM, BN, !A_K, !B_K) : ptx::make_idesc_bf16(BM, BN, !A_K, !B_K);
       int stage = 0; uint32_t phase = 0;
       int acc = 0; uint32_t acc_phase = 0;
-      const int total_tiles = TileWalk().total(p);
+      const int total_tiles = total_tiles_of(p);
       for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
         if (!ptx::mbar_wait(acc_empty + acc, acc_phase ^ 1u, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after_sync();
@@ -203,10 +200,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int half = ew >> 2;                        // which half of the tile's columns
     unsigned char* stg = smem + C_::stg_off + ew * kStgWarpBytes;
     int acc = 0; uint32_t acc_phase = 0;
-    TileWalk walk;
-    const int total_tiles = walk.total(p);
+    const int total_tiles = total_tiles_of(p);
+    TileCoord tn = (int)blockIdx.x < total_tiles ? decode(p, blockIdx.x) : TileCoord{};
     for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-      const TileCoord t = walk.decode(p, tile);
+      const TileCoord t = tn;
+      if (tile + (int)gridDim.x < total_tiles) tn = decode(p, tile + gridDim.x);
       if (!ptx::mbar_wait_warp(acc_full + acc, acc_phase, abort_flag, lane)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       epilogue_tile<BN, MASK>(p, p.tma_store ? &map_c : nullptr, t, t.mt * BM, tmem_base + (uint32_t)(acc * BN), q, half,
@@ -444,6 +442,9 @@ int launch_umma_gemm(const UmmaGemm& g, int* status, cudaStream_t st) {
   p.n_fastest = (g.rows > g.cols) ? 1 : 0;
   p.status = status;
   p.tile_base = g.tile_base;
+  p.pair_base = g.tile_base ? g.pair_base : nullptr;
+  p.tile_problem = g.tile_problem;
+  if (g.tile_base && !g.tile_problem) return GSHARD_ERR_INTERNAL;
   if (g.tile_base && g.tf32) return GSHARD_ERR_INTERNAL;
   if (g.tile_base) p.n_fastest = 0;            // ragged lists are walked with the row tiles fastest
   int sms = device_sms();
