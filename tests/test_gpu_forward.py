@@ -298,3 +298,39 @@ def test_full_size_sampled(name, groups, tokens):
     y2, l_aux2, rt2 = run_forward(cfg, inp)
     assert torch.equal(y.view(torch.int16), y2.view(torch.int16)) and torch.equal(l_aux, l_aux2)
     assert torch.equal(rt["slot"], rt2["slot"]) and torch.equal(rt["m"], rt2["m"])
+
+
+def test_compact_slots_tile_edges():
+    """Compacted slots with prescribed kept-row counts per expert at the edges of the tile lists: 0, 1,
+    128, 129 (one single tile / one pair tile), 255, 256, 257 (one pair tile + one single tile), 384,
+    385, 512 (= all slots).  The routing is forced through the inputs: token t carries two large
+    features a_t != b_t, wg is the identity on the first E features, so the token picks experts a_t and
+    b_t with g1 = g2 and keeps both (u = 0.5, capacity = the largest count).  The result must have the
+    bits of the uncompacted single-CTA form, and match the oracle on sampled tokens."""
+    E, M, H, C = 16, 64, 128, 512
+    counts = [0, 1, 128, 129, 255, 256, 257, 384, 385, 512, 3, 130, 258, 386, 64, 448]
+    assert len(counts) == E and sum(counts) % 2 == 0 and max(counts) <= C
+    ends = [e for e, n in enumerate(counts) for _ in range(n)]
+    S = len(ends) // 2
+    assert max(counts) <= S                                   # so that ends[i] != ends[i + S]
+    a, b = torch.tensor(ends[:S]), torch.tensor(ends[S:])
+    assert bool((a != b).all())
+    perm = torch.randperm(S, generator=torch.Generator().manual_seed(3))
+    a, b = a[perm], b[perm]
+    x = torch.randn(1, S, M, generator=torch.Generator().manual_seed(4)) * 0.05
+    x[0, :, :E] = 0.0
+    x[0, torch.arange(S), a] = 10.0
+    x[0, torch.arange(S), b] = 10.0
+    wg = torch.zeros(M, E)
+    wg[torch.arange(E), torch.arange(E)] = 1.0
+    cfg = MoEConfig("edges", G=1, S=S, M=M, H=H, E=E, C=C, dtype="bf16", seed=17)
+    inp = make_inputs(cfg, "cuda")
+    inp["x"], inp["wg"] = x.bfloat16().cuda(), wg.bfloat16().cuda()
+    inp["u"] = torch.full((1, S), 0.5, device="cuda")
+    y_c, l_c, rt_c = run_forward(cfg, inp, B.GSHARD_FLAG_COMPACT_SLOTS)
+    assert rt_c["total_count"][0].tolist() == counts          # the prescribed kept rows per expert
+    y_b, l_b, rt_b = run_forward(cfg, inp, B.GSHARD_FLAG_ONE_SM_MMA)
+    assert torch.equal(y_b.view(torch.int16), y_c.view(torch.int16)) and torch.equal(l_b, l_c)
+    y_s, _, _ = run_forward(cfg, inp, B.GSHARD_FLAG_COMPACT_SLOTS | B.GSHARD_FLAG_ONE_SM_MMA)   # single-CTA ragged list
+    assert torch.equal(y_b.view(torch.int16), y_s.view(torch.int16))
+    check_forward(cfg, inp, y_c, l_c, rt_c, [0], 24)
