@@ -127,16 +127,18 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
 #define GSHARD_FLAG_COMPACT_SLOTS 16384u      /* forward, bf16, grouped-GEMM form of the expert FFN
                                                  (more than 128 rows per expert): the filled slots of
                                                  each expert are compacted to the front of its block,
-                                                 the GEMMs run only the 128-row tiles that hold kept
-                                                 rows (13 to 30 % of the slots are empty at the
-                                                 paper's shapes), empty rows are neither zero-filled
+                                                 the GEMMs run only the row tiles that hold kept rows
+                                                 (13 to 30 % of the slots are empty at the paper's
+                                                 shapes: 256-row tiles on CTA pairs, then at most one
+                                                 128-row tile on a single CTA; with ONE_SM_MMA 128-row
+                                                 tiles throughout), empty rows are neither zero-filled
                                                  nor multiplied, and the combine finds its rows through
                                                  the compaction index.  Kept rows get the same bits.
-                                                 This is already the default where an expert has 768
-                                                 rows or more (unless ONE_SM_MMA, TWO_SM_MMA or FUSED_FFN
-                                                 names another form); the flag extends it
-                                                 to fewer rows.  Ignored with SAVE_FOR_BACKWARD and
-                                                 where the single-launch FFN runs */
+                                                 This is the default for that form of the FFN unless
+                                                 ONE_SM_MMA, TWO_SM_MMA or FUSED_FFN names another;
+                                                 the flag then adds it back.  Ignored with
+                                                 SAVE_FOR_BACKWARD and where the single-launch FFN
+                                                 runs */
 #define GSHARD_FLAG_DEBUG_CHECKS 32768u       /* forward: after the capacity stage a kernel verifies the
                                                  routing tensors (expert ids, positions, flags, weights,
                                                  the inverse slot list; every access bounds-checked) and
