@@ -147,7 +147,10 @@ typedef enum { GSHARD_F32 = 0, GSHARD_BF16 = 1 } gshard_dtype;
 #define GSHARD_FLAG_BULK_DISPATCH 65536u      /* dispatch: token rows move through the TMA unit (bulk
                                                  global->shared->global copies, empty slots as bulk
                                                  stores of a zero row) instead of 16-byte loads and
-                                                 stores; same bytes */
+                                                 stores; same bytes.  Applies to the dispatch into the
+                                                 full [E, G*C, M] buffer (gshard_moe_dispatch, the
+                                                 single-launch FFN, SAVE_FOR_BACKWARD), not to the
+                                                 dispatch into compacted rows */
 #define GSHARD_FLAG_ALL 131071u
 
 /* G groups of S tokens, model dim M, expert hidden dim H, E experts, per-group capacity C
