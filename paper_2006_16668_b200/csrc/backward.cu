@@ -365,6 +365,13 @@ int backward_expert_stage(const Dims& d, const void* dout, const void* h, const 
   // On request each read-heavy GEMM shares the GPU with a write-heavy one (half of the multiprocessors
   // each, two streams).  Measured at the MoE(512E) training shape this is slower than running the four
   // one after another on all multiprocessors, so it is not the default.
+  // dwo has 64 row tiles per column block at the paper's shapes: on CTA pairs each CTA keeps half of the
+  // resident B slice and an A ring of two row tiles instead of one.  Isolated launches at the MoE(512E)
+  // training shape: 2.15 against 2.43 ms.  dwi has only eight row tiles per column block; its pair form
+  // (two B slices, so that the next one loads during the current block) measures 2.28 against 2.32 ms
+  // and stays off.  Under the power cap the training step takes the same time either way (fewer
+  // cycles at a lower clock).
+  g_dwo.prefer_two_sm = d.H >= 16 * 128;
   const int share = d.bwd_paired ? (device_sms() / 2) & ~1 : 0;
   int rc = run_gemm_pair(d, g_dh, g_dwo, share, status, st);
   if (rc) return rc;

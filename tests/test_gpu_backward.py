@@ -62,6 +62,10 @@ BWD_CASES = [
     # full four k-blocks
     ("bf16_wgrad_resident_ragged", 2, 256, 512, 640, 16, 40, "bf16", 0, GRAD_TOL),
     ("bf16_wgrad_resident_k256", 2, 1024, 512, 512, 16, 128, "bf16", 0, GRAD_TOL),
+    # dwo on CTA pairs with the deep A ring (sixteen 256-row tiles per column block), dwi on single CTAs
+    ("bf16_wgrad_pairs_deep_ring", 2, 512, 256, 4096, 16, 64, "bf16", 0, GRAD_TOL),
+    # every weight gradient on pairs: few row tiles per column block, two resident B slices in turn
+    ("bf16_wgrad_pairs_two_slices", 2, 1024, 512, 1024, 16, 128, "bf16", B.GSHARD_FLAG_TWO_SM_MMA, GRAD_TOL),
     # dh beside dwo and dbuf beside dwi, half of the multiprocessors each
     ("bf16_paired_gemms", 2, 1024, 512, 512, 16, 128, "bf16", B.GSHARD_FLAG_BWD_PAIRED_GEMMS, GRAD_TOL),
 ]
