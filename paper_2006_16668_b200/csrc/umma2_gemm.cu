@@ -17,6 +17,11 @@
 //     barriers order barrier initialisation before, and teardown after, all cross-CTA traffic.
 // Every mbarrier wait is bounded in wall time and reports GSHARD_ERR_TIMEOUT; a CTA that gave up
 // still reaches the final cluster barrier, so its peer is not left waiting.
+//
+// Two kernels: umma2_gemm_kernel, the general one (tile list regular or ragged - compacted expert
+// rows -, ReLU / mask epilogues), and umma2_gemm_resident_b_kernel for the weight gradients, whose
+// contraction is an expert's rows (at most 256): a pair keeps a 256-column slice of B resident and walks
+// the row tiles of that column block.
 #include <cuda.h>
 
 #include "kernels.cuh"
